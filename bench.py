@@ -1,0 +1,463 @@
+#!/usr/bin/env python
+"""Benchmark of the paged-KV pack/unpack hot path on B200.
+
+One step = one pass of the hot path over one request of the workload:
+  block table -> chunk mapper -> ONE pack launch (gather the prefix into contiguous
+  chunks in a staging area) -> ONE unpack launch (scatter the chunks into a second,
+  independently drawn set of pool blocks).
+Default workload: Llama-3.1-8B KV shape (32 layers, 8 KV heads, head dim 128, 16-token
+blocks, 2-byte elements), one 80,000-token prefix = 5000 blocks scattered over a
+20,000-block pool (39 GiB), 256-token chunks.  All inputs are synthetic and seeded.
+
+`value` counts bytes read + bytes written by pack and unpack, with everything resident in
+HBM.  `e2e` is the same byte count when the prefix is offloaded to pinned HOST memory and
+loaded back through the bounded staging ring (device->host and host->device copies inside
+the timed region).  `cpu_baseline` is the CPU oracle timed on a bounded sample.
+
+  python bench.py [--gpus N --steps K --warmup W] [--impl reference]
+For N > 1 launch under torch.distributed.run; every rank runs an independent replica
+(the path needs no exchange between GPUs).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+METRIC = "pack+unpack GB/s (bytes read+written), 80k-token prefix, 8B KV shape"
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0]))
+                    mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for nm, v in zip(names, p[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(nm)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ------------------------------------------------------------------ CPU oracle timing
+class OracleSample:
+    """The CPU oracle (as it stands) on a bounded sample of the workload: `chunks_per_pass`
+    chunks of the same KV geometry over a host pool that holds only as many blocks as the sample
+    needs, pack then unpack, repeated until about `target_seconds` of work is done.  The work is
+    split over (layer, K|V) ranges across all usable cores."""
+
+    def __init__(self, shape: wl.KVShape, chunk_tokens: int, seed: int):
+        from oracle import oracle as orc
+        self.orc = orc
+        self.chunk_tokens = chunk_tokens
+        self.bpc = bpc = chunk_tokens // shape.B
+        budget_blocks = max(2 * bpc, (1 << 30) // shape.bytes_per_block)   # about 1 GiB of pool
+        self.chunks_per_pass = max(1, budget_blocks // 2 // bpc)
+        self.pool_blocks = 2 * self.chunks_per_pass * bpc
+        self.g = g = orc.Dims(shape.L, shape.P, self.pool_blocks, shape.B, shape.H, shape.D, shape.e)
+        self.pool = wl.random_bits(seed, g.pool_bytes)
+        self.src = wl.block_ids(seed + 1, self.pool_blocks, self.chunks_per_pass * bpc)
+        self.dst = wl.block_ids(seed + 2, self.pool_blocks, self.chunks_per_pass * bpc)
+        cores = len(os.sched_getaffinity(0))
+        lp_total = g.L * g.P
+        self.nthreads = max(1, min(cores, lp_total))
+        cuts = np.linspace(0, lp_total, self.nthreads + 1).astype(int)
+        self.ranges = [(int(a), int(b)) for a, b in zip(cuts[:-1], cuts[1:]) if b > a]
+        self.cb = orc.chunk_bytes(g, bpc)
+        self.bufs = [np.zeros(self.cb, dtype=np.uint8) for _ in range(self.chunks_per_pass)]
+
+    def _pass(self, n_chunks):
+        orc, g, bpc = self.orc, self.g, self.bpc
+        t0 = time.perf_counter()
+        with ThreadPoolExecutor(self.nthreads) as ex:
+            futs = [ex.submit(orc.pack_chunk_into, g, self.pool, self.src[c * bpc:(c + 1) * bpc],
+                              self.bufs[c], r) for c in range(n_chunks) for r in self.ranges]
+            for f in futs:
+                f.result()
+            t1 = time.perf_counter()
+            futs = [ex.submit(orc.unpack_chunk, g, self.pool, self.bufs[c],
+                              self.dst[c * bpc:(c + 1) * bpc], r)
+                    for c in range(n_chunks) for r in self.ranges]
+            for f in futs:
+                f.result()
+        return t1 - t0, time.perf_counter() - t1
+
+    def run(self, target_seconds: float):
+        p1, u1 = self._pass(1)
+        want = max(1, round(target_seconds / max(p1 + u1, 1e-6)))
+        tp = tu = 0.0
+        done = 0
+        while done < want:
+            k = min(self.chunks_per_pass, want - done)
+            a, b = self._pass(k)
+            tp, tu, done = tp + a, tu + b, done + k
+        moved = 2 * done * self.cb  # bytes read + written, per direction
+        return {
+            "value": 2 * moved / (tp + tu) / 1e9, "unit": "GB/s", "cores": self.nthreads,
+            "kind": "oracle",
+            "sample": "%d chunks of %d tokens (%d MiB each way in total) of the same KV shape, pack "
+                      "then unpack, host pool of %d blocks" % (done, self.chunk_tokens,
+                                                               done * self.cb >> 20, self.pool_blocks),
+            "pack_gbs": moved / tp / 1e9, "unpack_gbs": moved / tu / 1e9, "seconds": tp + tu,
+            "ms_per_80k_prefix_unpack_extrapolated": tu / done * (80000 / self.chunk_tokens) * 1e3,
+        }
+
+
+def run_reference(args, rank):
+    """Reference arm: the CPU oracle on the host cores, one bounded sample per step."""
+    if rank != 0:
+        return
+    w = wl.WORKLOADS[args.workload]
+    per_step = 4.0
+    vals, last = [], None
+    sample = OracleSample(w.shape, args.chunk_tokens, w.seed + 100)
+    for i in range(args.warmup + args.steps):
+        r = sample.run(per_step)
+        if i >= args.warmup:
+            vals.append(r)
+        last = r
+    total_s = sum(v["seconds"] for v in vals)
+    value = statistics.mean(v["value"] for v in vals)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_s / len(vals) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "chunk_tokens": args.chunk_tokens,
+                   "note": "CPU oracle on a bounded sample of the workload per step"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": last["cores"], "kind": "oracle",
+                         "sample": last["sample"]},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------ GPU arm
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_11744_b200 import cuda_rt, kvc
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    kvc.lib()  # fail loudly if the extension is missing
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    w = wl.WORKLOADS[args.workload]
+    s = w.shape
+    NB, n = w.pool_blocks, w.request_blocks
+    one_way = n * s.bytes_per_block
+    pool = wl.random_bits_cuda(w.seed + 17 * rank, NB * s.bytes_per_block, dev)
+    src = wl.block_ids(w.seed, NB, n)
+    dst = wl.block_ids(w.dst_seed, NB, n)
+    staging = torch.empty(one_way, dtype=torch.uint8, device=dev)
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, args.chunk_tokens)
+    kvc.kvc_layout_set_tuning(lay, variant=args.variant, order=args.order,
+                              tile_bytes=args.tile_bytes, stages=args.stages)
+    stream = torch.cuda.current_stream()
+
+    def step(evs=None):
+        ops, keep, nbytes, on_dev = kvc.request_chunk_ops(lay, src, staging)
+        if evs:
+            evs[0].record(stream)
+        kvc.kvc_pack_batch(lay, ops, on_dev)
+        if evs:
+            evs[1].record(stream)
+        ops2, keep2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+        kvc.kvc_unpack_batch(lay, ops2, on_dev)
+        if evs:
+            evs[2].record(stream)
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = kvc.kvc_layout_launch_count(lay)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(evs[i])
+    barrier()
+    wall = time.perf_counter() - t0
+    launches = kvc.kvc_layout_launch_count(lay) - launches0
+    clocks = sampler.stop()
+    total_ms = evs[0][0].elapsed_time(evs[-1][2])
+    pack_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    unpack_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    skipped, expired = kvc.kvc_poll_device_status(lay)
+    assert (skipped, expired) == (0, 0), "device status flags set: %r" % ((skipped, expired),)
+
+    # spot check of the timed configuration: staging holds pack(src) at sampled positions
+    check_sampled(torch, pool, staging, src, dst, s, NB, args.chunk_tokens, dev)
+
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    bytes_step = 4 * one_way  # pack: read+write; unpack: read+write
+    value = world * bytes_step * args.steps / (total_ms * 1e-3) / 1e9
+
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, dist)
+    peak, peak_kind = measured_peak()
+    launch_ms = statistics.mean(pack_ms + unpack_ms)
+    achieved = 2 * one_way / (launch_ms * 1e-3) / 1e9
+    roof = {
+        "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+        "traffic": args.traffic_bytes, "peak_kind": peak_kind,
+        "kernel": "kvc_bulk_kernel (pack and unpack instantiations)" if args.variant != 1
+                  else "kvc_vec_kernel (pack and unpack instantiations)",
+        "algorithmic_bytes_per_launch": 2 * one_way,
+        "avg_launch_ms": launch_ms,
+        "pack": {"ms": statistics.mean(pack_ms), "min_ms": min(pack_ms),
+                 "gbs": 2 * one_way / statistics.mean(pack_ms) / 1e6,
+                 "frac": 2 * one_way / statistics.mean(pack_ms) / 1e6 / peak},
+        "unpack": {"ms": statistics.mean(unpack_ms), "min_ms": min(unpack_ms),
+                   "gbs": 2 * one_way / statistics.mean(unpack_ms) / 1e6,
+                   "frac": 2 * one_way / statistics.mean(unpack_ms) / 1e6 / peak},
+        "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+    }
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cpu = OracleSample(s, args.chunk_tokens, w.seed + 50).run(12.0)
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": {"workload": args.workload, "kv_shape": "L32 H8 D128 B16 2-byte", "pool_blocks": NB,
+                   "request_tokens": w.request_tokens, "request_blocks": n,
+                   "chunk_tokens": args.chunk_tokens, "bytes_each_way": one_way,
+                   "launch": "one kvc_pack_batch + one kvc_unpack_batch per step",
+                   "l2": "inputs larger than L2 (9.8 GiB read and 9.8 GiB written per launch)",
+                   "parallelism": "replicas only" if world > 1 else "1 GPU"},
+        "ms_to_load_80k_prefix": statistics.mean(unpack_ms),
+        "pack_gbs": roof["pack"]["gbs"], "unpack_gbs": roof["unpack"]["gbs"],
+        "wall_ms_per_step": wall / args.steps * 1e3,
+        "clocks": clocks, "gpu_launches": int(launches), "roofline": roof,
+    }
+    if e2e:
+        line["e2e"] = e2e
+    if cpu:
+        line["cpu_baseline"] = cpu
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def check_sampled(torch, pool, staging, src, dst, s, NB, chunk_tokens, dev, n_samples=200_000):
+    """After the timed steps the staging area holds pack(src) (the later unpack into dst does not
+    change it) and the pool's dst blocks hold those bytes: compare sampled 2-byte elements with
+    positions computed by the CPU oracle's index formulas, one sample at a time (vectorised)."""
+    from oracle import oracle as orc
+    g = orc.Dims(s.L, s.P, NB, s.B, s.H, s.D, s.e)
+    bpc = chunk_tokens // s.B
+    n = len(src)
+    rng = np.random.default_rng(12345)
+    blk = rng.integers(0, n, n_samples)           # table position of the sampled block
+    c = blk // bpc
+    j = blk - c * bpc
+    nb_c = np.minimum(bpc, n - c * bpc)
+    l = rng.integers(0, s.L, n_samples)
+    p = rng.integers(0, s.P, n_samples)
+    t = rng.integers(0, s.B, n_samples)
+    h = rng.integers(0, s.H, n_samples)
+    d = rng.integers(0, s.D, n_samples)
+    chunk_base = c.astype(np.int64) * (orc.chunk_bytes(g, bpc) // s.e)   # chunks lie back to back
+    stage_idx = chunk_base + orc.chunk_elem(g, nb_c, l, p, j, t, h, d)
+    src_idx = orc.pool_elem(g, l, p, src[blk].astype(np.int64), t, h, d)
+    dst_idx = orc.pool_elem(g, l, p, dst[blk].astype(np.int64), t, h, d)
+    pool16, stage16 = pool.view(torch.int16), staging.view(torch.int16)
+    sv = stage16[torch.from_numpy(stage_idx).to(dev)]
+    dv = pool16[torch.from_numpy(dst_idx).to(dev)]
+    assert bool((sv == dv).all()), "unpack: sampled pool elements differ from the staged chunk"
+    # source blocks overwritten by the unpack (src and dst tables overlap) can no longer be compared
+    keep = ~np.isin(src[blk], dst)
+    pv = pool16[torch.from_numpy(src_idx[keep]).to(dev)]
+    assert bool((sv[torch.from_numpy(np.flatnonzero(keep)).to(dev)] == pv).all()), \
+        "pack: sampled staged elements differ from the pool"
+
+
+def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, dist):
+    """Offload the prefix to pinned host memory and load it back, chunk by chunk through a
+    bounded ring of device staging slots (pack -> slot -> D2H; H2D -> slot -> unpack)."""
+    descs = kvc.kvc_map_request(lay, len(src))
+    cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+    slot_bytes = (cb + 4095) // 4096 * 4096
+    ring = kvc.kvc_staging_ring_create(slot_bytes, args.ring_slots, kvc.KVC_RING_DEVICE)
+    host = torch.empty(one_way, dtype=torch.uint8, pin_memory=True)
+    hptr = host.data_ptr()
+    s_k, s_c = torch.cuda.Stream(), torch.cuda.Stream()
+    TO = 10_000_000
+
+    def offload():
+        off = 0
+        for (_, c, first, nb, nbytes) in descs:
+            slot, dptr, _ = kvc.kvc_staging_ring_acquire(ring, TO)
+            kvc.kvc_pack(lay, src[first:first + nb], dptr, nbytes, stream=s_k)
+            kvc.kvc_staging_ring_commit(ring, slot, s_k)
+            kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
+            cuda_rt.memcpy_async(hptr + off, dptr, nbytes, cuda_rt.D2H, s_c)
+            kvc.kvc_staging_ring_release(ring, slot, s_c)
+            off += nbytes
+
+    def load():
+        off = 0
+        for (_, c, first, nb, nbytes) in descs:
+            slot, dptr, _ = kvc.kvc_staging_ring_acquire(ring, TO)
+            cuda_rt.memcpy_async(dptr, hptr + off, nbytes, cuda_rt.H2D, s_c)
+            kvc.kvc_staging_ring_commit(ring, slot, s_c)
+            kvc.kvc_staging_ring_wait_filled(ring, slot, s_k)
+            kvc.kvc_unpack(lay, dptr, dst[first:first + nb], nbytes, stream=s_k)
+            kvc.kvc_staging_ring_release(ring, slot, s_k)
+            off += nbytes
+
+    offload()
+    load()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    t_off, t_load = [], []
+    for _ in range(args.e2e_steps):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        offload()
+        torch.cuda.synchronize()
+        t1 = time.perf_counter()
+        load()
+        torch.cuda.synchronize()
+        t2 = time.perf_counter()
+        t_off.append(t1 - t0)
+        t_load.append(t2 - t1)
+    step_s = statistics.mean(t_off) + statistics.mean(t_load)
+    if world > 1:
+        t = torch.tensor([step_s], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        step_s = float(t.item())
+    _, acquires, stalls = kvc.kvc_staging_ring_stats(ring)
+    kvc.kvc_staging_ring_destroy(ring)
+    return {
+        "value": world * 4 * one_way / step_s / 1e9, "unit": "GB/s",
+        "h2d_bytes_per_step": one_way, "d2h_bytes_per_step": one_way,
+        "ms_per_step": step_s * 1e3, "steps": args.e2e_steps,
+        "offload_ms": statistics.mean(t_off) * 1e3, "load_ms": statistics.mean(t_load) * 1e3,
+        "host_link_gbs_offload": one_way / statistics.mean(t_off) / 1e9,
+        "host_link_gbs_load": one_way / statistics.mean(t_load) / 1e9,
+        "path": "kvc_pack -> %d-slot device ring -> cudaMemcpyAsync D2H to pinned host; "
+                "cudaMemcpyAsync H2D -> ring -> kvc_unpack" % args.ring_slots,
+        "ring_acquires": acquires, "ring_stalls": stalls,
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b_80k", choices=["8b_80k", "8b_8k"])
+    ap.add_argument("--chunk-tokens", type=int, default=256)
+    ap.add_argument("--variant", type=int, default=0, help="0 auto, 1 vector kernel, 2 bulk-copy kernel")
+    ap.add_argument("--order", type=int, default=0)
+    ap.add_argument("--tile-bytes", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--ring-slots", type=int, default=8)
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--traffic-bytes", type=float, default=None,
+                    help="DRAM bytes per launch from an ncu capture, copied into the roofline object")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,252 @@
+/*
+ * kvc -- paged KV-cache pack / unpack and a bounded staging ring for external
+ * KV-cache offload, for NVIDIA B200 (sm_100a).
+ *
+ * The operations follow the problem statement of "Building py-kvcache":
+ *   - Sec. 2.1: the KV cache of a serving engine is a pool of fixed-size token
+ *     blocks; bytes per token = layers x 2 x KV heads x head dim x element size.
+ *   - Sec. 6.4: an external cache stores "storage blocks" (here: chunks) that
+ *     group several GPU blocks of one request, in request order; an operation
+ *     on a whole prefix is cut into one job per chunk; every job moves through
+ *     one slot of a fixed, bounded staging pool, and a slot is reused only after
+ *     the CUDA event guarding its last copy has completed.
+ *   - Sec. 6.4 (loads): all block mappings that are ready, from any number of
+ *     requests, are fused into a single launch.
+ *   - Sec. 6.5: requests with an identical prefix stage the shared chunks once.
+ *
+ * Memory model.  The paged pool is [layer][K|V][block][token][kv_head][head_dim]:
+ * every (layer, K|V) "plane" is an array of `num_blocks` blocks, each a run of
+ *     slab_bytes = block_size * num_kv_heads * head_dim * elem_bytes
+ * contiguous bytes, `block_stride` bytes apart.  A chunk of n blocks is the
+ * same layout with the block axis gathered: [layer][K|V][n][token][head][dim],
+ * exactly  layers * planes * n * slab_bytes  bytes, no padding (a short last
+ * chunk is stored compactly).
+ *
+ *   pack  : chunk[l][p][j][...] = pool[l][p][ids[j]][...]     (save / offload)
+ *   unpack: pool[l][p][ids[j]][...] = chunk[l][p][j][...]     (load / preload)
+ *
+ * Elements are opaque bytes.  All functions return a status and never abort.
+ * The library never owns the KV pool.  Handles are not thread-safe: use one
+ * layout handle and one ring per host thread.  Streams are `cudaStream_t`
+ * values passed as `void*` so that this header needs no CUDA include.
+ *
+ * Every copy runs in the library's CUDA kernels; there is no host fallback.
+ */
+#ifndef KVC_H
+#define KVC_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    KVC_OK = 0,
+    KVC_ERR_INVALID_ARG = 1,  /* NULL handle/pointer, zero size, slot too small, bad enum */
+    KVC_ERR_OUT_OF_RANGE = 2, /* a host-resident block id is < 0 or >= num_blocks */
+    KVC_ERR_ALIGNMENT = 3,    /* a pointer, stride or slab size is not a multiple of 16 bytes */
+    KVC_ERR_CONFLICT = 4,     /* unpack: the same destination block named twice (host ids) */
+    KVC_ERR_NOMEM = 5,        /* host or device allocation failed */
+    KVC_ERR_CUDA = 6,         /* a CUDA runtime call failed (no device, launch error, ...) */
+    KVC_ERR_WOULD_BLOCK = 7,  /* ring: no free slot and timeout_us == 0 */
+    KVC_ERR_TIMEOUT = 8,      /* ring: no free slot before the deadline */
+    KVC_ERR_STATE = 9         /* ring: call does not fit the slot's state */
+} kvc_status;
+
+const char *kvc_status_str(kvc_status s);
+
+/* ------------------------------------------------------------------ layout (Sec. 2.1) */
+
+typedef struct kvc_layout kvc_layout;
+
+typedef struct {
+    uint32_t num_layers;
+    uint32_t kv_planes;    /* planes per layer: 2 (K and V), or 1 for a fused cache */
+    uint32_t num_blocks;   /* blocks in every plane of the pool */
+    uint32_t block_size;   /* tokens per block */
+    uint32_t num_kv_heads;
+    uint32_t head_dim;
+    uint32_t elem_bytes;   /* 1, 2 or 4 */
+    uint32_t chunk_tokens; /* tokens per chunk; a positive multiple of block_size */
+    /* Either plane_ptrs != NULL: HOST array of num_layers*kv_planes DEVICE pointers,
+     * entry l*kv_planes+p is the base of plane (l,p) (the array is copied);
+     * or plane_ptrs == NULL: plane (l,p) starts at base + l*layer_stride + p*plane_stride. */
+    const void *const *plane_ptrs;
+    const void *base;      /* device pointer */
+    uint64_t layer_stride; /* bytes */
+    uint64_t plane_stride; /* bytes */
+    uint64_t block_stride; /* bytes between consecutive blocks of a plane; 0 means slab_bytes */
+} kvc_layout_desc;
+
+/* Validates and copies the descriptor.  Makes no CUDA call: the small device-side
+ * state a launch needs (plane-pointer table, status words, id-table arenas) is
+ * allocated by the first pack/unpack call on the handle, which therefore must not
+ * happen during stream capture.
+ * Errors: INVALID_ARG (NULL, zero dimension, chunk_tokens not a multiple of
+ * block_size, elem_bytes not 1/2/4, block_stride < slab_bytes), ALIGNMENT (slab
+ * bytes, a base pointer or a stride not a multiple of 16), NOMEM. */
+kvc_status kvc_layout_create(const kvc_layout_desc *desc, kvc_layout **out);
+/* Frees the handle and its device state (synchronises with work that still uses it). */
+kvc_status kvc_layout_destroy(kvc_layout *layout);
+
+uint64_t kvc_layout_slab_bytes(const kvc_layout *layout);
+uint64_t kvc_layout_bytes_per_token(const kvc_layout *layout);      /* Sec. 2.1 formula */
+uint32_t kvc_layout_blocks_per_chunk(const kvc_layout *layout);     /* chunk_tokens / block_size */
+uint64_t kvc_layout_chunk_bytes(const kvc_layout *layout, uint32_t n_blocks); /* L*P*n*slab */
+uint32_t kvc_layout_num_chunks(const kvc_layout *layout, uint32_t n_blocks);  /* ceil(n / bpc) */
+
+/* How the copy kernels run.  Zero in every field means "library default". */
+typedef enum {
+    KVC_VARIANT_AUTO = 0,
+    KVC_VARIANT_VEC = 1,  /* 16-byte vector loads/stores through registers */
+    KVC_VARIANT_BULK = 2  /* bulk async copies global->shared->global driven by one warp per SM */
+} kvc_variant;
+typedef enum {
+    KVC_ORDER_AUTO = 0,
+    KVC_ORDER_PLANE_MAJOR = 1, /* walk all blocks of one (layer,K|V) plane, then the next plane */
+    KVC_ORDER_BLOCK_MAJOR = 2  /* walk all planes of one block, then the next block */
+} kvc_order;
+typedef struct {
+    uint32_t variant;    /* kvc_variant */
+    uint32_t order;      /* kvc_order */
+    uint32_t max_ctas;   /* cap on thread blocks per launch (0 = fill the GPU); a small cap
+                            leaves SMs to a concurrent compute stream */
+    uint32_t tile_bytes; /* bytes of one slab moved per work item (0 = default); multiple of 16 */
+    uint32_t stages;     /* BULK: shared-memory stages per thread block (0 = default) */
+} kvc_tuning;
+/* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */
+kvc_status kvc_layout_set_tuning(kvc_layout *layout, const kvc_tuning *tuning);
+
+/* ------------------------------------------------------------------ mapper (Sec. 6.4, 6.5) */
+
+typedef struct {
+    uint32_t request;  /* index of the request the chunk belongs to */
+    uint32_t chunk;    /* chunk index inside that request */
+    uint32_t first;    /* first block-table entry covered */
+    uint32_t n_blocks; /* entries covered: blocks_per_chunk, or fewer in the last chunk */
+    uint64_t bytes;    /* kvc_layout_chunk_bytes(n_blocks) */
+} kvc_chunk_desc;
+
+#define KVC_MAP_FULL_CHUNKS_ONLY 1u /* drop a short last chunk (only whole storage blocks are cached) */
+
+/* Cuts one request of n_blocks table entries into chunks: chunk c covers entries
+ * [c*bpc, min((c+1)*bpc, n_blocks)).  Writes up to `cap` descriptors to `out` (may be NULL
+ * with cap 0 to query) and the total count to *n_out.  Host only.
+ * Errors: INVALID_ARG. */
+kvc_status kvc_map_request(const kvc_layout *layout, uint32_t n_blocks, uint32_t flags,
+                           kvc_chunk_desc *out, uint32_t cap, uint32_t *n_out);
+
+/* Same for many requests at once, staging every shared chunk once (Sec. 6.5): a chunk is
+ * dropped when another request's chunk with the same index already carries all of its blocks
+ * at the same table positions with an identical table before them.  tables[r] is a HOST array
+ * of lens[r] block ids.  Output is in (request, chunk) order.  *unique_blocks (may be NULL)
+ * receives the number of blocks covered by the kept chunks.  Host only. */
+kvc_status kvc_map_requests_shared(const kvc_layout *layout, const int32_t *const *tables,
+                                   const uint32_t *lens, uint32_t n_requests, uint32_t flags,
+                                   kvc_chunk_desc *out, uint32_t cap, uint32_t *n_out,
+                                   uint64_t *unique_blocks);
+
+/* ------------------------------------------------------------------ pack / unpack (Sec. 6.4) */
+
+/* One chunk.  `ids` is the chunk's slice of the request's block table, n_blocks entries,
+ * in HOST memory (ids_on_device == 0; may be reused as soon as the call returns) or in DEVICE
+ * memory (ids_on_device != 0; must stay valid until the kernel has run).  `slot` is DEVICE
+ * memory (or mapped pinned host memory), 16-byte aligned, slot_bytes >= chunk_bytes(n_blocks);
+ * bytes of the slot past the chunk are not touched, nor are pool blocks not named in ids.
+ * Asynchronous: the kernel is enqueued on `stream` and the call returns.
+ * Host ids are validated before anything is launched (OUT_OF_RANGE; unpack: CONFLICT on a
+ * repeated id).  Device ids are range-checked in the kernel: a bad id skips its block and
+ * is counted (see kvc_poll_device_status); repeated device ids in unpack are undefined.
+ * n_blocks == 0 is a no-op returning KVC_OK.
+ * Errors: INVALID_ARG, OUT_OF_RANGE, CONFLICT, ALIGNMENT, NOMEM, CUDA. */
+kvc_status kvc_pack(kvc_layout *layout, const int32_t *ids, uint32_t n_blocks, int ids_on_device,
+                    void *dst_slot, uint64_t slot_bytes, void *stream);
+kvc_status kvc_unpack(kvc_layout *layout, const void *src_slot, uint64_t slot_bytes,
+                      const int32_t *ids, uint32_t n_blocks, int ids_on_device, void *stream);
+
+/* Many chunks, possibly of many requests, in ONE launch (the fused launch of Sec. 6.4).
+ * ops is a HOST array; every op is one chunk as above with slot_bytes implied
+ * (= chunk_bytes(n_blocks)).  With host ids, unpack also rejects an id repeated across ops. */
+typedef struct {
+    void *slot;         /* device (or mapped host) memory of chunk_bytes(n_blocks) bytes */
+    const int32_t *ids; /* n_blocks ids, host or device as the call says */
+    uint32_t n_blocks;
+    uint32_t reserved;  /* must be 0 */
+} kvc_chunk_op;
+kvc_status kvc_pack_batch(kvc_layout *layout, const kvc_chunk_op *ops, uint32_t n_ops,
+                          int ids_on_device, void *stream);
+kvc_status kvc_unpack_batch(kvc_layout *layout, const kvc_chunk_op *ops, uint32_t n_ops,
+                            int ids_on_device, void *stream);
+
+/* Waits for `stream`, then reports and clears the handle's device-side counters:
+ * *n_skipped = blocks skipped because a device-resident id was out of range,
+ * *n_wait_expired = bounded waits inside a kernel that gave up (should be 0).
+ * Either pointer may be NULL. */
+kvc_status kvc_poll_device_status(kvc_layout *layout, void *stream, uint32_t *n_skipped,
+                                  uint32_t *n_wait_expired);
+
+/* Number of kernel launches issued through this handle so far. */
+uint64_t kvc_layout_launch_count(const kvc_layout *layout);
+
+/* ------------------------------------------------------------------ staging ring (Sec. 6.4) */
+
+typedef struct kvc_ring kvc_ring;
+typedef enum {
+    KVC_RING_DEVICE = 0,     /* slots in device memory; the caller drains them with async copies */
+    KVC_RING_HOST_MAPPED = 1 /* slots in mapped pinned host memory; kernels write them directly */
+} kvc_ring_kind;
+
+/* A ring of n_slots fixed slots of slot_bytes each (a multiple of 4096; use
+ * chunk_bytes(blocks_per_chunk) rounded up).  mem == NULL: the library allocates
+ * n_slots*slot_bytes (cudaMalloc, or cudaHostAlloc mapped) and frees it on destroy;
+ * otherwise the caller's buffer of mem_bytes >= n_slots*slot_bytes is used and not freed.
+ * Slot life cycle, strictly in slot order 0,1,..,n-1,0,.. (FIFO):
+ *   acquire -> [producer work on stream A] -> commit(A) -> wait_filled(C) ->
+ *   [consumer work on stream C] -> release(C) -> free again once the release event completes.
+ * Errors: INVALID_ARG, ALIGNMENT, NOMEM, CUDA. */
+kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ring_kind kind,
+                                   void *mem, uint64_t mem_bytes, kvc_ring **out);
+/* Waits for outstanding slot events, frees library-owned memory and the handle. */
+kvc_status kvc_staging_ring_destroy(kvc_ring *ring);
+/* Next slot in FIFO order.  It is handed out only if it was never used or the event recorded
+ * by its last release has completed (polled on the host; no device-wide synchronisation).
+ * timeout_us == 0: try once (WOULD_BLOCK); > 0: poll until the deadline (TIMEOUT);
+ * < 0: INVALID_ARG (unbounded waits are not offered).
+ * *dev_ptr is the address kernels and async copies use; *host_ptr the host address
+ * (HOST_MAPPED rings) or NULL.  Either may be NULL. */
+kvc_status kvc_staging_ring_acquire(kvc_ring *ring, int64_t timeout_us, uint32_t *slot,
+                                    void **dev_ptr, void **host_ptr);
+/* Records the slot's "filled" event on the producer stream.  STATE unless acquired. */
+kvc_status kvc_staging_ring_commit(kvc_ring *ring, uint32_t slot, void *producer_stream);
+/* Makes consumer_stream wait for the slot's "filled" event.  STATE unless committed. */
+kvc_status kvc_staging_ring_wait_filled(kvc_ring *ring, uint32_t slot, void *consumer_stream);
+/* Records the slot's "drained" event on the consumer stream; the slot becomes free when that
+ * event completes.  STATE unless committed. */
+kvc_status kvc_staging_ring_release(kvc_ring *ring, uint32_t slot, void *consumer_stream);
+/* in_flight = slots acquired and not yet observed free; stalls = acquire polls that found the
+ * next slot still busy.  Any pointer may be NULL. */
+kvc_status kvc_staging_ring_stats(const kvc_ring *ring, uint32_t *in_flight, uint64_t *acquires,
+                                  uint64_t *stalls);
+uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *ring);
+uint32_t kvc_staging_ring_num_slots(const kvc_ring *ring);
+
+/* Event provider used by a ring.  The default one wraps CUDA events.  Tests replace it to
+ * drive the slot state machine on a machine without a GPU (events that complete on command);
+ * it must be installed before the ring is created and applies to rings created afterwards.
+ * Passing NULL restores the CUDA provider. */
+typedef struct {
+    void *ctx;
+    int (*create)(void *ctx, void **event);               /* 0 on success */
+    int (*destroy)(void *ctx, void *event);
+    int (*record)(void *ctx, void *event, void *stream);
+    int (*query)(void *ctx, void *event);                 /* 0 done, 1 not yet, <0 error */
+    int (*stream_wait)(void *ctx, void *stream, void *event);
+    int (*synchronize)(void *ctx, void *event);
+} kvc_event_provider;
+kvc_status kvc_staging_ring_set_event_provider(const kvc_event_provider *provider);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVC_H */

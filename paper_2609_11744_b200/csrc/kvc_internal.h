@@ -1,0 +1,99 @@
+// Internal declarations shared by the host side and the kernels of libkvc.
+#ifndef KVC_INTERNAL_H
+#define KVC_INTERNAL_H
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "kvc.h"
+
+#define KVC_PARAM_IDS 128u      // block ids that travel inside the kernel parameters
+#define KVC_VEC_THREADS 256u    // threads per block of the vector kernels
+#define KVC_VEC_UNROLL 4u       // 16-byte vectors in flight per thread
+#define KVC_BULK_THREADS 32u    // one warp drives the bulk-copy pipeline
+#define KVC_BULK_MAX_STAGES 16u
+#define KVC_BULK_SMEM_HEADER 1024u  // mbarriers + per-stage bookkeeping ahead of the data stages
+#define KVC_WAIT_LIMIT (1u << 22)   // polls of an mbarrier before a kernel gives up
+
+// Where the planes of the paged pool live (kernel-side copy of the layout).
+struct KvcGeom {
+    const unsigned char *base;              // monolithic pool (plane_table == nullptr)
+    uint64_t layer_stride, plane_stride;
+    const unsigned char *const *plane_table;  // device array of LP plane bases, or nullptr
+    uint64_t block_stride;
+    uint32_t slab_bytes;                    // S
+    uint32_t planes_total;                  // LP = L*P
+    uint32_t planes_per_layer;              // P
+    uint32_t num_blocks;                    // NB
+    uint32_t tile_bytes;                    // bytes of a slab moved by one work item
+    uint32_t parts;                         // ceil(S / tile_bytes)
+};
+
+// One block of one chunk in a batched launch.
+struct KvcEnt {
+    uint64_t slot_addr;   // chunk base + j*S : where block j of the chunk starts in plane 0
+    uint64_t id_or_ptr;   // the pool block id, or the device address of it
+    uint32_t nb_c;        // blocks in this chunk (plane stride inside the chunk = nb_c*S)
+    uint32_t id_is_ptr;
+    uint64_t pad;
+};
+static_assert(sizeof(KvcEnt) == 32, "KvcEnt is loaded as two 16-byte vectors");
+
+// Kernel parameters.
+struct KvcLaunch {
+    KvcGeom g;
+    const KvcEnt *table;      // batched launch: n_ent entries in device memory; else nullptr
+    uint64_t slot;            // single-chunk launch: chunk base
+    const int32_t *dev_ids;   // single-chunk launch with device-resident ids; else nullptr
+    uint32_t *status;         // [0] blocks skipped (bad device id), [1] waits that gave up
+    uint64_t n_items;         // n_ent * LP * parts
+    uint32_t n_ent;
+    uint32_t order;           // kvc_order (never AUTO here)
+    uint32_t stages;          // bulk kernels
+    uint32_t lag;             // bulk kernels: loads issued ahead of the store they feed
+    int32_t ids[KVC_PARAM_IDS];
+};
+
+enum { KVC_DIR_PACK = 0, KVC_DIR_UNPACK = 1 };
+// Internal refinement of KVC_VARIANT_VEC: 32-byte vectors when everything is 32-byte aligned.
+enum { KVC_VARIANT_VEC32 = 100 };
+
+// Implemented in kvc_kernels.cu.
+cudaError_t kvc_launch_copy(int dir, int variant, const KvcLaunch &a, uint32_t grid,
+                            uint32_t smem_bytes, cudaStream_t stream);
+cudaError_t kvc_kernel_limits(int *sm_count, int *vec_blocks_per_sm, int *max_smem_optin);
+
+// A pinned-host + device pair that carries one batched launch's entry table.
+struct KvcArena {
+    KvcEnt *host = nullptr;
+    KvcEnt *dev = nullptr;
+    uint64_t cap = 0;           // entries
+    cudaEvent_t done = nullptr; // recorded after the kernel that reads `dev`
+    bool busy = false;
+};
+
+#define KVC_NUM_ARENAS 8
+
+struct kvc_layout {
+    kvc_layout_desc d;
+    std::vector<const void *> plane_ptrs;  // host copy (empty for monolithic pools)
+    uint64_t slab_bytes, row_bytes, block_stride;
+    uint32_t bpc, planes_total;
+    kvc_tuning tuning;
+    // device state, created by the first launch
+    bool dev_ready;
+    int device;
+    int sm_count, vec_blocks_per_sm, max_smem_optin;
+    const unsigned char **d_plane_table;
+    uint32_t *d_status;
+    uint32_t *h_status;  // pinned
+    KvcArena arenas[KVC_NUM_ARENAS];
+    uint32_t next_arena;
+    uint64_t launches;
+    std::vector<uint32_t> seen;  // scratch for duplicate detection: stamp per pool block
+    uint32_t seen_stamp;
+};
+
+#endif

@@ -1,0 +1,386 @@
+// Copy kernels of libkvc for sm_100a: paged-KV pack (gather) and unpack (scatter).
+//
+// A launch moves n_ent blocks x LP planes x `parts` tiles.  Work item w names one
+// tile of one slab (the contiguous bytes of one block in one (layer, K|V) plane):
+//     pool side : plane(lp) + id*block_stride + part*tile
+//     slot side : chunk + (lp*nb_c + j)*S    + part*tile        (Sec. 6.4 chunk layout)
+// pack copies pool -> slot, unpack slot -> pool.  Nothing is a contraction: the
+// kernels are bound by HBM bandwidth, so they only keep many full-line requests
+// in flight and touch every byte once.
+//
+// Two ways to move a tile:
+//   VEC  : every thread keeps KVC_VEC_UNROLL 16-byte loads in flight, then stores
+//          them; streaming cache hints; many resident blocks per SM.
+//   BULK : one warp per SM drives a ring of shared-memory stages with bulk async
+//          copies (global -> shared, completion on an mbarrier; shared -> global,
+//          completion by bulk group).  Lanes decode 32 work items at a time and
+//          hand them to the issuing lane by shuffle.  Almost no registers or
+//          issue slots are used, which leaves the SM's math pipes to other work.
+// No cluster, no multicast: every byte is read exactly once by exactly one SM.
+#include "kvc_internal.h"
+
+namespace {
+
+struct Item {
+    uint64_t pool;  // address on the paged-pool side
+    uint64_t slot;  // address on the staging side
+    uint32_t len;   // bytes; 0 = skip (block id out of range)
+};
+
+__device__ __forceinline__ uint64_t plane_base(const KvcGeom &g, uint32_t lp)
+{
+    if (g.plane_table != nullptr)
+        return __ldg(reinterpret_cast<const unsigned long long *>(g.plane_table) + lp);
+    uint32_t l = lp / g.planes_per_layer, p = lp - l * g.planes_per_layer;
+    return (uint64_t)g.base + (uint64_t)l * g.layer_stride + (uint64_t)p * g.plane_stride;
+}
+
+// Work item -> addresses.  TABLE: entries come from device memory (batched launch);
+// otherwise ids are in the kernel parameters or in a device id array (one chunk).
+template <bool TABLE>
+__device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool count_bad)
+{
+    const KvcGeom &g = a.g;
+    uint32_t part = w % g.parts;
+    uint32_t r = w / g.parts;
+    uint32_t ent, lp;
+    if (a.order == KVC_ORDER_PLANE_MAJOR) {
+        lp = r / a.n_ent;
+        ent = r - lp * a.n_ent;
+    } else {
+        ent = r / g.planes_total;
+        lp = r - ent * g.planes_total;
+    }
+    uint64_t slot_j;
+    uint32_t nb_c;
+    int64_t id;
+    if (TABLE) {
+        const uint4 *e = reinterpret_cast<const uint4 *>(a.table + ent);
+        uint4 lo = __ldg(e), hi = __ldg(e + 1);
+        slot_j = ((uint64_t)lo.y << 32) | lo.x;
+        uint64_t idp = ((uint64_t)lo.w << 32) | lo.z;
+        nb_c = hi.x;
+        id = hi.y ? (int64_t)__ldg(reinterpret_cast<const int32_t *>(idp)) : (int64_t)(int32_t)lo.z;
+    } else {
+        slot_j = a.slot + (uint64_t)ent * g.slab_bytes;
+        nb_c = a.n_ent;
+        id = a.dev_ids ? (int64_t)__ldg(a.dev_ids + ent) : (int64_t)a.ids[ent];
+    }
+    Item it;
+    uint32_t off = part * g.tile_bytes;
+    it.len = min(g.tile_bytes, g.slab_bytes - off);
+    if (id < 0 || id >= (int64_t)g.num_blocks) {
+        // never touch memory for a bad id: count the block once and skip it
+        if (count_bad && part == 0 && lp == 0)
+            atomicAdd(a.status, 1u);
+        it.len = 0;
+        id = 0;
+    }
+    it.pool = plane_base(g, lp) + (uint64_t)id * g.block_stride + off;
+    it.slot = slot_j + (uint64_t)lp * nb_c * g.slab_bytes + off;
+    return it;
+}
+
+// ------------------------------------------------------------------------------------ VEC
+
+// A VB-byte vector held in registers.  VB = 32 uses the 256-bit global accesses of sm_100,
+// which also accept an L2 evict-first priority (the data is touched once); VB = 16 is the
+// path for layouts that are only 16-byte aligned.
+template <int VB>
+struct Vec;
+
+template <>
+struct Vec<16> {
+    uint32_t r[4];
+    __device__ __forceinline__ void load(uint64_t addr)
+    {
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                     : "l"(addr));
+    }
+    __device__ __forceinline__ void store(uint64_t addr) const
+    {
+        asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(addr), "r"(r[0]), "r"(r[1]),
+                     "r"(r[2]), "r"(r[3])
+                     : "memory");
+    }
+};
+
+template <>
+struct Vec<32> {
+    uint32_t r[8];
+    __device__ __forceinline__ void load(uint64_t addr)
+    {
+        asm volatile(
+            "ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+            : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+              "=r"(r[7])
+            : "l"(addr));
+    }
+    __device__ __forceinline__ void store(uint64_t addr) const
+    {
+        asm volatile(
+            "st.global.L1::no_allocate.L2::evict_first.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(
+                addr),
+            "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+            : "memory");
+    }
+};
+
+template <int DIR, bool TABLE, int VB>
+__global__ void __launch_bounds__(KVC_VEC_THREADS)
+kvc_vec_kernel(const __grid_constant__ KvcLaunch a)
+{
+    constexpr uint32_t SH = VB == 32 ? 5 : 4;
+    const uint32_t tid = threadIdx.x;
+    const uint32_t n_items = (uint32_t)a.n_items;
+    uint32_t w = blockIdx.x;
+    if (w >= n_items)
+        return;
+    Item cur = decode<TABLE>(a, w, tid == 0);
+    while (true) {
+        // decode the next item before the copy so its table read overlaps the data loads
+        uint32_t wn = w + gridDim.x;
+        bool more = wn < n_items && wn > w;
+        Item nxt = cur;
+        if (more)
+            nxt = decode<TABLE>(a, wn, tid == 0);
+        const uint64_t src = DIR == KVC_DIR_PACK ? cur.pool : cur.slot;
+        const uint64_t dst = DIR == KVC_DIR_PACK ? cur.slot : cur.pool;
+        const uint32_t nvec = cur.len >> SH;
+        for (uint32_t v0 = 0; v0 < nvec; v0 += KVC_VEC_THREADS * KVC_VEC_UNROLL) {
+            Vec<VB> r[KVC_VEC_UNROLL];
+#pragma unroll
+            for (uint32_t u = 0; u < KVC_VEC_UNROLL; ++u) {
+                uint32_t v = v0 + u * KVC_VEC_THREADS + tid;
+                if (v < nvec)
+                    r[u].load(src + ((uint64_t)v << SH));
+            }
+#pragma unroll
+            for (uint32_t u = 0; u < KVC_VEC_UNROLL; ++u) {
+                uint32_t v = v0 + u * KVC_VEC_THREADS + tid;
+                if (v < nvec)
+                    r[u].store(dst + ((uint64_t)v << SH));
+            }
+        }
+        if (!more)
+            break;
+        cur = nxt;
+        w = wn;
+    }
+}
+
+// ------------------------------------------------------------------------------------ BULK
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+
+// Bounded wait for a phase of an mbarrier.  Returns false if it gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity)
+{
+    for (uint32_t i = 0; i < KVC_WAIT_LIMIT; ++i) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(parity)
+            : "memory");
+        if (done)
+            return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ void bulk_load(uint32_t dst_smem, uint64_t src, uint32_t bytes,
+                                          uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+            "r"(dst_smem),
+        "l"(src), "r"(bytes), "r"(bar)
+        : "memory");
+}
+
+__device__ __forceinline__ void bulk_store(uint64_t dst, uint32_t src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst),
+                 "r"(src_smem), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ void bulk_commit()
+{
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+// Wait until at most N of this thread's most recent bulk groups still read shared memory.
+template <int N>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+__device__ __forceinline__ void bulk_wait_all()
+{
+    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+#define KVC_BULK_PENDING 1  // stores allowed to be still reading shared memory when a stage is reused
+
+// One warp per block.  Item k of this block uses stage k % stages.  Step k issues the load of
+// item k and the store of item k - lag, so `lag` loads are in flight while stores drain.
+template <int DIR, bool TABLE>
+__global__ void __launch_bounds__(KVC_BULK_THREADS, 1)
+kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem);                       // [stages]
+    uint64_t *st_dst = reinterpret_cast<uint64_t *>(smem + 128);               // [stages]
+    uint32_t *st_len = reinterpret_cast<uint32_t *>(smem + 256);               // [stages]
+    unsigned char *data = smem + KVC_BULK_SMEM_HEADER;
+
+    const uint32_t lane = threadIdx.x;
+    const uint32_t stages = a.stages, lag = a.lag, tile = a.g.tile_bytes;
+    const uint32_t n_items = (uint32_t)a.n_items;
+    if (blockIdx.x >= n_items)
+        return;
+    const uint32_t K = (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x;  // my items
+
+    if (lane == 0) {
+        for (uint32_t s = 0; s < stages; ++s)
+            mbar_init(smem_u32(&bars[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncwarp();
+
+    bool ok = true;          // lane 0: no wait has expired
+    uint32_t loads_done = 0; // lane 0: items whose load was issued (for the drain on failure)
+    uint32_t stores_done = 0;
+    Item mine;
+    mine.pool = mine.slot = 0;
+    mine.len = 0;
+    for (uint32_t k0 = 0; k0 < K + lag; k0 += 32) {
+        // every lane decodes one of the next 32 items of this block
+        uint32_t kk = k0 + lane;
+        if (kk < K)
+            mine = decode<TABLE>(a, blockIdx.x + kk * gridDim.x, true);
+        else
+            mine.len = 0;
+        for (uint32_t i = 0; i < 32; ++i) {
+            const uint32_t k = k0 + i;
+            if (k >= K + lag)
+                break;
+            // broadcast item k from lane i
+            uint64_t pool = __shfl_sync(0xffffffffu, mine.pool, i);
+            uint64_t slot = __shfl_sync(0xffffffffu, mine.slot, i);
+            uint32_t len = __shfl_sync(0xffffffffu, mine.len, i);
+            if (lane == 0 && ok) {
+                if (k < K) {
+                    const uint32_t s = k % stages;
+                    if (k >= stages)
+                        bulk_wait_read<KVC_BULK_PENDING>();  // store of item k-stages has left stage s
+                    const uint32_t bar = smem_u32(&bars[s]);
+                    st_dst[s] = DIR == KVC_DIR_PACK ? slot : pool;
+                    st_len[s] = len;
+                    mbar_expect_tx(bar, len);
+                    if (len)
+                        bulk_load(smem_u32(data + (size_t)s * tile),
+                                  DIR == KVC_DIR_PACK ? pool : slot, len, bar);
+                    loads_done = k + 1;
+                }
+                if (k >= lag) {
+                    const uint32_t m = k - lag;
+                    const uint32_t s = m % stages;
+                    if (mbar_wait(smem_u32(&bars[s]), (m / stages) & 1u)) {
+                        const uint32_t l2 = st_len[s];
+                        if (l2) {
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            bulk_store(st_dst[s], smem_u32(data + (size_t)s * tile), l2);
+                        }
+                        bulk_commit();
+                        stores_done = m + 1;
+                    } else {
+                        ok = false;
+                        atomicAdd(a.status + 1, 1u);
+                    }
+                }
+            }
+        }
+    }
+    if (lane == 0) {
+        if (!ok) {
+            // A wait gave up.  Loads that were issued may still land in shared memory: give each
+            // one more bounded wait so the block does not retire under an incoming copy.
+            for (uint32_t m = stores_done; m < loads_done; ++m)
+                (void)mbar_wait(smem_u32(&bars[m % stages]), (m / stages) & 1u);
+        }
+        bulk_wait_all();
+    }
+}
+
+template <int DIR, bool TABLE>
+cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t smem,
+                       cudaStream_t stream)
+{
+    if (variant == KVC_VARIANT_BULK) {
+        static int configured_smem[2][2] = {{0, 0}, {0, 0}};
+        if ((int)smem > configured_smem[DIR][TABLE]) {
+            cudaError_t e = cudaFuncSetAttribute(kvc_bulk_kernel<DIR, TABLE>,
+                                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)smem);
+            if (e != cudaSuccess)
+                return e;
+            configured_smem[DIR][TABLE] = (int)smem;
+        }
+        kvc_bulk_kernel<DIR, TABLE><<<grid, KVC_BULK_THREADS, smem, stream>>>(a);
+    } else if (variant == KVC_VARIANT_VEC32) {
+        kvc_vec_kernel<DIR, TABLE, 32><<<grid, KVC_VEC_THREADS, 0, stream>>>(a);
+    } else {
+        kvc_vec_kernel<DIR, TABLE, 16><<<grid, KVC_VEC_THREADS, 0, stream>>>(a);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t kvc_launch_copy(int dir, int variant, const KvcLaunch &a, uint32_t grid,
+                            uint32_t smem_bytes, cudaStream_t stream)
+{
+    const bool table = a.table != nullptr;
+    if (dir == KVC_DIR_PACK)
+        return table ? launch_one<KVC_DIR_PACK, true>(variant, a, grid, smem_bytes, stream)
+                     : launch_one<KVC_DIR_PACK, false>(variant, a, grid, smem_bytes, stream);
+    return table ? launch_one<KVC_DIR_UNPACK, true>(variant, a, grid, smem_bytes, stream)
+                 : launch_one<KVC_DIR_UNPACK, false>(variant, a, grid, smem_bytes, stream);
+}
+
+cudaError_t kvc_kernel_limits(int *sm_count, int *vec_blocks_per_sm, int *max_smem_optin)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess)
+        return e;
+    if ((e = cudaDeviceGetAttribute(sm_count, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess)
+        return e;
+    if ((e = cudaDeviceGetAttribute(max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) !=
+        cudaSuccess)
+        return e;
+    return cudaOccupancyMaxActiveBlocksPerMultiprocessor(
+        vec_blocks_per_sm, kvc_vec_kernel<KVC_DIR_PACK, true, 32>, KVC_VEC_THREADS, 0);
+}

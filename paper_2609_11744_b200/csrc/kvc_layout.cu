@@ -1,0 +1,644 @@
+// Host side of libkvc: layout descriptor (Sec. 2.1), block-table -> chunk mapper (Sec. 6.4,
+// shared prefixes Sec. 6.5), argument validation and the launch front ends of pack / unpack.
+#include <string.h>
+
+#include <algorithm>
+#include <chrono>
+#include <map>
+#include <new>
+#include <utility>
+
+#include "kvc_internal.h"
+
+namespace {
+
+inline bool mult16(uint64_t v) { return (v & 15u) == 0; }
+
+kvc_status ensure_device(kvc_layout *lay)
+{
+    if (lay->dev_ready)
+        return KVC_OK;
+    if (cudaGetDevice(&lay->device) != cudaSuccess)
+        return KVC_ERR_CUDA;
+    if (kvc_kernel_limits(&lay->sm_count, &lay->vec_blocks_per_sm, &lay->max_smem_optin) !=
+        cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVC_ERR_CUDA;
+    }
+    if (lay->vec_blocks_per_sm < 1)
+        lay->vec_blocks_per_sm = 1;
+    if (cudaMalloc(&lay->d_status, 2 * sizeof(uint32_t)) != cudaSuccess)
+        return KVC_ERR_NOMEM;
+    if (cudaMemset(lay->d_status, 0, 2 * sizeof(uint32_t)) != cudaSuccess)
+        return KVC_ERR_CUDA;
+    if (cudaHostAlloc(&lay->h_status, 2 * sizeof(uint32_t), cudaHostAllocDefault) != cudaSuccess)
+        return KVC_ERR_NOMEM;
+    if (!lay->plane_ptrs.empty()) {
+        size_t bytes = lay->plane_ptrs.size() * sizeof(void *);
+        if (cudaMalloc(&lay->d_plane_table, bytes) != cudaSuccess)
+            return KVC_ERR_NOMEM;
+        if (cudaMemcpy(lay->d_plane_table, lay->plane_ptrs.data(), bytes, cudaMemcpyHostToDevice) !=
+            cudaSuccess)
+            return KVC_ERR_CUDA;
+    }
+    lay->dev_ready = true;
+    return KVC_OK;
+}
+
+// Fills the geometry and the launch shape that do not depend on the ids.
+struct Plan {
+    int variant;
+    uint32_t grid, smem, stages, lag;
+};
+
+kvc_status make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe, KvcLaunch *a,
+                     Plan *plan)
+{
+    const kvc_tuning &t = lay->tuning;
+    KvcGeom &g = a->g;
+    g.base = static_cast<const unsigned char *>(lay->d.base);
+    g.layer_stride = lay->d.layer_stride;
+    g.plane_stride = lay->d.plane_stride;
+    g.plane_table = lay->d_plane_table;
+    g.block_stride = lay->block_stride;
+    g.slab_bytes = (uint32_t)lay->slab_bytes;
+    g.planes_total = lay->planes_total;
+    g.planes_per_layer = lay->d.kv_planes;
+    g.num_blocks = lay->d.num_blocks;
+
+    int variant = t.variant ? (int)t.variant : KVC_VARIANT_BULK;
+    if (variant == KVC_VARIANT_BULK) {
+        // Bulk copies are used for device memory only; a slot in mapped host memory is
+        // written with ordinary vector stores.
+        cudaPointerAttributes attr;
+        if (cudaPointerGetAttributes(&attr, slot_probe) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KVC_ERR_CUDA;
+        }
+        if (attr.type != cudaMemoryTypeDevice)
+            variant = KVC_VARIANT_VEC;
+    }
+    uint32_t tile = t.tile_bytes;
+    if (tile == 0)
+        tile = variant == KVC_VARIANT_BULK ? 32768u : 16384u;
+    tile = (uint32_t)std::min<uint64_t>(tile, lay->slab_bytes);
+    uint32_t stages = 0, lag = 0, smem = 0;
+    if (variant == KVC_VARIANT_BULK) {
+        const uint32_t room = (uint32_t)lay->max_smem_optin - KVC_BULK_SMEM_HEADER;
+        if (tile > room / 2)
+            tile = (room / 2) & ~15u;
+        stages = t.stages ? t.stages : KVC_BULK_MAX_STAGES;
+        stages = std::min<uint32_t>(std::min<uint32_t>(stages, room / tile), KVC_BULK_MAX_STAGES);
+        if (stages < 2)
+            return KVC_ERR_INVALID_ARG;
+        lag = stages - 2;  // one store may still read its stage when the stage after next is reloaded
+        smem = KVC_BULK_SMEM_HEADER + stages * tile;
+    } else {
+        // 32-byte vectors need every address the kernel forms to be 32-byte aligned
+        bool a32 = (lay->slab_bytes % 32 == 0) && (tile % 32 == 0) && (lay->block_stride % 32 == 0) &&
+                   ((uintptr_t)slot_probe % 32 == 0);
+        if (lay->plane_ptrs.empty()) {
+            a32 = a32 && ((uintptr_t)lay->d.base % 32 == 0) && (lay->d.layer_stride % 32 == 0) &&
+                  (lay->d.plane_stride % 32 == 0);
+        } else {
+            for (const void *p : lay->plane_ptrs)
+                a32 = a32 && ((uintptr_t)p % 32 == 0);
+        }
+        variant = a32 ? (int)KVC_VARIANT_VEC32 : (int)KVC_VARIANT_VEC;
+    }
+    g.tile_bytes = tile;
+    g.parts = (uint32_t)((lay->slab_bytes + tile - 1) / tile);
+    const uint64_t n_items = n_ent * lay->planes_total * g.parts;
+    if (n_items == 0 || n_items > 0xFFFFFFFFull)
+        return KVC_ERR_INVALID_ARG;
+    a->n_items = n_items;
+    a->n_ent = (uint32_t)n_ent;
+    a->order = t.order ? t.order : KVC_ORDER_PLANE_MAJOR;
+    a->stages = stages;
+    a->lag = lag;
+    a->status = lay->d_status;
+    uint64_t grid = variant == KVC_VARIANT_BULK
+                        ? (uint64_t)lay->sm_count
+                        : (uint64_t)lay->sm_count * (uint64_t)lay->vec_blocks_per_sm;
+    if (t.max_ctas)
+        grid = std::min<uint64_t>(grid, t.max_ctas);
+    grid = std::min<uint64_t>(grid, n_items);
+    plan->variant = variant;
+    plan->grid = (uint32_t)grid;
+    plan->smem = smem;
+    plan->stages = stages;
+    plan->lag = lag;
+    return KVC_OK;
+}
+
+// Range check, and for unpack a duplicate check across the whole call, on host-resident ids.
+kvc_status check_host_ids(kvc_layout *lay, const int32_t *ids, uint32_t n, bool reject_dup)
+{
+    const uint32_t nb = lay->d.num_blocks;
+    for (uint32_t j = 0; j < n; ++j)
+        if (ids[j] < 0 || (uint32_t)ids[j] >= nb)
+            return KVC_ERR_OUT_OF_RANGE;
+    if (reject_dup) {
+        for (uint32_t j = 0; j < n; ++j) {
+            uint32_t &s = lay->seen[(uint32_t)ids[j]];
+            if (s == lay->seen_stamp)
+                return KVC_ERR_CONFLICT;
+            s = lay->seen_stamp;
+        }
+    }
+    return KVC_OK;
+}
+
+void begin_dup_scope(kvc_layout *lay)
+{
+    if (lay->seen.size() != lay->d.num_blocks)
+        lay->seen.assign(lay->d.num_blocks, 0);
+    if (++lay->seen_stamp == 0) {  // stamp wrapped: clear and restart
+        std::fill(lay->seen.begin(), lay->seen.end(), 0u);
+        lay->seen_stamp = 1;
+    }
+}
+
+kvc_status copy_one(kvc_layout *lay, int dir, const int32_t *ids, uint32_t n_blocks,
+                    int ids_on_device, void *slot, uint64_t slot_bytes, void *stream)
+{
+    if (!lay || (!ids && n_blocks) || (!slot && n_blocks))
+        return KVC_ERR_INVALID_ARG;
+    if (n_blocks == 0)
+        return KVC_OK;
+    const uint64_t need = kvc_layout_chunk_bytes(lay, n_blocks);
+    if (slot_bytes < need)
+        return KVC_ERR_INVALID_ARG;
+    if (!mult16((uintptr_t)slot))
+        return KVC_ERR_ALIGNMENT;
+    if (!ids_on_device) {
+        try {
+            begin_dup_scope(lay);
+        } catch (const std::bad_alloc &) {
+            return KVC_ERR_NOMEM;
+        }
+        kvc_status s = check_host_ids(lay, ids, n_blocks, dir == KVC_DIR_UNPACK);
+        if (s != KVC_OK)
+            return s;
+        if (n_blocks > KVC_PARAM_IDS) {
+            // too many ids for the kernel parameters: go through the table path
+            kvc_chunk_op op;
+            op.slot = slot;
+            op.ids = ids;
+            op.n_blocks = n_blocks;
+            op.reserved = 0;
+            return dir == KVC_DIR_PACK ? kvc_pack_batch(lay, &op, 1, 0, stream)
+                                       : kvc_unpack_batch(lay, &op, 1, 0, stream);
+        }
+    }
+    kvc_status s = ensure_device(lay);
+    if (s != KVC_OK)
+        return s;
+    KvcLaunch a;
+    memset(&a, 0, sizeof(a));
+    Plan plan;
+    s = make_plan(lay, n_blocks, slot, &a, &plan);
+    if (s != KVC_OK)
+        return s;
+    a.slot = (uint64_t)(uintptr_t)slot;
+    if (ids_on_device)
+        a.dev_ids = ids;
+    else
+        memcpy(a.ids, ids, n_blocks * sizeof(int32_t));
+    if (kvc_launch_copy(dir, plan.variant, a, plan.grid, plan.smem, (cudaStream_t)stream) !=
+        cudaSuccess)
+        return KVC_ERR_CUDA;
+    ++lay->launches;
+    return KVC_OK;
+}
+
+// Picks the next table arena, waiting (on the host) for the kernel that last read it.
+kvc_status take_arena(kvc_layout *lay, uint64_t n_ent, KvcArena **out)
+{
+    KvcArena &ar = lay->arenas[lay->next_arena];
+    lay->next_arena = (lay->next_arena + 1) % KVC_NUM_ARENAS;
+    if (ar.busy) {
+        if (cudaEventSynchronize(ar.done) != cudaSuccess)
+            return KVC_ERR_CUDA;
+        ar.busy = false;
+    }
+    if (!ar.done && cudaEventCreateWithFlags(&ar.done, cudaEventDisableTiming) != cudaSuccess)
+        return KVC_ERR_CUDA;
+    if (ar.cap < n_ent) {
+        if (ar.host)
+            cudaFreeHost(ar.host);
+        if (ar.dev)
+            cudaFree(ar.dev);
+        ar.host = nullptr;
+        ar.dev = nullptr;
+        ar.cap = 0;
+        uint64_t cap = std::max<uint64_t>(n_ent, 4096);
+        if (cudaHostAlloc(&ar.host, cap * sizeof(KvcEnt), cudaHostAllocDefault) != cudaSuccess) {
+            (void)cudaGetLastError();
+            ar.host = nullptr;
+            return KVC_ERR_NOMEM;
+        }
+        if (cudaMalloc(&ar.dev, cap * sizeof(KvcEnt)) != cudaSuccess) {
+            (void)cudaGetLastError();
+            cudaFreeHost(ar.host);
+            ar.host = nullptr;
+            ar.dev = nullptr;
+            return KVC_ERR_NOMEM;
+        }
+        ar.cap = cap;
+    }
+    *out = &ar;
+    return KVC_OK;
+}
+
+kvc_status copy_batch(kvc_layout *lay, int dir, const kvc_chunk_op *ops, uint32_t n_ops,
+                      int ids_on_device, void *stream)
+{
+    if (!lay || (!ops && n_ops))
+        return KVC_ERR_INVALID_ARG;
+    uint64_t n_ent = 0;
+    const void *probe = nullptr;
+    for (uint32_t i = 0; i < n_ops; ++i) {
+        if (ops[i].reserved != 0)
+            return KVC_ERR_INVALID_ARG;
+        if (ops[i].n_blocks == 0)
+            continue;
+        if (!ops[i].slot || !ops[i].ids)
+            return KVC_ERR_INVALID_ARG;
+        if (!mult16((uintptr_t)ops[i].slot))
+            return KVC_ERR_ALIGNMENT;
+        if (!probe || ((uintptr_t)ops[i].slot % 32) != 0)
+            probe = ops[i].slot;  // the least aligned slot decides the vector width
+        n_ent += ops[i].n_blocks;
+    }
+    if (n_ent == 0)
+        return KVC_OK;
+    if (!ids_on_device) {
+        try {
+            begin_dup_scope(lay);
+        } catch (const std::bad_alloc &) {
+            return KVC_ERR_NOMEM;
+        }
+        for (uint32_t i = 0; i < n_ops; ++i) {
+            kvc_status s = check_host_ids(lay, ops[i].ids, ops[i].n_blocks, dir == KVC_DIR_UNPACK);
+            if (s != KVC_OK)
+                return s;
+        }
+    }
+    kvc_status s = ensure_device(lay);
+    if (s != KVC_OK)
+        return s;
+    KvcLaunch a;
+    memset(&a, 0, sizeof(a));
+    Plan plan;
+    s = make_plan(lay, n_ent, probe, &a, &plan);
+    if (s != KVC_OK)
+        return s;
+    KvcArena *ar = nullptr;
+    s = take_arena(lay, n_ent, &ar);
+    if (s != KVC_OK)
+        return s;
+    uint64_t k = 0;
+    for (uint32_t i = 0; i < n_ops; ++i) {
+        for (uint32_t j = 0; j < ops[i].n_blocks; ++j, ++k) {
+            KvcEnt &e = ar->host[k];
+            e.slot_addr = (uint64_t)(uintptr_t)ops[i].slot + (uint64_t)j * lay->slab_bytes;
+            e.nb_c = ops[i].n_blocks;
+            e.pad = 0;
+            if (ids_on_device) {
+                e.id_or_ptr = (uint64_t)(uintptr_t)(ops[i].ids + j);
+                e.id_is_ptr = 1;
+            } else {
+                e.id_or_ptr = (uint64_t)(uint32_t)ops[i].ids[j];
+                e.id_is_ptr = 0;
+            }
+        }
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(ar->dev, ar->host, n_ent * sizeof(KvcEnt), cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return KVC_ERR_CUDA;
+    a.table = ar->dev;
+    if (kvc_launch_copy(dir, plan.variant, a, plan.grid, plan.smem, st) != cudaSuccess)
+        return KVC_ERR_CUDA;
+    if (cudaEventRecord(ar->done, st) != cudaSuccess)
+        return KVC_ERR_CUDA;
+    ar->busy = true;
+    ++lay->launches;
+    return KVC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *kvc_status_str(kvc_status s)
+{
+    switch (s) {
+    case KVC_OK: return "ok";
+    case KVC_ERR_INVALID_ARG: return "invalid argument";
+    case KVC_ERR_OUT_OF_RANGE: return "block id out of range";
+    case KVC_ERR_ALIGNMENT: return "pointer, stride or slab size not a multiple of 16 bytes";
+    case KVC_ERR_CONFLICT: return "destination block named twice";
+    case KVC_ERR_NOMEM: return "out of memory";
+    case KVC_ERR_CUDA: return "CUDA runtime call failed";
+    case KVC_ERR_WOULD_BLOCK: return "no free staging slot";
+    case KVC_ERR_TIMEOUT: return "timed out waiting for a staging slot";
+    case KVC_ERR_STATE: return "call does not fit the slot's state";
+    }
+    return "unknown status";
+}
+
+kvc_status kvc_layout_create(const kvc_layout_desc *d, kvc_layout **out)
+{
+    if (!d || !out)
+        return KVC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!d->num_layers || !d->kv_planes || !d->num_blocks || !d->block_size || !d->num_kv_heads ||
+        !d->head_dim || !d->chunk_tokens)
+        return KVC_ERR_INVALID_ARG;
+    if (d->elem_bytes != 1 && d->elem_bytes != 2 && d->elem_bytes != 4)
+        return KVC_ERR_INVALID_ARG;
+    if (d->chunk_tokens % d->block_size)
+        return KVC_ERR_INVALID_ARG;
+    if (!d->plane_ptrs && !d->base)
+        return KVC_ERR_INVALID_ARG;
+    const uint64_t row = (uint64_t)d->num_kv_heads * d->head_dim * d->elem_bytes;
+    const uint64_t slab = row * d->block_size;
+    const uint64_t planes = (uint64_t)d->num_layers * d->kv_planes;
+    if (slab > 0x7FFFFFFFull || planes > 0xFFFFFFull)
+        return KVC_ERR_INVALID_ARG;
+    const uint64_t bstride = d->block_stride ? d->block_stride : slab;
+    if (bstride < slab)
+        return KVC_ERR_INVALID_ARG;
+    if (!mult16(slab) || !mult16(bstride))
+        return KVC_ERR_ALIGNMENT;
+    if (d->plane_ptrs) {
+        for (uint64_t i = 0; i < planes; ++i) {
+            if (!d->plane_ptrs[i])
+                return KVC_ERR_INVALID_ARG;
+            if (!mult16((uintptr_t)d->plane_ptrs[i]))
+                return KVC_ERR_ALIGNMENT;
+        }
+    } else {
+        if (!mult16((uintptr_t)d->base) || !mult16(d->layer_stride) || !mult16(d->plane_stride))
+            return KVC_ERR_ALIGNMENT;
+        const uint64_t plane_span = (uint64_t)(d->num_blocks - 1) * bstride + slab;
+        if (d->kv_planes > 1 && d->plane_stride < plane_span)
+            return KVC_ERR_INVALID_ARG;
+        if (d->num_layers > 1 && d->layer_stride < plane_span)
+            return KVC_ERR_INVALID_ARG;
+    }
+    kvc_layout *lay = new (std::nothrow) kvc_layout();
+    if (!lay)
+        return KVC_ERR_NOMEM;
+    lay->d = *d;
+    try {
+        if (d->plane_ptrs)
+            lay->plane_ptrs.assign(d->plane_ptrs, d->plane_ptrs + planes);
+    } catch (const std::bad_alloc &) {
+        delete lay;
+        return KVC_ERR_NOMEM;
+    }
+    lay->d.plane_ptrs = nullptr;  // the caller's array is not kept
+    lay->slab_bytes = slab;
+    lay->row_bytes = row;
+    lay->block_stride = bstride;
+    lay->bpc = d->chunk_tokens / d->block_size;
+    lay->planes_total = (uint32_t)planes;
+    memset(&lay->tuning, 0, sizeof(lay->tuning));
+    lay->dev_ready = false;
+    lay->device = -1;
+    lay->sm_count = lay->vec_blocks_per_sm = lay->max_smem_optin = 0;
+    lay->d_plane_table = nullptr;
+    lay->d_status = nullptr;
+    lay->h_status = nullptr;
+    lay->next_arena = 0;
+    lay->launches = 0;
+    lay->seen_stamp = 0;
+    *out = lay;
+    return KVC_OK;
+}
+
+kvc_status kvc_layout_destroy(kvc_layout *lay)
+{
+    if (!lay)
+        return KVC_ERR_INVALID_ARG;
+    kvc_status rc = KVC_OK;
+    for (KvcArena &ar : lay->arenas) {
+        if (ar.busy && cudaEventSynchronize(ar.done) != cudaSuccess)
+            rc = KVC_ERR_CUDA;
+        if (ar.done)
+            cudaEventDestroy(ar.done);
+        if (ar.host)
+            cudaFreeHost(ar.host);
+        if (ar.dev)
+            cudaFree(ar.dev);
+    }
+    if (lay->d_plane_table)
+        cudaFree((void *)lay->d_plane_table);
+    if (lay->d_status)
+        cudaFree(lay->d_status);
+    if (lay->h_status)
+        cudaFreeHost(lay->h_status);
+    delete lay;
+    return rc;
+}
+
+uint64_t kvc_layout_slab_bytes(const kvc_layout *lay) { return lay ? lay->slab_bytes : 0; }
+
+uint64_t kvc_layout_bytes_per_token(const kvc_layout *lay)
+{
+    return lay ? (uint64_t)lay->planes_total * lay->row_bytes : 0;
+}
+
+uint32_t kvc_layout_blocks_per_chunk(const kvc_layout *lay) { return lay ? lay->bpc : 0; }
+
+uint64_t kvc_layout_chunk_bytes(const kvc_layout *lay, uint32_t n_blocks)
+{
+    return lay ? (uint64_t)lay->planes_total * n_blocks * lay->slab_bytes : 0;
+}
+
+uint32_t kvc_layout_num_chunks(const kvc_layout *lay, uint32_t n_blocks)
+{
+    return lay ? (uint32_t)(((uint64_t)n_blocks + lay->bpc - 1) / lay->bpc) : 0;
+}
+
+kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
+{
+    if (!lay || !t)
+        return KVC_ERR_INVALID_ARG;
+    if (t->variant > KVC_VARIANT_BULK || t->order > KVC_ORDER_BLOCK_MAJOR)
+        return KVC_ERR_INVALID_ARG;
+    if (t->tile_bytes % 16)
+        return KVC_ERR_INVALID_ARG;
+    if (t->stages == 1 || t->stages > KVC_BULK_MAX_STAGES)
+        return KVC_ERR_INVALID_ARG;
+    lay->tuning = *t;
+    return KVC_OK;
+}
+
+kvc_status kvc_map_request(const kvc_layout *lay, uint32_t n_blocks, uint32_t flags,
+                           kvc_chunk_desc *out, uint32_t cap, uint32_t *n_out)
+{
+    if (!lay || !n_out || (!out && cap) || (flags & ~KVC_MAP_FULL_CHUNKS_ONLY))
+        return KVC_ERR_INVALID_ARG;
+    uint32_t n = 0;
+    for (uint64_t first = 0; first < n_blocks; first += lay->bpc) {
+        uint32_t nb = (uint32_t)std::min<uint64_t>(lay->bpc, n_blocks - first);
+        if (nb < lay->bpc && (flags & KVC_MAP_FULL_CHUNKS_ONLY))
+            break;
+        if (n < cap) {
+            out[n].request = 0;
+            out[n].chunk = n;
+            out[n].first = (uint32_t)first;
+            out[n].n_blocks = nb;
+            out[n].bytes = kvc_layout_chunk_bytes(lay, nb);
+        }
+        ++n;
+    }
+    *n_out = n;
+    return KVC_OK;
+}
+
+kvc_status kvc_map_requests_shared(const kvc_layout *lay, const int32_t *const *tables,
+                                   const uint32_t *lens, uint32_t n_requests, uint32_t flags,
+                                   kvc_chunk_desc *out, uint32_t cap, uint32_t *n_out,
+                                   uint64_t *unique_blocks)
+{
+    if (!lay || !n_out || (!out && cap) || (n_requests && (!tables || !lens)) ||
+        (flags & ~KVC_MAP_FULL_CHUNKS_ONLY))
+        return KVC_ERR_INVALID_ARG;
+    for (uint32_t r = 0; r < n_requests; ++r)
+        if (lens[r] && !tables[r])
+            return KVC_ERR_INVALID_ARG;
+    try {
+        // A trie over block tables: node = (parent node, block id).  Two table positions are the
+        // same staged block exactly when they reach the same node.  Longer requests go first, so
+        // a chunk that is a truncation of another request's chunk arrives after it and finds its
+        // last node already covered.
+        std::map<std::pair<uint32_t, int32_t>, uint32_t> child;
+        std::vector<char> covered(1, 0);  // node 0 = root
+        std::vector<uint32_t> order(n_requests);
+        for (uint32_t r = 0; r < n_requests; ++r)
+            order[r] = r;
+        std::stable_sort(order.begin(), order.end(),
+                         [&](uint32_t x, uint32_t y) { return lens[x] > lens[y]; });
+        std::vector<kvc_chunk_desc> kept;
+        std::vector<uint32_t> kept_end;            // trie node where each kept chunk ends
+        std::map<uint32_t, uint32_t> owner;        // chunk end node -> lowest request ending a chunk there
+        std::vector<uint32_t> path;
+        uint64_t uniq = 0;
+        for (uint32_t r : order) {
+            const uint32_t n = lens[r];
+            path.resize(n);
+            uint32_t node = 0;
+            for (uint32_t i = 0; i < n; ++i) {
+                auto key = std::make_pair(node, tables[r][i]);
+                auto it = child.find(key);
+                if (it == child.end()) {
+                    uint32_t id = (uint32_t)covered.size();
+                    covered.push_back(0);
+                    it = child.emplace(key, id).first;
+                }
+                node = it->second;
+                path[i] = node;
+            }
+            uint32_t c = 0;
+            for (uint64_t first = 0; first < n; first += lay->bpc, ++c) {
+                uint32_t nb = (uint32_t)std::min<uint64_t>(lay->bpc, n - first);
+                if (nb < lay->bpc && (flags & KVC_MAP_FULL_CHUNKS_ONLY))
+                    break;
+                const uint32_t end = path[first + nb - 1];
+                auto ow = owner.find(end);
+                if (ow == owner.end())
+                    owner[end] = r;
+                else if (r < ow->second)
+                    ow->second = r;
+                if (covered[end])
+                    continue;
+                for (uint32_t i = 0; i < nb; ++i) {
+                    if (!covered[path[first + i]]) {
+                        covered[path[first + i]] = 1;
+                        ++uniq;
+                    }
+                }
+                kvc_chunk_desc cd;
+                cd.request = r;
+                cd.chunk = c;
+                cd.first = (uint32_t)first;
+                cd.n_blocks = nb;
+                cd.bytes = kvc_layout_chunk_bytes(lay, nb);
+                kept.push_back(cd);
+                kept_end.push_back(end);
+            }
+        }
+        // identical chunks of several requests are attributed to the lowest request index
+        for (size_t i = 0; i < kept.size(); ++i)
+            kept[i].request = owner[kept_end[i]];
+        std::sort(kept.begin(), kept.end(), [](const kvc_chunk_desc &x, const kvc_chunk_desc &y) {
+            return x.request != y.request ? x.request < y.request : x.chunk < y.chunk;
+        });
+        for (size_t i = 0; i < kept.size() && i < cap; ++i)
+            out[i] = kept[i];
+        *n_out = (uint32_t)kept.size();
+        if (unique_blocks)
+            *unique_blocks = uniq;
+    } catch (const std::bad_alloc &) {
+        return KVC_ERR_NOMEM;
+    }
+    return KVC_OK;
+}
+
+kvc_status kvc_pack(kvc_layout *lay, const int32_t *ids, uint32_t n_blocks, int ids_on_device,
+                    void *dst_slot, uint64_t slot_bytes, void *stream)
+{
+    return copy_one(lay, KVC_DIR_PACK, ids, n_blocks, ids_on_device, dst_slot, slot_bytes, stream);
+}
+
+kvc_status kvc_unpack(kvc_layout *lay, const void *src_slot, uint64_t slot_bytes,
+                      const int32_t *ids, uint32_t n_blocks, int ids_on_device, void *stream)
+{
+    return copy_one(lay, KVC_DIR_UNPACK, ids, n_blocks, ids_on_device, const_cast<void *>(src_slot),
+                    slot_bytes, stream);
+}
+
+kvc_status kvc_pack_batch(kvc_layout *lay, const kvc_chunk_op *ops, uint32_t n_ops,
+                          int ids_on_device, void *stream)
+{
+    return copy_batch(lay, KVC_DIR_PACK, ops, n_ops, ids_on_device, stream);
+}
+
+kvc_status kvc_unpack_batch(kvc_layout *lay, const kvc_chunk_op *ops, uint32_t n_ops,
+                            int ids_on_device, void *stream)
+{
+    return copy_batch(lay, KVC_DIR_UNPACK, ops, n_ops, ids_on_device, stream);
+}
+
+kvc_status kvc_poll_device_status(kvc_layout *lay, void *stream, uint32_t *n_skipped,
+                                  uint32_t *n_wait_expired)
+{
+    if (!lay)
+        return KVC_ERR_INVALID_ARG;
+    if (n_skipped)
+        *n_skipped = 0;
+    if (n_wait_expired)
+        *n_wait_expired = 0;
+    if (!lay->dev_ready)
+        return KVC_OK;  // nothing was ever launched
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(lay->h_status, lay->d_status, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost,
+                        st) != cudaSuccess ||
+        cudaMemsetAsync(lay->d_status, 0, 2 * sizeof(uint32_t), st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return KVC_ERR_CUDA;
+    if (n_skipped)
+        *n_skipped = lay->h_status[0];
+    if (n_wait_expired)
+        *n_wait_expired = lay->h_status[1];
+    return KVC_OK;
+}
+
+uint64_t kvc_layout_launch_count(const kvc_layout *lay) { return lay ? lay->launches : 0; }
+
+}  // extern "C"

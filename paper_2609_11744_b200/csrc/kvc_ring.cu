@@ -1,0 +1,321 @@
+// Bounded staging ring (Sec. 6.4): a fixed pool of equal slots shared by every transfer; a
+// slot returns to the pool only after the event recorded behind its last copy has completed.
+// Host bookkeeping plus two events per slot; no kernel, no device-wide synchronisation.
+#include <chrono>
+#include <new>
+#include <thread>
+#include <vector>
+
+#include "kvc_internal.h"
+
+namespace {
+
+// ---- default event provider: CUDA events
+int cu_create(void *, void **ev)
+{
+    cudaEvent_t e;
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess)
+        return -1;
+    *ev = e;
+    return 0;
+}
+int cu_destroy(void *, void *ev) { return cudaEventDestroy((cudaEvent_t)ev) == cudaSuccess ? 0 : -1; }
+int cu_record(void *, void *ev, void *st)
+{
+    return cudaEventRecord((cudaEvent_t)ev, (cudaStream_t)st) == cudaSuccess ? 0 : -1;
+}
+int cu_query(void *, void *ev)
+{
+    cudaError_t e = cudaEventQuery((cudaEvent_t)ev);
+    if (e == cudaSuccess)
+        return 0;
+    if (e == cudaErrorNotReady) {
+        (void)cudaGetLastError();
+        return 1;
+    }
+    return -1;
+}
+int cu_stream_wait(void *, void *st, void *ev)
+{
+    return cudaStreamWaitEvent((cudaStream_t)st, (cudaEvent_t)ev, 0) == cudaSuccess ? 0 : -1;
+}
+int cu_sync(void *, void *ev) { return cudaEventSynchronize((cudaEvent_t)ev) == cudaSuccess ? 0 : -1; }
+
+const kvc_event_provider kCudaEvents = {nullptr, cu_create, cu_destroy, cu_record,
+                                        cu_query, cu_stream_wait, cu_sync};
+kvc_event_provider g_events = kCudaEvents;
+bool g_events_custom = false;
+
+enum SlotState {
+    SLOT_FREE = 0,      // never used, or seen drained
+    SLOT_ACQUIRED = 1,  // handed to a producer
+    SLOT_FILLED = 2,    // "filled" event recorded
+    SLOT_DRAINING = 3   // "drained" event recorded, not yet seen complete
+};
+
+struct Slot {
+    SlotState state = SLOT_FREE;
+    void *filled = nullptr;
+    void *drained = nullptr;
+};
+
+}  // namespace
+
+struct kvc_ring {
+    kvc_event_provider ev;
+    bool custom_events;
+    kvc_ring_kind kind;
+    uint64_t slot_bytes;
+    uint32_t n_slots;
+    unsigned char *dev_base;   // address for kernels and async copies
+    unsigned char *host_base;  // host address (HOST_MAPPED) or nullptr
+    bool owns_mem;
+    std::vector<Slot> slots;
+    uint32_t head;             // next slot to hand out
+    uint64_t acquires, stalls;
+};
+
+namespace {
+
+// FREE, or DRAINING whose event has completed.  Returns 0 free, 1 busy, <0 error.
+int slot_is_free(kvc_ring *r, Slot &s)
+{
+    if (s.state == SLOT_FREE)
+        return 0;
+    if (s.state != SLOT_DRAINING)
+        return 1;
+    int q = r->ev.query(r->ev.ctx, s.drained);
+    if (q == 0)
+        s.state = SLOT_FREE;
+    return q;
+}
+
+}  // namespace
+
+extern "C" {
+
+kvc_status kvc_staging_ring_set_event_provider(const kvc_event_provider *p)
+{
+    if (!p) {
+        g_events = kCudaEvents;
+        g_events_custom = false;
+        return KVC_OK;
+    }
+    if (!p->create || !p->destroy || !p->record || !p->query || !p->stream_wait || !p->synchronize)
+        return KVC_ERR_INVALID_ARG;
+    g_events = *p;
+    g_events_custom = true;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ring_kind kind,
+                                   void *mem, uint64_t mem_bytes, kvc_ring **out)
+{
+    if (!out)
+        return KVC_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (slot_bytes == 0 || n_slots == 0 || (kind != KVC_RING_DEVICE && kind != KVC_RING_HOST_MAPPED))
+        return KVC_ERR_INVALID_ARG;
+    if (slot_bytes % 4096)
+        return KVC_ERR_ALIGNMENT;
+    const uint64_t total = slot_bytes * n_slots;
+    if (total / n_slots != slot_bytes)
+        return KVC_ERR_INVALID_ARG;
+    if (mem) {
+        if (mem_bytes < total)
+            return KVC_ERR_INVALID_ARG;
+        if ((uintptr_t)mem % 16)
+            return KVC_ERR_ALIGNMENT;
+    }
+    kvc_ring *r = new (std::nothrow) kvc_ring();
+    if (!r)
+        return KVC_ERR_NOMEM;
+    r->ev = g_events;
+    r->custom_events = g_events_custom;
+    r->kind = kind;
+    r->slot_bytes = slot_bytes;
+    r->n_slots = n_slots;
+    r->dev_base = r->host_base = nullptr;
+    r->owns_mem = false;
+    r->head = 0;
+    r->acquires = r->stalls = 0;
+    try {
+        r->slots.resize(n_slots);
+    } catch (const std::bad_alloc &) {
+        delete r;
+        return KVC_ERR_NOMEM;
+    }
+    kvc_status rc = KVC_OK;
+    if (mem) {
+        r->dev_base = static_cast<unsigned char *>(mem);
+        if (kind == KVC_RING_HOST_MAPPED) {
+            // the caller's pinned buffer: kernels use its device alias
+            r->host_base = static_cast<unsigned char *>(mem);
+            if (!r->custom_events) {
+                void *d = nullptr;
+                if (cudaHostGetDevicePointer(&d, mem, 0) != cudaSuccess) {
+                    (void)cudaGetLastError();
+                    rc = KVC_ERR_CUDA;
+                } else {
+                    r->dev_base = static_cast<unsigned char *>(d);
+                }
+            }
+        }
+    } else if (kind == KVC_RING_DEVICE) {
+        void *p = nullptr;
+        if (cudaMalloc(&p, total) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = KVC_ERR_NOMEM;
+        }
+        r->dev_base = static_cast<unsigned char *>(p);
+        r->owns_mem = rc == KVC_OK;
+    } else {
+        void *h = nullptr, *d = nullptr;
+        if (cudaHostAlloc(&h, total, cudaHostAllocMapped) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = KVC_ERR_NOMEM;
+        } else if (cudaHostGetDevicePointer(&d, h, 0) != cudaSuccess) {
+            (void)cudaGetLastError();
+            cudaFreeHost(h);
+            rc = KVC_ERR_CUDA;
+        } else {
+            r->host_base = static_cast<unsigned char *>(h);
+            r->dev_base = static_cast<unsigned char *>(d);
+            r->owns_mem = true;
+        }
+    }
+    for (uint32_t i = 0; rc == KVC_OK && i < n_slots; ++i) {
+        if (r->ev.create(r->ev.ctx, &r->slots[i].filled) != 0 ||
+            r->ev.create(r->ev.ctx, &r->slots[i].drained) != 0)
+            rc = KVC_ERR_CUDA;
+    }
+    if (rc != KVC_OK) {
+        kvc_staging_ring_destroy(r);
+        return rc;
+    }
+    *out = r;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_destroy(kvc_ring *r)
+{
+    if (!r)
+        return KVC_ERR_INVALID_ARG;
+    kvc_status rc = KVC_OK;
+    for (Slot &s : r->slots) {
+        // work recorded behind a slot may still touch ring memory: wait for it before freeing
+        if (s.state == SLOT_FILLED && s.filled && r->ev.synchronize(r->ev.ctx, s.filled) != 0)
+            rc = KVC_ERR_CUDA;
+        if (s.state == SLOT_DRAINING && s.drained && r->ev.synchronize(r->ev.ctx, s.drained) != 0)
+            rc = KVC_ERR_CUDA;
+        if (s.filled)
+            r->ev.destroy(r->ev.ctx, s.filled);
+        if (s.drained)
+            r->ev.destroy(r->ev.ctx, s.drained);
+    }
+    if (r->owns_mem) {
+        if (r->kind == KVC_RING_DEVICE)
+            cudaFree(r->dev_base);
+        else
+            cudaFreeHost(r->host_base);
+    }
+    delete r;
+    return rc;
+}
+
+kvc_status kvc_staging_ring_acquire(kvc_ring *r, int64_t timeout_us, uint32_t *slot, void **dev_ptr,
+                                    void **host_ptr)
+{
+    if (!r || !slot || timeout_us < 0)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[r->head];
+    const auto deadline =
+        std::chrono::steady_clock::now() + std::chrono::microseconds(timeout_us);
+    for (;;) {
+        int q = slot_is_free(r, s);
+        if (q < 0)
+            return KVC_ERR_CUDA;
+        if (q == 0)
+            break;
+        ++r->stalls;
+        if (timeout_us == 0)
+            return KVC_ERR_WOULD_BLOCK;
+        if (std::chrono::steady_clock::now() >= deadline)
+            return KVC_ERR_TIMEOUT;
+        if (s.state != SLOT_DRAINING)
+            // held by a producer or consumer of this same thread: only the caller can move it on
+            std::this_thread::sleep_for(std::chrono::microseconds(50));
+        else
+            std::this_thread::yield();
+    }
+    s.state = SLOT_ACQUIRED;
+    *slot = r->head;
+    if (dev_ptr)
+        *dev_ptr = r->dev_base + (uint64_t)r->head * r->slot_bytes;
+    if (host_ptr)
+        *host_ptr = r->host_base ? r->host_base + (uint64_t)r->head * r->slot_bytes : nullptr;
+    r->head = (r->head + 1) % r->n_slots;
+    ++r->acquires;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_commit(kvc_ring *r, uint32_t slot, void *producer_stream)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[slot];
+    if (s.state != SLOT_ACQUIRED)
+        return KVC_ERR_STATE;
+    if (r->ev.record(r->ev.ctx, s.filled, producer_stream) != 0)
+        return KVC_ERR_CUDA;
+    s.state = SLOT_FILLED;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_wait_filled(kvc_ring *r, uint32_t slot, void *consumer_stream)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[slot];
+    if (s.state != SLOT_FILLED)
+        return KVC_ERR_STATE;
+    if (r->ev.stream_wait(r->ev.ctx, consumer_stream, s.filled) != 0)
+        return KVC_ERR_CUDA;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_release(kvc_ring *r, uint32_t slot, void *consumer_stream)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[slot];
+    if (s.state != SLOT_FILLED)
+        return KVC_ERR_STATE;
+    if (r->ev.record(r->ev.ctx, s.drained, consumer_stream) != 0)
+        return KVC_ERR_CUDA;
+    s.state = SLOT_DRAINING;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_stats(const kvc_ring *r, uint32_t *in_flight, uint64_t *acquires,
+                                  uint64_t *stalls)
+{
+    if (!r)
+        return KVC_ERR_INVALID_ARG;
+    if (in_flight) {
+        uint32_t n = 0;
+        for (const Slot &s : r->slots)
+            n += s.state != SLOT_FREE;
+        *in_flight = n;
+    }
+    if (acquires)
+        *acquires = r->acquires;
+    if (stalls)
+        *stalls = r->stalls;
+    return KVC_OK;
+}
+
+uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *r) { return r ? r->slot_bytes : 0; }
+uint32_t kvc_staging_ring_num_slots(const kvc_ring *r) { return r ? r->n_slots : 0; }
+
+}  // extern "C"

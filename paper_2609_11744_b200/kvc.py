@@ -1,0 +1,458 @@
+"""ctypes binding of libkvc: one Python function per C entry point, same names.
+
+Only argument marshalling happens here.  Every copy runs in the library's CUDA
+kernels; if ``libkvc.so`` has not been built the import of the library fails
+with an error -- there is no fallback path of any kind.
+
+Pointers may be given as ints, as torch tensors (their ``data_ptr()``) or as
+numpy arrays (host memory).  Streams may be ``None`` (torch's current stream
+when torch has a CUDA context, else the default stream), a ``torch.cuda.Stream``
+or a raw ``cudaStream_t`` value.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkvc.so")
+
+KVC_OK, KVC_ERR_INVALID_ARG, KVC_ERR_OUT_OF_RANGE, KVC_ERR_ALIGNMENT, KVC_ERR_CONFLICT, \
+    KVC_ERR_NOMEM, KVC_ERR_CUDA, KVC_ERR_WOULD_BLOCK, KVC_ERR_TIMEOUT, KVC_ERR_STATE = range(10)
+KVC_VARIANT_AUTO, KVC_VARIANT_VEC, KVC_VARIANT_BULK = 0, 1, 2
+KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR = 0, 1, 2
+KVC_RING_DEVICE, KVC_RING_HOST_MAPPED = 0, 1
+KVC_MAP_FULL_CHUNKS_ONLY = 1
+
+
+class KvcError(RuntimeError):
+    """A libkvc call returned a status other than KVC_OK."""
+
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__("%s: %s (status %d)" % (where, kvc_status_str(status), status))
+
+
+class kvc_layout_desc(ctypes.Structure):
+    _fields_ = [("num_layers", ctypes.c_uint32), ("kv_planes", ctypes.c_uint32),
+                ("num_blocks", ctypes.c_uint32), ("block_size", ctypes.c_uint32),
+                ("num_kv_heads", ctypes.c_uint32), ("head_dim", ctypes.c_uint32),
+                ("elem_bytes", ctypes.c_uint32), ("chunk_tokens", ctypes.c_uint32),
+                ("plane_ptrs", ctypes.POINTER(ctypes.c_void_p)), ("base", ctypes.c_void_p),
+                ("layer_stride", ctypes.c_uint64), ("plane_stride", ctypes.c_uint64),
+                ("block_stride", ctypes.c_uint64)]
+
+
+class kvc_tuning(ctypes.Structure):
+    _fields_ = [("variant", ctypes.c_uint32), ("order", ctypes.c_uint32),
+                ("max_ctas", ctypes.c_uint32), ("tile_bytes", ctypes.c_uint32),
+                ("stages", ctypes.c_uint32)]
+
+
+class kvc_chunk_desc(ctypes.Structure):
+    _fields_ = [("request", ctypes.c_uint32), ("chunk", ctypes.c_uint32),
+                ("first", ctypes.c_uint32), ("n_blocks", ctypes.c_uint32),
+                ("bytes", ctypes.c_uint64)]
+
+
+# kvc_chunk_op as a numpy record so that thousands of ops can be filled without a Python loop
+CHUNK_OP_DTYPE = np.dtype([("slot", np.uint64), ("ids", np.uint64), ("n_blocks", np.uint32),
+                           ("reserved", np.uint32)])
+assert CHUNK_OP_DTYPE.itemsize == 24
+
+_EVENT_FN = {
+    "create": ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.POINTER(ctypes.c_void_p)),
+    "destroy": ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p),
+    "record": ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p),
+    "query": ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p),
+    "stream_wait": ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p),
+    "synchronize": ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p),
+}
+
+
+class kvc_event_provider(ctypes.Structure):
+    _fields_ = [("ctx", ctypes.c_void_p)] + [(k, v) for k, v in _EVENT_FN.items()]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "libkvc.so is missing (%s). Build it with `python -m paper_2609_11744_b200.build`; "
+            "there is no fallback implementation." % LIB_PATH)
+    L = ctypes.CDLL(LIB_PATH)
+    vp, u32, u64, i64, ci = ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint64, ctypes.c_int64, ctypes.c_int
+    P = ctypes.POINTER
+    sig = {
+        "kvc_status_str": (ctypes.c_char_p, [ci]),
+        "kvc_layout_create": (ci, [P(kvc_layout_desc), P(vp)]),
+        "kvc_layout_destroy": (ci, [vp]),
+        "kvc_layout_slab_bytes": (u64, [vp]),
+        "kvc_layout_bytes_per_token": (u64, [vp]),
+        "kvc_layout_blocks_per_chunk": (u32, [vp]),
+        "kvc_layout_chunk_bytes": (u64, [vp, u32]),
+        "kvc_layout_num_chunks": (u32, [vp, u32]),
+        "kvc_layout_set_tuning": (ci, [vp, P(kvc_tuning)]),
+        "kvc_map_request": (ci, [vp, u32, u32, P(kvc_chunk_desc), u32, P(u32)]),
+        "kvc_map_requests_shared": (ci, [vp, P(vp), P(u32), u32, u32, P(kvc_chunk_desc), u32, P(u32),
+                                         P(u64)]),
+        "kvc_pack": (ci, [vp, vp, u32, ci, vp, u64, vp]),
+        "kvc_unpack": (ci, [vp, vp, u64, vp, u32, ci, vp]),
+        "kvc_pack_batch": (ci, [vp, vp, u32, ci, vp]),
+        "kvc_unpack_batch": (ci, [vp, vp, u32, ci, vp]),
+        "kvc_poll_device_status": (ci, [vp, vp, P(u32), P(u32)]),
+        "kvc_layout_launch_count": (u64, [vp]),
+        "kvc_staging_ring_create": (ci, [u64, u32, ci, vp, u64, P(vp)]),
+        "kvc_staging_ring_destroy": (ci, [vp]),
+        "kvc_staging_ring_acquire": (ci, [vp, i64, P(u32), P(vp), P(vp)]),
+        "kvc_staging_ring_commit": (ci, [vp, u32, vp]),
+        "kvc_staging_ring_wait_filled": (ci, [vp, u32, vp]),
+        "kvc_staging_ring_release": (ci, [vp, u32, vp]),
+        "kvc_staging_ring_stats": (ci, [vp, P(u32), P(u64), P(u64)]),
+        "kvc_staging_ring_slot_bytes": (u64, [vp]),
+        "kvc_staging_ring_num_slots": (u32, [vp]),
+        "kvc_staging_ring_set_event_provider": (ci, [P(kvc_event_provider)]),
+    }
+    for name, (res, args) in sig.items():
+        f = getattr(L, name)
+        f.restype, f.argtypes = res, args
+    _lib = L
+    return L
+
+
+# ------------------------------------------------------------------ marshalling helpers
+def _ptr(x) -> int:
+    """Address of a torch tensor, numpy array, ctypes object or a plain int."""
+    if x is None:
+        return 0
+    if isinstance(x, int):
+        return x
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    if isinstance(x, np.ndarray):
+        return int(x.ctypes.data)
+    if isinstance(x, ctypes.c_void_p):
+        return int(x.value or 0)
+    raise TypeError("cannot take the address of %r" % type(x))
+
+
+def _nbytes(x) -> int:
+    if hasattr(x, "data_ptr"):
+        return int(x.numel() * x.element_size())
+    if isinstance(x, np.ndarray):
+        return int(x.nbytes)
+    raise TypeError("need an explicit size for %r" % type(x))
+
+
+def _stream(s) -> int:
+    if s is None:
+        try:
+            import torch
+            if torch.cuda.is_available() and torch.cuda.is_initialized():
+                return int(torch.cuda.current_stream().cuda_stream)
+        except ImportError:
+            pass
+        return 0
+    if isinstance(s, int):
+        return s
+    return int(s.cuda_stream)
+
+
+def _ids(ids) -> Tuple[object, int, int, int]:
+    """(keep-alive object, address, count, on_device) of a block-id list.
+    Host ids are converted to a contiguous int32 array; a CUDA tensor must already be int32."""
+    if hasattr(ids, "data_ptr"):
+        import torch
+        if ids.is_cuda:
+            if ids.dtype != torch.int32 or not ids.is_contiguous():
+                raise TypeError("device-resident block ids must be a contiguous int32 tensor")
+            return ids, int(ids.data_ptr()), int(ids.numel()), 1
+        ids = ids.numpy()
+    a = np.ascontiguousarray(np.asarray(ids, dtype=np.int32))
+    return a, int(a.ctypes.data), int(a.size), 0
+
+
+def _check(status: int, where: str) -> None:
+    if status != KVC_OK:
+        raise KvcError(status, where)
+
+
+def kvc_status_str(status: int) -> str:
+    return lib().kvc_status_str(int(status)).decode()
+
+
+# ------------------------------------------------------------------ layout
+class LayoutHandle:
+    """Owns a ``kvc_layout*``."""
+
+    def __init__(self, handle: int, keep):
+        self.handle = handle
+        self._keep = keep
+
+    def __del__(self):
+        try:
+            if self.handle and _lib is not None:
+                _lib.kvc_layout_destroy(self.handle)
+        except Exception:
+            pass
+        self.handle = 0
+
+
+def kvc_layout_create(num_layers: int, kv_planes: int, num_blocks: int, block_size: int,
+                      num_kv_heads: int, head_dim: int, elem_bytes: int, chunk_tokens: int,
+                      base=None, layer_stride: int = 0, plane_stride: int = 0,
+                      block_stride: int = 0, plane_ptrs: Optional[Sequence] = None) -> LayoutHandle:
+    d = kvc_layout_desc(num_layers, kv_planes, num_blocks, block_size, num_kv_heads, head_dim,
+                        elem_bytes, chunk_tokens)
+    keep = [base, plane_ptrs]
+    if plane_ptrs is not None:
+        arr = (ctypes.c_void_p * len(plane_ptrs))(*[_ptr(p) for p in plane_ptrs])
+        if len(plane_ptrs) != num_layers * kv_planes:
+            raise ValueError("plane_ptrs needs num_layers*kv_planes entries")
+        d.plane_ptrs = ctypes.cast(arr, ctypes.POINTER(ctypes.c_void_p))
+    else:
+        d.base = _ptr(base)
+        d.layer_stride, d.plane_stride = layer_stride, plane_stride
+    d.block_stride = block_stride
+    out = ctypes.c_void_p()
+    _check(lib().kvc_layout_create(ctypes.byref(d), ctypes.byref(out)), "kvc_layout_create")
+    return LayoutHandle(out.value, keep)
+
+
+def kvc_layout_create_dense(pool, num_layers, kv_planes, num_blocks, block_size, num_kv_heads,
+                            head_dim, elem_bytes, chunk_tokens) -> LayoutHandle:
+    """Layout over one dense allocation [L][P][NB][B][H][D] (a tensor or a device address)."""
+    slab = block_size * num_kv_heads * head_dim * elem_bytes
+    plane = slab * num_blocks
+    return kvc_layout_create(num_layers, kv_planes, num_blocks, block_size, num_kv_heads, head_dim,
+                             elem_bytes, chunk_tokens, base=pool, layer_stride=plane * kv_planes,
+                             plane_stride=plane)
+
+
+def kvc_layout_destroy(layout: LayoutHandle) -> None:
+    h, layout.handle = layout.handle, 0
+    if h:
+        _check(lib().kvc_layout_destroy(h), "kvc_layout_destroy")
+
+
+def kvc_layout_slab_bytes(layout) -> int:
+    return lib().kvc_layout_slab_bytes(layout.handle)
+
+
+def kvc_layout_bytes_per_token(layout) -> int:
+    return lib().kvc_layout_bytes_per_token(layout.handle)
+
+
+def kvc_layout_blocks_per_chunk(layout) -> int:
+    return lib().kvc_layout_blocks_per_chunk(layout.handle)
+
+
+def kvc_layout_chunk_bytes(layout, n_blocks: int) -> int:
+    return lib().kvc_layout_chunk_bytes(layout.handle, n_blocks)
+
+
+def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
+    return lib().kvc_layout_num_chunks(layout.handle, n_blocks)
+
+
+def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0) -> None:
+    t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages)
+    _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
+
+
+def kvc_layout_launch_count(layout) -> int:
+    return lib().kvc_layout_launch_count(layout.handle)
+
+
+# ------------------------------------------------------------------ mapper
+def _descs(arr, n) -> List[Tuple[int, int, int, int, int]]:
+    return [(d.request, d.chunk, d.first, d.n_blocks, d.bytes) for d in arr[:n]]
+
+
+def kvc_map_request(layout, n_blocks: int, flags: int = 0):
+    """[(request, chunk, first, n_blocks, bytes)] for one request."""
+    n = ctypes.c_uint32()
+    _check(lib().kvc_map_request(layout.handle, n_blocks, flags, None, 0, ctypes.byref(n)),
+           "kvc_map_request")
+    arr = (kvc_chunk_desc * max(1, n.value))()
+    _check(lib().kvc_map_request(layout.handle, n_blocks, flags, arr, n.value, ctypes.byref(n)),
+           "kvc_map_request")
+    return _descs(arr, n.value)
+
+
+def kvc_map_requests_shared(layout, tables: Sequence, flags: int = 0):
+    """([(request, chunk, first, n_blocks, bytes)], unique_blocks) with shared chunks staged once."""
+    tabs = [np.ascontiguousarray(np.asarray(t, dtype=np.int32)) for t in tables]
+    nreq = len(tabs)
+    ptrs = (ctypes.c_void_p * max(1, nreq))(*[t.ctypes.data for t in tabs])
+    lens = (ctypes.c_uint32 * max(1, nreq))(*[t.size for t in tabs])
+    n, uniq = ctypes.c_uint32(), ctypes.c_uint64()
+    L = lib()
+    _check(L.kvc_map_requests_shared(layout.handle, ptrs, lens, nreq, flags, None, 0,
+                                     ctypes.byref(n), ctypes.byref(uniq)), "kvc_map_requests_shared")
+    arr = (kvc_chunk_desc * max(1, n.value))()
+    _check(L.kvc_map_requests_shared(layout.handle, ptrs, lens, nreq, flags, arr, n.value,
+                                     ctypes.byref(n), ctypes.byref(uniq)), "kvc_map_requests_shared")
+    return _descs(arr, n.value), uniq.value
+
+
+# ------------------------------------------------------------------ pack / unpack
+def kvc_pack(layout, ids, dst_slot, slot_bytes: Optional[int] = None, stream=None) -> None:
+    keep, p, n, dev = _ids(ids)
+    nb = _nbytes(dst_slot) if slot_bytes is None else slot_bytes
+    _check(lib().kvc_pack(layout.handle, p, n, dev, _ptr(dst_slot), nb, _stream(stream)), "kvc_pack")
+
+
+def kvc_unpack(layout, src_slot, ids, slot_bytes: Optional[int] = None, stream=None) -> None:
+    keep, p, n, dev = _ids(ids)
+    nb = _nbytes(src_slot) if slot_bytes is None else slot_bytes
+    _check(lib().kvc_unpack(layout.handle, _ptr(src_slot), nb, p, n, dev, _stream(stream)),
+           "kvc_unpack")
+
+
+def make_chunk_ops(slot_addrs, ids_addrs, n_blocks) -> np.ndarray:
+    """Array of kvc_chunk_op records from three equally long sequences."""
+    ops = np.zeros(len(n_blocks), dtype=CHUNK_OP_DTYPE)
+    ops["slot"] = np.asarray(slot_addrs, dtype=np.uint64)
+    ops["ids"] = np.asarray(ids_addrs, dtype=np.uint64)
+    ops["n_blocks"] = np.asarray(n_blocks, dtype=np.uint32)
+    return ops
+
+
+def request_chunk_ops(layout, ids, staging, flags: int = 0):
+    """Ops that move one request's chunks to/from a staging area where the chunks lie back to
+    back in request order.  Returns (ops, keep_alive, total_bytes, ids_on_device)."""
+    keep, p, n, dev = _ids(ids)
+    descs = kvc_map_request(layout, n, flags)
+    nb = np.array([d[3] for d in descs], dtype=np.uint64)
+    first = np.array([d[2] for d in descs], dtype=np.uint64)
+    sizes = np.array([d[4] for d in descs], dtype=np.uint64)
+    offs = np.concatenate([[0], np.cumsum(sizes)[:-1]]).astype(np.uint64) if len(descs) else sizes
+    ops = make_chunk_ops(np.uint64(_ptr(staging)) + offs, np.uint64(p) + first * np.uint64(4), nb)
+    return ops, keep, int(sizes.sum()), dev
+
+
+def _batch(fn_name: str, layout, ops: np.ndarray, ids_on_device: int, stream) -> None:
+    if ops.dtype != CHUNK_OP_DTYPE or not ops.flags.c_contiguous:
+        raise TypeError("ops must be a contiguous array of CHUNK_OP_DTYPE")
+    fn = getattr(lib(), fn_name)
+    _check(fn(layout.handle, ops.ctypes.data, len(ops), int(ids_on_device), _stream(stream)), fn_name)
+
+
+def kvc_pack_batch(layout, ops: np.ndarray, ids_on_device: int = 0, stream=None) -> None:
+    _batch("kvc_pack_batch", layout, ops, ids_on_device, stream)
+
+
+def kvc_unpack_batch(layout, ops: np.ndarray, ids_on_device: int = 0, stream=None) -> None:
+    _batch("kvc_unpack_batch", layout, ops, ids_on_device, stream)
+
+
+def kvc_poll_device_status(layout, stream=None) -> Tuple[int, int]:
+    """(blocks skipped for a bad device-resident id, in-kernel waits that gave up), then clears."""
+    a, b = ctypes.c_uint32(), ctypes.c_uint32()
+    _check(lib().kvc_poll_device_status(layout.handle, _stream(stream), ctypes.byref(a),
+                                        ctypes.byref(b)), "kvc_poll_device_status")
+    return a.value, b.value
+
+
+# ------------------------------------------------------------------ staging ring
+class RingHandle:
+    """Owns a ``kvc_ring*``."""
+
+    def __init__(self, handle: int, keep):
+        self.handle = handle
+        self._keep = keep
+
+    def __del__(self):
+        try:
+            if self.handle and _lib is not None:
+                _lib.kvc_staging_ring_destroy(self.handle)
+        except Exception:
+            pass
+        self.handle = 0
+
+
+def kvc_staging_ring_create(slot_bytes: int, n_slots: int, kind: int = KVC_RING_DEVICE, mem=None,
+                            mem_bytes: Optional[int] = None) -> RingHandle:
+    out = ctypes.c_void_p()
+    mb = 0 if mem is None else (_nbytes(mem) if mem_bytes is None else mem_bytes)
+    _check(lib().kvc_staging_ring_create(slot_bytes, n_slots, kind, _ptr(mem), mb, ctypes.byref(out)),
+           "kvc_staging_ring_create")
+    return RingHandle(out.value, mem)
+
+
+def kvc_staging_ring_destroy(ring: RingHandle) -> None:
+    h, ring.handle = ring.handle, 0
+    if h:
+        _check(lib().kvc_staging_ring_destroy(h), "kvc_staging_ring_destroy")
+
+
+def kvc_staging_ring_acquire(ring, timeout_us: int = 0) -> Tuple[int, int, int]:
+    """(slot index, device address, host address or 0).  Raises KvcError(WOULD_BLOCK/TIMEOUT)."""
+    slot, dp, hp = ctypes.c_uint32(), ctypes.c_void_p(), ctypes.c_void_p()
+    _check(lib().kvc_staging_ring_acquire(ring.handle, timeout_us, ctypes.byref(slot),
+                                          ctypes.byref(dp), ctypes.byref(hp)),
+           "kvc_staging_ring_acquire")
+    return slot.value, int(dp.value or 0), int(hp.value or 0)
+
+
+def kvc_staging_ring_commit(ring, slot: int, producer_stream=None) -> None:
+    _check(lib().kvc_staging_ring_commit(ring.handle, slot, _stream(producer_stream)),
+           "kvc_staging_ring_commit")
+
+
+def kvc_staging_ring_wait_filled(ring, slot: int, consumer_stream=None) -> None:
+    _check(lib().kvc_staging_ring_wait_filled(ring.handle, slot, _stream(consumer_stream)),
+           "kvc_staging_ring_wait_filled")
+
+
+def kvc_staging_ring_release(ring, slot: int, consumer_stream=None) -> None:
+    _check(lib().kvc_staging_ring_release(ring.handle, slot, _stream(consumer_stream)),
+           "kvc_staging_ring_release")
+
+
+def kvc_staging_ring_stats(ring) -> Tuple[int, int, int]:
+    """(in_flight, acquires, stalls)."""
+    a, b, c = ctypes.c_uint32(), ctypes.c_uint64(), ctypes.c_uint64()
+    _check(lib().kvc_staging_ring_stats(ring.handle, ctypes.byref(a), ctypes.byref(b),
+                                        ctypes.byref(c)), "kvc_staging_ring_stats")
+    return a.value, b.value, c.value
+
+
+def kvc_staging_ring_slot_bytes(ring) -> int:
+    return lib().kvc_staging_ring_slot_bytes(ring.handle)
+
+
+def kvc_staging_ring_num_slots(ring) -> int:
+    return lib().kvc_staging_ring_num_slots(ring.handle)
+
+
+_provider_keep = None
+
+
+def kvc_staging_ring_set_event_provider(provider: Optional[dict]) -> None:
+    """Install callables {create, destroy, record, query, stream_wait, synchronize} (each
+    taking the C callback's arguments, ctx first), or None for CUDA events.  Used by
+    host-only tests."""
+    global _provider_keep
+    if provider is None:
+        _check(lib().kvc_staging_ring_set_event_provider(None), "kvc_staging_ring_set_event_provider")
+        _provider_keep = None
+        return
+    p = kvc_event_provider()
+    fns = {}
+    for name, ftype in _EVENT_FN.items():
+        fns[name] = ftype(provider[name])
+        setattr(p, name, fns[name])
+    _check(lib().kvc_staging_ring_set_event_provider(ctypes.byref(p)),
+           "kvc_staging_ring_set_event_provider")
+    _provider_keep = (p, fns)

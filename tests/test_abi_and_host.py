@@ -1,0 +1,302 @@
+"""Host-side checks that need no GPU: the library loads, exports what the header declares,
+validates arguments before any CUDA call, and the mapper / ring state machine behave."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import oracle as orc
+from paper_2609_11744_b200 import kvc
+import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _layout(chunk_tokens=64, NB=32, base=0x10000, **kw):
+    args = dict(num_layers=2, kv_planes=2, num_blocks=NB, block_size=16, num_kv_heads=4,
+                head_dim=64, elem_bytes=2, chunk_tokens=chunk_tokens)
+    args.update(kw)
+    if "plane_ptrs" in args:
+        return kvc.kvc_layout_create(**args)
+    return kvc.kvc_layout_create_dense(base, *[args[k] for k in (
+        "num_layers", "kv_planes", "num_blocks", "block_size", "num_kv_heads", "head_dim",
+        "elem_bytes", "chunk_tokens")])
+
+
+def test_library_exports_every_declared_symbol():
+    text = open(os.path.join(ROOT, "include", "kvc.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    declared = set(re.findall(r"\b(kvc_[a-z0-9_]+)\s*\(", text))
+    declared -= {"kvc_status"}
+    assert len(declared) >= 25
+    L = kvc.lib()
+    for name in sorted(declared):
+        assert hasattr(L, name), name
+    assert kvc.kvc_status_str(kvc.KVC_OK) == "ok"
+    assert all(kvc.kvc_status_str(i) for i in range(10))
+
+
+def test_layout_sizes_and_mapper_match_paper_numbers():
+    # Llama-3.2-3B shape (Sec. 2.1: 112 KiB per token; Sec. 6.4: ~28 MiB per 256-token block)
+    lay = kvc.kvc_layout_create_dense(0x100000, 28, 2, 1000, 16, 8, 128, 2, 256)
+    assert kvc.kvc_layout_bytes_per_token(lay) == 114688
+    assert kvc.kvc_layout_slab_bytes(lay) == 32768
+    assert kvc.kvc_layout_blocks_per_chunk(lay) == 16
+    assert kvc.kvc_layout_chunk_bytes(lay, 16) == 28 * 2**20
+    assert kvc.kvc_layout_bytes_per_token(lay) * 81920 == int(8.75 * 2**30)
+    assert kvc.kvc_layout_num_chunks(lay, 5000) == 313
+    d = kvc.kvc_map_request(lay, 5000)
+    assert len(d) == 313 and d[-1] == (0, 312, 4992, 8, 8 * 28 * 2 * 32768)
+    assert len(kvc.kvc_map_request(lay, 5000, kvc.KVC_MAP_FULL_CHUNKS_ONLY)) == 312
+    assert kvc.kvc_map_request(lay, 0) == []
+    kvc.kvc_layout_destroy(lay)
+
+
+@pytest.mark.parametrize("n,chunk_tokens", [(64, 256), (5000, 16), (5000, 2048), (3, 256), (129, 2048)])
+def test_mapper_matches_oracle_ranges(n, chunk_tokens):
+    lay = _layout(chunk_tokens=chunk_tokens, NB=8192)
+    g = orc.Dims(2, 2, 8192, 16, 4, 64, 2)
+    want = orc.chunk_ranges(n, chunk_tokens // 16)
+    got = kvc.kvc_map_request(lay, n)
+    assert [(f, nb) for _, _, f, nb, _ in got] == want
+    assert [b for *_, b in got] == [orc.chunk_bytes(g, nb) for _, nb in want]
+    assert [c for _, c, *_ in got] == list(range(len(want)))
+
+
+def test_shared_prefix_mapper_matches_bruteforce():
+    lay = _layout(chunk_tokens=32, NB=4096)   # 2 blocks per chunk
+    shared = [10, 11, 12, 13]
+    cases = [
+        [shared + [20, 21, 22], shared + [30], shared[:2], shared + [20, 21, 22]],
+        [[1, 2, 3, 4], [9, 2, 3, 4]],
+        [[1, 2, 3], [1, 2, 3, 4]],
+        [[5], [5], [5, 6], []],
+        [[1, 2, 3, 4, 5], [1, 2, 3, 9, 9], [1, 2, 3]],
+    ]
+    rng = np.random.default_rng(0)
+    for _ in range(30):   # random forests of tables with common prefixes
+        root = rng.permutation(200)[:12].tolist()
+        tabs = []
+        for _ in range(int(rng.integers(1, 7))):
+            k = int(rng.integers(0, 13))
+            tabs.append(root[:k] + rng.integers(200, 400, int(rng.integers(0, 6))).tolist())
+        cases.append(tabs)
+    for tabs in cases:
+        got, uniq = kvc.kvc_map_requests_shared(lay, tabs)
+        want = orc.dedup_ops(tabs, 2)
+        assert [(r, c, f, nb) for r, c, f, nb, _ in got] == want, tabs
+        keys = {tuple(t[:i + 1]) for t in tabs for i in range(len(t))}
+        assert uniq == len(keys)
+
+
+def test_shared_prefix_mapper_on_batch_workload():
+    w = wl.WORKLOADS["70b_batch"]
+    nb_pool, tables = wl.batch_workload(w, scale=1 / 16)
+    lay = kvc.kvc_layout_create_dense(0x100000, 80, 2, nb_pool, 16, 8, 128, 2, 256 // 16 * 16 // 16 * 16)
+    got, uniq = kvc.kvc_map_requests_shared(lay, tables)
+    want = orc.dedup_ops([t.tolist() for t in tables], kvc.kvc_layout_blocks_per_chunk(lay))
+    assert [(r, c, f, nb) for r, c, f, nb, _ in got] == want
+    assert uniq == len({int(b) for t in tables for b in t})
+    assert uniq < sum(len(t) for t in tables)
+
+
+def test_create_rejects_bad_descriptors():
+    def status(**kw):
+        with pytest.raises(kvc.KvcError) as e:
+            _layout(**kw)
+        return e.value.status
+    assert status(chunk_tokens=24) == kvc.KVC_ERR_INVALID_ARG          # not a multiple of block_size
+    assert status(elem_bytes=3) == kvc.KVC_ERR_INVALID_ARG
+    assert status(num_layers=0) == kvc.KVC_ERR_INVALID_ARG
+    assert status(base=0) == kvc.KVC_ERR_INVALID_ARG
+    assert status(base=0x10008) == kvc.KVC_ERR_ALIGNMENT
+    assert status(num_kv_heads=1, head_dim=1, block_size=4, chunk_tokens=4) == kvc.KVC_ERR_ALIGNMENT
+    with pytest.raises(kvc.KvcError) as e:   # block stride smaller than a slab
+        kvc.kvc_layout_create(2, 2, 8, 16, 4, 64, 2, 64, base=0x10000, layer_stride=1 << 20,
+                              plane_stride=1 << 19, block_stride=4096)
+    assert e.value.status == kvc.KVC_ERR_INVALID_ARG
+    with pytest.raises(kvc.KvcError) as e:   # planes overlap
+        kvc.kvc_layout_create(2, 2, 8, 16, 4, 64, 2, 64, base=0x10000, layer_stride=1 << 20,
+                              plane_stride=4096)
+    assert e.value.status == kvc.KVC_ERR_INVALID_ARG
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_layout_create(1, 2, 8, 16, 4, 64, 2, 64, plane_ptrs=[0x10000, 0x20004])
+    assert e.value.status == kvc.KVC_ERR_ALIGNMENT
+
+
+def test_pack_unpack_validate_before_any_launch():
+    """Bad arguments are refused on the host; nothing reaches CUDA (there is no GPU here anyway)."""
+    lay = _layout(chunk_tokens=64, NB=32)
+    chunk = kvc.kvc_layout_chunk_bytes(lay, 4)
+    slot = 0x7f0000000000
+    def st(fn, *a, **k):
+        with pytest.raises(kvc.KvcError) as e:
+            fn(*a, **k)
+        return e.value.status
+    assert st(kvc.kvc_pack, lay, [0, 1, 32, 3], slot, chunk) == kvc.KVC_ERR_OUT_OF_RANGE
+    assert st(kvc.kvc_pack, lay, [0, -1], slot, chunk) == kvc.KVC_ERR_OUT_OF_RANGE
+    assert st(kvc.kvc_pack, lay, [0, 1, 2, 3], slot, chunk - 1) == kvc.KVC_ERR_INVALID_ARG
+    assert st(kvc.kvc_pack, lay, [0, 1, 2, 3], slot + 8, chunk) == kvc.KVC_ERR_ALIGNMENT
+    assert st(kvc.kvc_unpack, lay, slot, [5, 6, 5], chunk) == kvc.KVC_ERR_CONFLICT
+    assert st(kvc.kvc_unpack, lay, slot, [99], chunk) == kvc.KVC_ERR_OUT_OF_RANGE
+    kvc.kvc_pack(lay, [], slot, 0)            # empty chunk: a no-op that succeeds
+    kvc.kvc_unpack(lay, slot, [], 0)
+    ids = np.array([1, 2, 3, 4, 2], dtype=np.int32)
+    ops = kvc.make_chunk_ops([slot, slot + chunk], [ids.ctypes.data, ids.ctypes.data + 12], [3, 2])
+    assert st(kvc.kvc_unpack_batch, lay, ops) == kvc.KVC_ERR_CONFLICT      # id 2 in two ops
+    ops["reserved"][0] = 1
+    assert st(kvc.kvc_pack_batch, lay, ops) == kvc.KVC_ERR_INVALID_ARG
+    kvc.kvc_pack_batch(lay, ops[:0])          # no ops: no-op
+    assert kvc.kvc_layout_launch_count(lay) == 0
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+def test_set_tuning_validation():
+    lay = _layout()
+    kvc.kvc_layout_set_tuning(lay, variant=kvc.KVC_VARIANT_VEC, max_ctas=8, tile_bytes=8192)
+    for bad in (dict(variant=3), dict(order=3), dict(tile_bytes=24), dict(stages=1), dict(stages=99)):
+        with pytest.raises(kvc.KvcError):
+            kvc.kvc_layout_set_tuning(lay, **bad)
+
+
+def test_product_never_imports_the_oracle():
+    pkg = os.path.join(ROOT, "paper_2609_11744_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".h", ".cpp")):
+                assert "oracle" not in open(os.path.join(dirpath, f)).read().lower(), f
+
+
+# ------------------------------------------------------------------ ring state machine with fake events
+class FakeEvents:
+    """Events that complete only when the test says so."""
+
+    def __init__(self):
+        self.done = {}
+        self.recorded = []
+        self.next = 1
+
+    def provider(self):
+        def create(ctx, out):
+            out[0] = self.next
+            self.done[self.next] = True
+            self.next += 1
+            return 0
+        def destroy(ctx, ev):
+            self.done.pop(ev, None)
+            return 0
+        def record(ctx, ev, stream):
+            self.done[ev] = False
+            self.recorded.append((ev, stream))
+            return 0
+        def query(ctx, ev):
+            return 0 if self.done[ev] else 1
+        def stream_wait(ctx, stream, ev):
+            return 0
+        def synchronize(ctx, ev):
+            self.done[ev] = True
+            return 0
+        return dict(create=create, destroy=destroy, record=record, query=query,
+                    stream_wait=stream_wait, synchronize=synchronize)
+
+    def complete_all(self):
+        for k in self.done:
+            self.done[k] = True
+
+
+@pytest.fixture
+def fake_events():
+    fe = FakeEvents()
+    kvc.kvc_staging_ring_set_event_provider(fe.provider())
+    yield fe
+    kvc.kvc_staging_ring_set_event_provider(None)
+
+
+def test_ring_state_machine(fake_events):
+    n, sb = 4, 8192
+    mem = np.zeros(n * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    ring = kvc.kvc_staging_ring_create(sb, n, kvc.KVC_RING_DEVICE, base, n * sb)
+    assert kvc.kvc_staging_ring_num_slots(ring) == n and kvc.kvc_staging_ring_slot_bytes(ring) == sb
+    got = [kvc.kvc_staging_ring_acquire(ring) for _ in range(n)]
+    assert [g[0] for g in got] == [0, 1, 2, 3]                       # FIFO
+    assert [g[1] for g in got] == [base + i * sb for i in range(n)]
+    with pytest.raises(kvc.KvcError) as e:                           # N+1-th: all slots held
+        kvc.kvc_staging_ring_acquire(ring)
+    assert e.value.status == kvc.KVC_ERR_WOULD_BLOCK
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_acquire(ring, timeout_us=2000)
+    assert e.value.status == kvc.KVC_ERR_TIMEOUT
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_acquire(ring, timeout_us=-1)
+    assert e.value.status == kvc.KVC_ERR_INVALID_ARG
+    # wrong-order calls are refused
+    for fn in (kvc.kvc_staging_ring_wait_filled, kvc.kvc_staging_ring_release):
+        with pytest.raises(kvc.KvcError) as e:
+            fn(ring, 0, 0)
+        assert e.value.status == kvc.KVC_ERR_STATE
+    kvc.kvc_staging_ring_commit(ring, 0, 11)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_commit(ring, 0, 11)
+    assert e.value.status == kvc.KVC_ERR_STATE
+    kvc.kvc_staging_ring_wait_filled(ring, 0, 22)
+    kvc.kvc_staging_ring_release(ring, 0, 22)
+    assert [s for _, s in fake_events.recorded] == [11, 22]
+    # released but its event has not completed: still not reusable (Sec. 6.4)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_acquire(ring)
+    assert e.value.status == kvc.KVC_ERR_WOULD_BLOCK
+    assert kvc.kvc_staging_ring_stats(ring)[0] == 4
+    fake_events.complete_all()
+    assert kvc.kvc_staging_ring_acquire(ring)[0] == 0                # exactly one more succeeds
+    with pytest.raises(kvc.KvcError):
+        kvc.kvc_staging_ring_acquire(ring)
+    in_flight, acquires, stalls = kvc.kvc_staging_ring_stats(ring)
+    assert (in_flight, acquires) == (4, 5) and stalls >= 4
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_commit(ring, 9, 0)
+    assert e.value.status == kvc.KVC_ERR_INVALID_ARG
+    kvc.kvc_staging_ring_destroy(ring)
+
+
+def test_ring_streams_a_request_larger_than_itself(fake_events):
+    """A prefix of many chunks passes through a few slots; every slot is reused only after the
+    test has let its release event complete, and chunks come out in order."""
+    n, sb, chunks = 3, 4096, 17
+    mem = np.zeros(n * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    view = mem[base - mem.ctypes.data:][:n * sb].reshape(n, sb)
+    ring = kvc.kvc_staging_ring_create(sb, n, kvc.KVC_RING_DEVICE, base, n * sb)
+    out, pending = [], []
+    for c in range(chunks):
+        try:
+            slot, dp, _ = kvc.kvc_staging_ring_acquire(ring)
+        except kvc.KvcError as e:
+            assert e.status == kvc.KVC_ERR_WOULD_BLOCK and len(pending) == n
+            fake_events.complete_all()          # "the copies finished"
+            pending.clear()
+            slot, dp, _ = kvc.kvc_staging_ring_acquire(ring)
+        assert slot == c % n and dp == base + slot * sb
+        view[slot, :] = c                        # producer fills the slot
+        kvc.kvc_staging_ring_commit(ring, slot, 1)
+        kvc.kvc_staging_ring_wait_filled(ring, slot, 2)
+        out.append(int(view[slot, 0]))           # consumer drains it
+        kvc.kvc_staging_ring_release(ring, slot, 2)
+        pending.append(slot)
+    assert out == list(range(chunks))
+    assert kvc.kvc_staging_ring_stats(ring)[1] == chunks
+    kvc.kvc_staging_ring_destroy(ring)
+
+
+def test_ring_create_validation(fake_events):
+    for args, want in [((4096, 0, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
+                       ((0, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
+                       ((4100, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_ALIGNMENT),
+                       ((4096, 2, 7, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
+                       ((4096, 4, 0, 0x1000, 8192), kvc.KVC_ERR_INVALID_ARG),
+                       ((4096, 2, 0, 0x1008, 1 << 20), kvc.KVC_ERR_ALIGNMENT)]:
+        with pytest.raises(kvc.KvcError) as e:
+            kvc.kvc_staging_ring_create(*args)
+        assert e.value.status == want, args

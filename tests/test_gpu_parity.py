@@ -1,0 +1,397 @@
+"""GPU parity: the CUDA path, called through the C-ABI binding, against the CPU oracle on the
+same seeded inputs, byte for byte.  Pure byte movement, so the bar is bit-exact equality."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import oracle as orc
+from paper_2609_11744_b200 import cuda_rt, kvc
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+VARIANTS = [kvc.KVC_VARIANT_VEC, kvc.KVC_VARIANT_BULK]
+
+
+def dims_of(shape: wl.KVShape, NB: int) -> orc.Dims:
+    return orc.Dims(shape.L, shape.P, NB, shape.B, shape.H, shape.D, shape.e)
+
+
+def dense_layout(pool_t, g: orc.Dims, chunk_tokens: int):
+    return kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, chunk_tokens)
+
+
+def to_dev(a: np.ndarray):
+    return torch.from_numpy(a).to(DEV)
+
+
+def staged_chunks(staging_t, sizes):
+    host = staging_t.cpu().numpy()
+    out, off = [], 0
+    for s in sizes:
+        out.append(host[off:off + s])
+        off += s
+    return out, host[off:]
+
+
+_ORACLE_CACHE = {}
+
+
+def _oracle_results(g, pool_np, src_ids, dst_ids, chunk_tokens):
+    """Oracle chunks of pack(src) and the pool after unpacking them into dst (cached: the
+    oracle is slow and many launch configurations share the same expected bytes)."""
+    key = (g, id(pool_np), src_ids.tobytes(), dst_ids.tobytes(), chunk_tokens)
+    if key not in _ORACLE_CACHE:
+        chunks = orc.pack_request(g, pool_np, src_ids, chunk_tokens)
+        pool2 = pool_np.copy()
+        orc.unpack_request(g, pool2, chunks, dst_ids, chunk_tokens)
+        if len(_ORACLE_CACHE) > 4:
+            _ORACLE_CACHE.clear()
+        _ORACLE_CACHE[key] = (chunks, pool2, pool_np)
+    return _ORACLE_CACHE[key][:2]
+
+
+def run_pack_unpack(g, pool_np, src_ids, dst_ids, chunk_tokens, variant, order, mode, tile=0,
+                    layout_factory=None, pool_dev=None):
+    """Pack src_ids into a staging area, unpack into dst_ids of the same pool, and compare both
+    results with the oracle.  mode: 'chunk' (one call per chunk, host ids), 'chunk_dev'
+    (device ids), 'batch' / 'batch_dev' (one launch)."""
+    pool_t = to_dev(pool_np) if pool_dev is None else pool_dev
+    lay = (layout_factory or dense_layout)(pool_t, g, chunk_tokens)
+    kvc.kvc_layout_set_tuning(lay, variant=variant, order=order, tile_bytes=tile)
+    descs = kvc.kvc_map_request(lay, len(src_ids))
+    sizes = [d[4] for d in descs]
+    total = sum(sizes)
+    guard = 4096
+    staging = torch.full((total + guard,), 0xAB, dtype=torch.uint8, device=DEV)
+    want_chunks, want_pool = _oracle_results(g, pool_np, src_ids, dst_ids, chunk_tokens)
+
+    def go(direction, ids_np):
+        ids_dev = to_dev(ids_np) if mode.endswith("_dev") else None
+        if mode.startswith("batch"):
+            ops, keep, nbytes, dev = kvc.request_chunk_ops(
+                lay, ids_dev if ids_dev is not None else ids_np, staging)
+            assert nbytes == total
+            (kvc.kvc_pack_batch if direction == "pack" else kvc.kvc_unpack_batch)(lay, ops, dev)
+        else:
+            off = 0
+            for (_, _, first, nb, nbytes) in descs:
+                ids_c = (ids_dev if ids_dev is not None else ids_np)[first:first + nb]
+                if ids_dev is not None:
+                    ids_c = ids_c.contiguous()
+                slot = staging[off:off + nbytes]
+                if direction == "pack":
+                    kvc.kvc_pack(lay, ids_c, slot)
+                else:
+                    kvc.kvc_unpack(lay, slot, ids_c)
+                off += nbytes
+        torch.cuda.synchronize()
+
+    go("pack", src_ids)
+    got_chunks, tail = staged_chunks(staging, sizes)
+    for c, (a, b) in enumerate(zip(got_chunks, want_chunks)):
+        assert np.array_equal(a, b), "pack chunk %d differs" % c
+    assert (tail == 0xAB).all(), "bytes past the last chunk were written"
+
+    go("unpack", dst_ids)
+    got_pool = pool_t.cpu().numpy().reshape(-1)
+    assert np.array_equal(got_pool, want_pool), "pool after unpack differs"
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+    kvc.kvc_layout_destroy(lay)
+
+
+# ------------------------------------------------------------------ config 1: tiny, K/V separate buffers
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("mode", ["chunk", "chunk_dev", "batch", "batch_dev"])
+def test_tiny_separate_planes(variant, mode):
+    w = wl.WORKLOADS["tiny"]
+    g = dims_of(w.shape, w.pool_blocks)
+    plane_bytes = g.NB * g.slab_bytes
+    planes_np = [wl.random_bits(w.seed + 10 + i, plane_bytes) for i in range(g.L * g.P)]
+    src = wl.block_ids(w.seed, g.NB, w.request_blocks)
+    dst = wl.block_ids(w.dst_seed, g.NB, w.request_blocks)
+    assert not np.array_equal(src, dst)
+    planes_t = [to_dev(p) for p in planes_np]
+    lay = kvc.kvc_layout_create(g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256, plane_ptrs=planes_t)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    assert kvc.kvc_layout_num_chunks(lay, len(src)) == 4
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    assert cb == 512 * 1024
+    staging = torch.full((4 * cb + 4096,), 0x5C, dtype=torch.uint8, device=DEV)
+    ids_s = to_dev(src) if mode.endswith("dev") else src
+    ids_d = to_dev(dst) if mode.endswith("dev") else dst
+    if mode.startswith("batch"):
+        ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, ids_s, staging)
+        kvc.kvc_pack_batch(lay, ops, dev)
+    else:
+        for c in range(4):
+            kvc.kvc_pack(lay, ids_s[c * 16:(c + 1) * 16], staging[c * cb:(c + 1) * cb])
+    torch.cuda.synchronize()
+    host = staging.cpu().numpy()
+    for c in range(4):
+        want = orc.pack_chunk_planes(g, planes_np, src[c * 16:(c + 1) * 16])
+        assert np.array_equal(host[c * cb:(c + 1) * cb], want)
+    assert (host[4 * cb:] == 0x5C).all()
+    # the separate-plane chunk equals the chunk of the same data laid out as one dense pool
+    mono = np.concatenate(planes_np)
+    assert np.array_equal(host[:cb], orc.pack_chunk(g, mono, src[:16]))
+    if mode.startswith("batch"):
+        ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, ids_d, staging)
+        kvc.kvc_unpack_batch(lay, ops, dev)
+    else:
+        for c in range(4):
+            kvc.kvc_unpack(lay, staging[c * cb:(c + 1) * cb], ids_d[c * 16:(c + 1) * 16])
+    torch.cuda.synchronize()
+    want_planes = [p.copy() for p in planes_np]
+    for c in range(4):
+        orc.unpack_chunk_planes(g, want_planes, host[c * cb:(c + 1) * cb], dst[c * 16:(c + 1) * 16])
+    for t, wnt in zip(planes_t, want_planes):
+        assert np.array_equal(t.cpu().numpy(), wnt)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+# ------------------------------------------------------------------ 8B shape, several tiles + ragged tail
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("order", [kvc.KVC_ORDER_PLANE_MAJOR, kvc.KVC_ORDER_BLOCK_MAJOR])
+@pytest.mark.parametrize("mode,chunk_tokens", [("chunk", 256), ("batch", 256), ("batch", 16),
+                                               ("batch_dev", 2048), ("chunk", 2048)])
+def test_8b_shape_reduced_pool(variant, order, mode, chunk_tokens):
+    """Llama-3.1-8B KV shape with a 384-block pool (768 MiB); 136-block request: 8 full
+    256-token chunks and a short one of 8 blocks; one full 2048-token chunk plus the same tail."""
+    w = wl.WORKLOADS["8b_8k"]
+    g = dims_of(w.shape, 384)
+    pool = _pool_8b_384()
+    src = wl.block_ids(w.seed, g.NB, 136)
+    dst = wl.block_ids(w.dst_seed, g.NB, 136)
+    run_pack_unpack(g, pool, src, dst, chunk_tokens, variant, order, mode)
+
+
+_POOL_CACHE = {}
+
+
+def _pool_8b_384():
+    if "p" not in _POOL_CACHE:
+        w = wl.WORKLOADS["8b_8k"]
+        _POOL_CACHE["p"] = wl.random_bits(w.seed + 1, dims_of(w.shape, 384).pool_bytes)
+    return _POOL_CACHE["p"]
+
+
+def test_single_call_with_more_ids_than_fit_in_parameters():
+    w = wl.WORKLOADS["8b_8k"]
+    g = dims_of(w.shape, 384)
+    pool = _pool_8b_384()
+    src = wl.block_ids(5, g.NB, 136)
+    dst = wl.block_ids(6, g.NB, 136)
+    # one chunk of 136 blocks: more ids than the kernel parameters hold (128) -> id-table path
+    run_pack_unpack(g, pool, src, dst, 136 * 16, kvc.KVC_VARIANT_AUTO, 0, "chunk")
+
+
+# ------------------------------------------------------------------ odd geometries
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("geom,tile", [
+    ((3, 2, 40, 4, 2, 8, 1), 0),        # fp8-like, S = 64 B
+    ((2, 1, 33, 1, 1, 24, 2), 0),       # one plane per layer, S = 48 B: 16-byte vectors only
+    ((2, 2, 50, 16, 4, 64, 2), 3088),   # S = 8 KiB cut into ragged tiles 3088+3088+2016
+    ((1, 2, 19, 16, 8, 128, 4), 20480), # fp32, S = 64 KiB, tiles 20480*3 + 4096
+    ((5, 2, 64, 8, 2, 128, 2), 0),      # block_size 8
+])
+def test_odd_geometries(variant, geom, tile):
+    g = orc.Dims(*geom)
+    pool = wl.random_bits(99 + g.L, g.pool_bytes)
+    n = min(g.NB - 2, 27)
+    src = wl.block_ids(1, g.NB, n)
+    dst = wl.block_ids(2, g.NB, n)
+    for mode in ("chunk", "batch"):
+        run_pack_unpack(g, pool, src, dst, 4 * g.B, variant, kvc.KVC_ORDER_PLANE_MAJOR, mode, tile)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_padded_block_stride_and_plane_pointers(variant):
+    """Blocks 1.5 slabs apart inside separately allocated planes: padding is never read or written."""
+    g = orc.Dims(3, 2, 24, 16, 4, 64, 2)
+    bs = g.slab_bytes * 3 // 2
+    planes_np = []
+    for i in range(g.L * g.P):
+        q = np.full(g.NB * bs, 0xCC, dtype=np.uint8)
+        q.reshape(g.NB, bs)[:, :g.slab_bytes] = wl.random_bits(40 + i, g.NB * g.slab_bytes).reshape(
+            g.NB, g.slab_bytes)
+        planes_np.append(q)
+    planes_t = [to_dev(p) for p in planes_np]
+    lay = kvc.kvc_layout_create(g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 64, block_stride=bs,
+                                plane_ptrs=planes_t)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    src = wl.block_ids(3, g.NB, 10)
+    dst = wl.block_ids(4, g.NB, 10)
+    staging = torch.zeros(10 * g.bytes_per_block, dtype=torch.uint8, device=DEV)
+    ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, src, staging)
+    kvc.kvc_pack_batch(lay, ops, dev)
+    ops2, keep2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+    kvc.kvc_unpack_batch(lay, ops2, dev)
+    torch.cuda.synchronize()
+    host = staging.cpu().numpy()
+    want_planes = [p.copy() for p in planes_np]
+    off = 0
+    for f, nb in orc.chunk_ranges(10, 4):
+        want = orc.pack_chunk_planes(g, planes_np, src[f:f + nb], bs)
+        assert np.array_equal(host[off:off + want.size], want)
+        orc.unpack_chunk_planes(g, want_planes, want, dst[f:f + nb], bs)
+        off += want.size
+    for t, wnt in zip(planes_t, want_planes):
+        got = t.cpu().numpy()
+        assert np.array_equal(got, wnt)
+        assert (got.reshape(g.NB, bs)[:, g.slab_bytes:] == 0xCC).all()
+
+
+# ------------------------------------------------------------------ device-side id check
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_bad_device_ids_are_skipped_and_counted(variant):
+    g = orc.Dims(2, 2, 32, 16, 4, 64, 2)
+    pool = wl.random_bits(77, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 128)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    ids = np.array([3, 32, 7, -1, 9, 1 << 30, 0, 31], dtype=np.int32)   # three bad ids
+    good = (ids >= 0) & (ids < g.NB)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 8)
+    staging = torch.full((cb,), 0x11, dtype=torch.uint8, device=DEV)
+    kvc.kvc_pack(lay, to_dev(ids), staging)
+    assert kvc.kvc_poll_device_status(lay) == (3, 0)
+    got = staging.cpu().numpy().reshape(g.L * g.P, 8, g.slab_bytes)
+    safe = np.where(good, ids, 0).astype(np.int32)
+    want = orc.pack_chunk(g, pool, safe).reshape(g.L * g.P, 8, g.slab_bytes)
+    assert np.array_equal(got[:, good], want[:, good])
+    assert (got[:, ~good] == 0x11).all()           # slabs of bad ids are left alone
+    # unpack with bad ids: only the good blocks change
+    chunk = wl.random_bits(78, cb)
+    kvc.kvc_unpack(lay, to_dev(chunk), to_dev(ids))
+    assert kvc.kvc_poll_device_status(lay) == (3, 0)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)   # cleared by the poll
+    want_pool = pool.copy()
+    c3 = chunk.reshape(g.L * g.P, 8, g.slab_bytes)
+    p3 = want_pool.reshape(g.L * g.P, g.NB, g.slab_bytes)
+    for j in np.flatnonzero(good):
+        p3[:, ids[j]] = c3[:, j]
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+
+
+def test_duplicate_source_blocks_in_pack():
+    g = orc.Dims(2, 2, 16, 16, 4, 64, 2)
+    pool = wl.random_bits(79, g.pool_bytes)
+    lay = dense_layout(to_dev(pool), g, 16 * 6)
+    ids = np.array([5, 5, 0, 15, 5, 0], dtype=np.int32)
+    staging = torch.zeros(kvc.kvc_layout_chunk_bytes(lay, 6), dtype=torch.uint8, device=DEV)
+    kvc.kvc_pack(lay, ids, staging)
+    torch.cuda.synchronize()
+    assert np.array_equal(staging.cpu().numpy(), orc.pack_chunk(g, pool, ids))
+
+
+def test_limited_grid_still_correct():
+    """max_ctas caps the launch (used to leave SMs to a compute stream); results do not change."""
+    w = wl.WORKLOADS["8b_8k"]
+    g = dims_of(w.shape, 384)
+    pool = _pool_8b_384()
+    src, dst = wl.block_ids(8, g.NB, 40), wl.block_ids(9, g.NB, 40)
+    for variant in VARIANTS:
+        pool_t = to_dev(pool)
+        lay = dense_layout(pool_t, g, 256)
+        kvc.kvc_layout_set_tuning(lay, variant=variant, max_ctas=3, stages=3)
+        staging = torch.zeros(40 * g.bytes_per_block, dtype=torch.uint8, device=DEV)
+        ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, src, staging)
+        kvc.kvc_pack_batch(lay, ops, dev)
+        torch.cuda.synchronize()
+        want = np.concatenate(orc.pack_request(g, pool, src, 256))
+        assert np.array_equal(staging.cpu().numpy(), want)
+
+
+# ------------------------------------------------------------------ config 4 (reduced): many requests, one launch
+def test_batched_unpack_of_many_requests_with_shared_prefix():
+    """70B-class geometry cut to 4 layers, lengths scaled by 1/8, chunk 64 tokens: every kept
+    chunk of every request unpacked by ONE kvc_unpack_batch call; shared chunks staged once."""
+    w = wl.WORKLOADS["70b_batch"]
+    nb_pool, tables = wl.batch_workload(w, scale=1 / 8)
+    g = orc.Dims(4, 2, nb_pool, 16, 8, 128, 2)
+    chunk_tokens = 64
+    pool = wl.random_bits(w.seed + 1, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, chunk_tokens)
+    descs, uniq = kvc.kvc_map_requests_shared(lay, tables)
+    assert uniq == len({int(b) for t in tables for b in t}) < sum(len(t) for t in tables)
+    total = sum(d[4] for d in descs)
+    assert total == uniq * g.bytes_per_block
+    staged = wl.random_bits(w.seed + 2, total)            # "chunks as read from storage"
+    staging = to_dev(staged)
+    tabs_dev = [to_dev(t) for t in tables]
+    launches0 = kvc.kvc_layout_launch_count(lay)
+    for ids_on_device in (0, 1):
+        pool_t.copy_(to_dev(pool))
+        slot_addrs, ids_addrs, nbs, off = [], [], [], 0
+        for (r, c, first, nb, nbytes) in descs:
+            slot_addrs.append(staging.data_ptr() + off)
+            base = tabs_dev[r].data_ptr() if ids_on_device else tables[r].ctypes.data
+            ids_addrs.append(base + 4 * first)
+            nbs.append(nb)
+            off += nbytes
+        ops = kvc.make_chunk_ops(slot_addrs, ids_addrs, nbs)
+        kvc.kvc_unpack_batch(lay, ops, ids_on_device)
+        torch.cuda.synchronize()
+        want = pool.copy()
+        off = 0
+        for (r, c, first, nb, nbytes) in descs:
+            orc.unpack_chunk(g, want, staged[off:off + nbytes], tables[r][first:first + nb])
+            off += nbytes
+        assert np.array_equal(pool_t.cpu().numpy(), want)
+    assert kvc.kvc_layout_launch_count(lay) - launches0 == 2
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+# ------------------------------------------------------------------ config 5 (reduced): ring streaming
+@pytest.mark.parametrize("kind", [kvc.KVC_RING_DEVICE, kvc.KVC_RING_HOST_MAPPED])
+def test_prefix_streamed_through_ring_equals_one_shot_pack(kind):
+    """A 2048-token prefix (8 chunks of 256 tokens) through a 3-slot ring while the copy stream
+    drains each slot to host memory: host bytes equal the oracle's pack of the whole prefix; then
+    the reverse (host -> ring -> unpack) restores a second pool."""
+    w = wl.WORKLOADS["8b_ring"]
+    g = dims_of(w.shape, 384)
+    pool = _pool_8b_384()
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 256)
+    src = wl.block_ids(w.seed, g.NB, 128)
+    dst = wl.block_ids(w.dst_seed, g.NB, 128)
+    descs = kvc.kvc_map_request(lay, len(src))
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    ring = kvc.kvc_staging_ring_create(cb, 3, kind)
+    host_out = torch.empty(len(descs) * cb, dtype=torch.uint8).pin_memory()
+    s_pack, s_copy = torch.cuda.Stream(), torch.cuda.Stream()
+    for (_, c, first, nb, nbytes) in descs:
+        slot, dptr, hptr = kvc.kvc_staging_ring_acquire(ring, timeout_us=5_000_000)
+        assert slot == c % 3
+        kvc.kvc_pack(lay, src[first:first + nb], dptr, cb, stream=s_pack)
+        kvc.kvc_staging_ring_commit(ring, slot, s_pack)
+        kvc.kvc_staging_ring_wait_filled(ring, slot, s_copy)
+        src_addr = dptr if kind == kvc.KVC_RING_DEVICE else hptr
+        kind_flag = cuda_rt.D2H if kind == kvc.KVC_RING_DEVICE else cuda_rt.H2H
+        cuda_rt.memcpy_async(host_out.data_ptr() + c * cb, src_addr, nbytes, kind_flag, s_copy)
+        kvc.kvc_staging_ring_release(ring, slot, s_copy)
+    torch.cuda.synchronize()
+    want = np.concatenate(orc.pack_request(g, pool, src, 256))
+    assert np.array_equal(host_out.numpy(), want)
+    in_flight, acquires, stalls = kvc.kvc_staging_ring_stats(ring)
+    assert acquires == len(descs)
+    # load direction: host -> ring slot -> unpack into other blocks
+    for (_, c, first, nb, nbytes) in descs:
+        slot, dptr, hptr = kvc.kvc_staging_ring_acquire(ring, timeout_us=5_000_000)
+        dst_addr = dptr if kind == kvc.KVC_RING_DEVICE else hptr
+        kind_flag = cuda_rt.H2D if kind == kvc.KVC_RING_DEVICE else cuda_rt.H2H
+        cuda_rt.memcpy_async(dst_addr, host_out.data_ptr() + c * cb, nbytes, kind_flag, s_copy)
+        kvc.kvc_staging_ring_commit(ring, slot, s_copy)       # here the copy stream is the producer
+        kvc.kvc_staging_ring_wait_filled(ring, slot, s_pack)
+        kvc.kvc_unpack(lay, dptr, dst[first:first + nb], cb, stream=s_pack)
+        kvc.kvc_staging_ring_release(ring, slot, s_pack)
+    torch.cuda.synchronize()
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, orc.pack_request(g, pool, src, 256), dst, 256)
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    kvc.kvc_staging_ring_destroy(ring)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
