@@ -24,9 +24,8 @@ import argparse
 import json
 import os
 import statistics
-import subprocess
 import sys
-import tempfile
+import threading
 import time
 from concurrent.futures import ThreadPoolExecutor
 
@@ -52,56 +51,59 @@ def measured_peak():
 
 
 # ------------------------------------------------------------------ clocks
-class ClockSampler:
-    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
-              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-              "clocks_event_reasons.sw_power_cap")
+class ClockSampler(threading.Thread):
+    """Reads SM clock and clock-event (throttle) reasons through NVML every ~10 ms while the
+    timed region runs; `summary(t0, t1)` keeps the samples taken inside that window."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
 
-    def __init__(self, gpu_index: int):
-        self.gpu, self.proc, self.path = gpu_index, None, None
+    def __init__(self, torch, cuda_index: int):
+        super().__init__(daemon=True)
+        self.samples, self._halt, self.h, self.nv = [], threading.Event(), None, None
+        self.sm_max = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            try:
+                uuid = "GPU-" + str(torch.cuda.get_device_properties(cuda_index).uuid)
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid)
+            except Exception:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(cuda_index)
+            self.nv = pynvml
+            self.sm_max = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.h = None
 
-    def start(self):
-        try:
-            fd, self.path = tempfile.mkstemp(suffix=".csv")
-            os.close(fd)
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
-                stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
-        except Exception:
-            self.proc = None
+    def run(self):
+        if self.h is None:
+            return
+        nv = self.nv
+        reasons_fn = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            nv.nvmlDeviceGetCurrentClocksThrottleReasons
+        while not self._halt.is_set():
+            try:
+                sm = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                rs = int(reasons_fn(self.h))
+                self.samples.append((time.perf_counter(), float(sm), rs))
+            except Exception:
+                pass
+            time.sleep(0.01)
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
-        if self.proc is None:
-            return out
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        try:
-            for line in open(self.path):
-                p = [x.strip() for x in line.split(",")]
-                if len(p) < 7:
-                    continue
-                try:
-                    sm.append(float(p[0]))
-                    mx.append(float(p[1]))
-                except ValueError:
-                    continue
-                for nm, v in zip(names, p[3:7]):
-                    if v.lower().startswith("active"):
-                        reasons.add(nm)
-            os.unlink(self.path)
-        except Exception:
-            pass
-        if sm:
-            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), samples=len(sm))
-        out["reasons"] = sorted(reasons)
+    def summary(self, t0: float, t1: float):
+        self._halt.set()
+        self.join(timeout=2)
+        inside = [x for x in self.samples if t0 <= x[0] <= t1]
+        window = "timed region"
+        if len(inside) < 3:   # a very short timed region: fall back to everything sampled under load
+            inside, window = self.samples, "warm-up + timed region"
+        out = {"sm_mhz": None, "sm_max_mhz": self.sm_max, "reasons": [], "samples": len(inside),
+               "window": window}
+        if inside:
+            out["sm_mhz"] = statistics.median(x[1] for x in inside)
+            bits = 0
+            for x in inside:
+                bits |= x[2]
+            out["reasons"] = sorted(v for k, v in self.REASONS.items() if bits & k)
         return out
 
 
@@ -220,7 +222,8 @@ def run_ours(args, rank, world, local_rank):
 
     w = wl.WORKLOADS[args.workload]
     s = w.shape
-    NB, n = w.pool_blocks, w.request_blocks
+    NB = args.pool_blocks or w.pool_blocks
+    n = args.request_blocks or w.request_blocks
     one_way = n * s.bytes_per_block
     pool = wl.random_bits_cuda(w.seed + 17 * rank, NB * s.bytes_per_block, dev)
     src = wl.block_ids(w.seed, NB, n)
@@ -228,7 +231,8 @@ def run_ours(args, rank, world, local_rank):
     staging = torch.empty(one_way, dtype=torch.uint8, device=dev)
     lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, args.chunk_tokens)
     kvc.kvc_layout_set_tuning(lay, variant=args.variant, order=args.order,
-                              tile_bytes=args.tile_bytes, stages=args.stages)
+                              tile_bytes=args.tile_bytes, stages=args.stages, lag=args.lag,
+                              max_ctas=args.max_ctas)
     stream = torch.cuda.current_stream()
 
     def step(evs=None):
@@ -243,21 +247,22 @@ def run_ours(args, rank, world, local_rank):
         if evs:
             evs[2].record(stream)
 
+    sampler = ClockSampler(torch, local_rank)
+    sampler.start()
     for _ in range(args.warmup):
         step()
     barrier()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     launches0 = kvc.kvc_layout_launch_count(lay)
     barrier()
     t0 = time.perf_counter()
     for i in range(args.steps):
         step(evs[i])
     barrier()
-    wall = time.perf_counter() - t0
+    t1 = time.perf_counter()
+    wall = t1 - t0
     launches = kvc.kvc_layout_launch_count(lay) - launches0
-    clocks = sampler.stop()
+    clocks = sampler.summary(t0, t1)
     total_ms = evs[0][0].elapsed_time(evs[-1][2])
     pack_ms = [e[0].elapsed_time(e[1]) for e in evs]
     unpack_ms = [e[1].elapsed_time(e[2]) for e in evs]
@@ -307,7 +312,7 @@ def run_ours(args, rank, world, local_rank):
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": {"workload": args.workload, "kv_shape": "L32 H8 D128 B16 2-byte", "pool_blocks": NB,
-                   "request_tokens": w.request_tokens, "request_blocks": n,
+                   "request_tokens": n * s.B, "request_blocks": n,
                    "chunk_tokens": args.chunk_tokens, "bytes_each_way": one_way,
                    "launch": "one kvc_pack_batch + one kvc_unpack_batch per step",
                    "l2": "inputs larger than L2 (9.8 GiB read and 9.8 GiB written per launch)",
@@ -442,6 +447,12 @@ def main():
     ap.add_argument("--order", type=int, default=0)
     ap.add_argument("--tile-bytes", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--lag", type=int, default=0)
+    ap.add_argument("--max-ctas", type=int, default=0)
+    ap.add_argument("--pool-blocks", type=int, default=0,
+                    help="override the workload's pool size (small cases for profiler captures)")
+    ap.add_argument("--request-blocks", type=int, default=0,
+                    help="override the workload's request length in blocks")
     ap.add_argument("--ring-slots", type=int, default=8)
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")

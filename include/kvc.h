@@ -114,6 +114,9 @@ typedef struct {
                             leaves SMs to a concurrent compute stream */
     uint32_t tile_bytes; /* bytes of one slab moved per work item (0 = default); multiple of 16 */
     uint32_t stages;     /* BULK: shared-memory stages per thread block (0 = default) */
+    uint32_t ctas_per_sm; /* BULK: resident thread blocks per SM, 1..4 (0 = default) */
+    uint32_t l2_hint;    /* BULK: 0 = default, 1 = no L2 priority hint, 2 = evict-first on loads and stores */
+    uint32_t lag;        /* BULK: loads issued ahead of the store they feed, 1..stages-2 (0 = default) */
 } kvc_tuning;
 /* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */
 kvc_status kvc_layout_set_tuning(kvc_layout *layout, const kvc_tuning *tuning);

@@ -223,6 +223,32 @@ __device__ __forceinline__ void bulk_store(uint64_t dst, uint32_t src_smem, uint
                  : "memory");
 }
 
+__device__ __forceinline__ uint64_t policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+__device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, uint64_t src, uint32_t bytes,
+                                               uint32_t bar, uint64_t pol)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1], %2, [%3], %4;" ::"r"(dst_smem),
+        "l"(src), "r"(bytes), "r"(bar), "l"(pol)
+        : "memory");
+}
+
+__device__ __forceinline__ void bulk_store_hint(uint64_t dst, uint32_t src_smem, uint32_t bytes,
+                                                uint64_t pol)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group.L2::cache_hint [%0], [%1], %2, %3;" ::
+                     "l"(dst),
+                 "r"(src_smem), "r"(bytes), "l"(pol)
+                 : "memory");
+}
+
 __device__ __forceinline__ void bulk_commit()
 {
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
@@ -269,6 +295,8 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
     }
     __syncwarp();
 
+    const bool hint = a.l2_evict_first != 0;
+    const uint64_t pol = policy_evict_first();
     bool ok = true;          // lane 0: no wait has expired
     uint32_t loads_done = 0; // lane 0: items whose load was issued (for the drain on failure)
     uint32_t stores_done = 0;
@@ -299,9 +327,13 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
                     st_dst[s] = DIR == KVC_DIR_PACK ? slot : pool;
                     st_len[s] = len;
                     mbar_expect_tx(bar, len);
-                    if (len)
-                        bulk_load(smem_u32(data + (size_t)s * tile),
-                                  DIR == KVC_DIR_PACK ? pool : slot, len, bar);
+                    if (len) {
+                        const uint64_t from = DIR == KVC_DIR_PACK ? pool : slot;
+                        if (hint)
+                            bulk_load_hint(smem_u32(data + (size_t)s * tile), from, len, bar, pol);
+                        else
+                            bulk_load(smem_u32(data + (size_t)s * tile), from, len, bar);
+                    }
                     loads_done = k + 1;
                 }
                 if (k >= lag) {
@@ -311,7 +343,10 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
                         const uint32_t l2 = st_len[s];
                         if (l2) {
                             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                            bulk_store(st_dst[s], smem_u32(data + (size_t)s * tile), l2);
+                            if (hint)
+                                bulk_store_hint(st_dst[s], smem_u32(data + (size_t)s * tile), l2, pol);
+                            else
+                                bulk_store(st_dst[s], smem_u32(data + (size_t)s * tile), l2);
                         }
                         bulk_commit();
                         stores_done = m + 1;

@@ -33,6 +33,9 @@ kvc_status ensure_device(kvc_layout *lay)
         return KVC_ERR_CUDA;
     if (cudaHostAlloc(&lay->h_status, 2 * sizeof(uint32_t), cudaHostAllocDefault) != cudaSuccess)
         return KVC_ERR_NOMEM;
+    if (cudaStreamCreateWithFlags(&lay->upload_stream, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&lay->upload_done, cudaEventDisableTiming) != cudaSuccess)
+        return KVC_ERR_CUDA;
     if (!lay->plane_ptrs.empty()) {
         size_t bytes = lay->plane_ptrs.size() * sizeof(void *);
         if (cudaMalloc(&lay->d_plane_table, bytes) != cudaSuccess)
@@ -84,14 +87,21 @@ kvc_status make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe, Kv
     tile = (uint32_t)std::min<uint64_t>(tile, lay->slab_bytes);
     uint32_t stages = 0, lag = 0, smem = 0;
     if (variant == KVC_VARIANT_BULK) {
-        const uint32_t room = (uint32_t)lay->max_smem_optin - KVC_BULK_SMEM_HEADER;
+        const uint32_t per_sm = t.ctas_per_sm ? t.ctas_per_sm : 1u;
+        // every resident block also costs 1 KiB of system-reserved shared memory
+        const uint32_t room = ((uint32_t)lay->max_smem_optin + 1024u) / per_sm - 1024u - KVC_BULK_SMEM_HEADER;
         if (tile > room / 2)
             tile = (room / 2) & ~15u;
-        stages = t.stages ? t.stages : KVC_BULK_MAX_STAGES;
+        stages = t.stages ? t.stages : KVC_BULK_DEFAULT_STAGES;
         stages = std::min<uint32_t>(std::min<uint32_t>(stages, room / tile), KVC_BULK_MAX_STAGES);
         if (stages < 2)
             return KVC_ERR_INVALID_ARG;
-        lag = stages - 2;  // one store may still read its stage when the stage after next is reloaded
+        // a stage is reloaded only when at most one newer store still reads shared memory, so
+        // loads can run at most stages-2 items ahead of the stores
+        lag = stages - 2;
+        const uint32_t want_lag = t.lag ? t.lag : KVC_BULK_DEFAULT_LAG;
+        if (want_lag < lag)
+            lag = want_lag;
         smem = KVC_BULK_SMEM_HEADER + stages * tile;
     } else {
         // 32-byte vectors need every address the kernel forms to be 32-byte aligned
@@ -116,9 +126,10 @@ kvc_status make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe, Kv
     a->order = t.order ? t.order : KVC_ORDER_PLANE_MAJOR;
     a->stages = stages;
     a->lag = lag;
+    a->l2_evict_first = t.l2_hint == 2;
     a->status = lay->d_status;
     uint64_t grid = variant == KVC_VARIANT_BULK
-                        ? (uint64_t)lay->sm_count
+                        ? (uint64_t)lay->sm_count * (t.ctas_per_sm ? t.ctas_per_sm : 1u)
                         : (uint64_t)lay->sm_count * (uint64_t)lay->vec_blocks_per_sm;
     if (t.max_ctas)
         grid = std::min<uint64_t>(grid, t.max_ctas);
@@ -314,9 +325,13 @@ kvc_status copy_batch(kvc_layout *lay, int dir, const kvc_chunk_op *ops, uint32_
             }
         }
     }
+    // The table travels on the handle's own stream so that the copy overlaps whatever still runs
+    // on the caller's stream; the kernel waits for it through an event.
     cudaStream_t st = (cudaStream_t)stream;
-    if (cudaMemcpyAsync(ar->dev, ar->host, n_ent * sizeof(KvcEnt), cudaMemcpyHostToDevice, st) !=
-        cudaSuccess)
+    if (cudaMemcpyAsync(ar->dev, ar->host, n_ent * sizeof(KvcEnt), cudaMemcpyHostToDevice,
+                        lay->upload_stream) != cudaSuccess ||
+        cudaEventRecord(lay->upload_done, lay->upload_stream) != cudaSuccess ||
+        cudaStreamWaitEvent(st, lay->upload_done, 0) != cudaSuccess)
         return KVC_ERR_CUDA;
     a.table = ar->dev;
     if (kvc_launch_copy(dir, plan.variant, a, plan.grid, plan.smem, st) != cudaSuccess)
@@ -414,6 +429,8 @@ kvc_status kvc_layout_create(const kvc_layout_desc *d, kvc_layout **out)
     lay->d_status = nullptr;
     lay->h_status = nullptr;
     lay->next_arena = 0;
+    lay->upload_stream = nullptr;
+    lay->upload_done = nullptr;
     lay->launches = 0;
     lay->seen_stamp = 0;
     *out = lay;
@@ -435,6 +452,10 @@ kvc_status kvc_layout_destroy(kvc_layout *lay)
         if (ar.dev)
             cudaFree(ar.dev);
     }
+    if (lay->upload_done)
+        cudaEventDestroy(lay->upload_done);
+    if (lay->upload_stream)
+        cudaStreamDestroy(lay->upload_stream);
     if (lay->d_plane_table)
         cudaFree((void *)lay->d_plane_table);
     if (lay->d_status)
@@ -473,6 +494,8 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
     if (t->tile_bytes % 16)
         return KVC_ERR_INVALID_ARG;
     if (t->stages == 1 || t->stages > KVC_BULK_MAX_STAGES)
+        return KVC_ERR_INVALID_ARG;
+    if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES)
         return KVC_ERR_INVALID_ARG;
     lay->tuning = *t;
     return KVC_OK;

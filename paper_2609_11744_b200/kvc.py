@@ -49,7 +49,8 @@ class kvc_layout_desc(ctypes.Structure):
 class kvc_tuning(ctypes.Structure):
     _fields_ = [("variant", ctypes.c_uint32), ("order", ctypes.c_uint32),
                 ("max_ctas", ctypes.c_uint32), ("tile_bytes", ctypes.c_uint32),
-                ("stages", ctypes.c_uint32)]
+                ("stages", ctypes.c_uint32), ("ctas_per_sm", ctypes.c_uint32),
+                ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32)]
 
 
 class kvc_chunk_desc(ctypes.Structure):
@@ -264,8 +265,9 @@ def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
     return lib().kvc_layout_num_chunks(layout.handle, n_blocks)
 
 
-def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0) -> None:
-    t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages)
+def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
+                          ctas_per_sm=0, l2_hint=0, lag=0) -> None:
+    t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
 
 
