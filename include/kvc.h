@@ -51,7 +51,8 @@ typedef enum {
     KVC_ERR_CUDA = 6,         /* a CUDA runtime call failed (no device, launch error, ...) */
     KVC_ERR_WOULD_BLOCK = 7,  /* ring: no free slot and timeout_us == 0 */
     KVC_ERR_TIMEOUT = 8,      /* ring: no free slot before the deadline */
-    KVC_ERR_STATE = 9         /* ring: call does not fit the slot's state */
+    KVC_ERR_STATE = 9,        /* ring: call does not fit the slot's state */
+    KVC_ERR_TOO_LARGE = 10    /* more work than a fixed-capacity entry point can take in one call */
 } kvc_status;
 
 const char *kvc_status_str(kvc_status s);
@@ -188,6 +189,29 @@ kvc_status kvc_unpack_batch(kvc_layout *layout, const kvc_chunk_op *ops, uint32_
  * Either pointer may be NULL. */
 kvc_status kvc_poll_device_status(kvc_layout *layout, void *stream, uint32_t *n_skipped,
                                   uint32_t *n_wait_expired);
+
+/* Batched pack for callers that must not allocate (the paper has no counterpart: this is a
+ * deployment aid).  Serving engines that gave every spare byte of device memory to their KV pool,
+ * scheduler threads that cannot afford the device-wide stall an allocation may cause, and code
+ * running under an allocator policy that forbids raw cudaMalloc can all still offload KV blocks
+ * through this call: it allocates and frees nothing, on the device or on the host, and neither
+ * does anything it calls.  Same result as kvc_pack_batch with ids_on_device == 0 (ids must be in
+ * HOST memory; they are fully validated before anything is enqueued).
+ * The id table, the plane-pointer table and the status words live in a fixed array inside the
+ * library image (about 264 KiB of device memory on every GPU that loads the library, held until
+ * the process exits).  Limits: at most KVC_STATIC_MAX_BLOCKS blocks per call, summed over the
+ * ops, and at most KVC_STATIC_MAX_PLANES planes for layouts given as plane pointers; beyond
+ * either the call returns KVC_ERR_TOO_LARGE and enqueues nothing.
+ * The first call on a device looks up the array's device address and the device's limits; make
+ * that first call outside any stream capture.  Every call shares the one array, which keeps the
+ * previous call's contents (the call clears what must start at zero): calls whose GPU work can
+ * overlap -- different streams, or several host threads -- race on it, so serialise them on
+ * one stream.  The handle's device status counters are not touched by this call.
+ * Errors: INVALID_ARG, ALIGNMENT, OUT_OF_RANGE, TOO_LARGE, CUDA. */
+#define KVC_STATIC_MAX_BLOCKS 8192u
+#define KVC_STATIC_MAX_PLANES 1024u
+kvc_status kvc_pack_batch_static(kvc_layout *layout, const kvc_chunk_op *ops, uint32_t n_ops,
+                                 void *stream);
 
 /* Number of kernel launches issued through this handle so far. */
 uint64_t kvc_layout_launch_count(const kvc_layout *layout);

@@ -103,4 +103,14 @@ struct kvc_layout {
     uint32_t seen_stamp;
 };
 
+
+// Launch shape chosen by the host for one call.
+struct KvcPlan {
+    int variant;
+    uint32_t grid, smem, stages, lag;
+};
+// Implemented in kvc_layout.cu.  Reads the handle's tuning and the device limits cached in it.
+kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe, KvcLaunch *a,
+                         KvcPlan *plan);
+
 #endif

@@ -48,14 +48,11 @@ kvc_status ensure_device(kvc_layout *lay)
     return KVC_OK;
 }
 
-// Fills the geometry and the launch shape that do not depend on the ids.
-struct Plan {
-    int variant;
-    uint32_t grid, smem, stages, lag;
-};
+}  // namespace
 
-kvc_status make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe, KvcLaunch *a,
-                     Plan *plan)
+// Fills the geometry and the launch shape that do not depend on the ids.
+kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe, KvcLaunch *a,
+                         KvcPlan *plan)
 {
     const kvc_tuning &t = lay->tuning;
     KvcGeom &g = a->g;
@@ -142,6 +139,8 @@ kvc_status make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe, Kv
     return KVC_OK;
 }
 
+namespace {
+
 // Range check, and for unpack a duplicate check across the whole call, on host-resident ids.
 kvc_status check_host_ids(kvc_layout *lay, const int32_t *ids, uint32_t n, bool reject_dup)
 {
@@ -207,8 +206,8 @@ kvc_status copy_one(kvc_layout *lay, int dir, const int32_t *ids, uint32_t n_blo
         return s;
     KvcLaunch a;
     memset(&a, 0, sizeof(a));
-    Plan plan;
-    s = make_plan(lay, n_blocks, slot, &a, &plan);
+    KvcPlan plan;
+    s = kvc_make_plan(lay, n_blocks, slot, &a, &plan);
     if (s != KVC_OK)
         return s;
     a.slot = (uint64_t)(uintptr_t)slot;
@@ -301,8 +300,8 @@ kvc_status copy_batch(kvc_layout *lay, int dir, const kvc_chunk_op *ops, uint32_
         return s;
     KvcLaunch a;
     memset(&a, 0, sizeof(a));
-    Plan plan;
-    s = make_plan(lay, n_ent, probe, &a, &plan);
+    KvcPlan plan;
+    s = kvc_make_plan(lay, n_ent, probe, &a, &plan);
     if (s != KVC_OK)
         return s;
     KvcArena *ar = nullptr;
@@ -360,6 +359,7 @@ const char *kvc_status_str(kvc_status s)
     case KVC_ERR_WOULD_BLOCK: return "no free staging slot";
     case KVC_ERR_TIMEOUT: return "timed out waiting for a staging slot";
     case KVC_ERR_STATE: return "call does not fit the slot's state";
+    case KVC_ERR_TOO_LARGE: return "more blocks or planes than this fixed-capacity entry point takes per call";
     }
     return "unknown status";
 }

@@ -21,7 +21,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkvc.so")
 
 KVC_OK, KVC_ERR_INVALID_ARG, KVC_ERR_OUT_OF_RANGE, KVC_ERR_ALIGNMENT, KVC_ERR_CONFLICT, \
-    KVC_ERR_NOMEM, KVC_ERR_CUDA, KVC_ERR_WOULD_BLOCK, KVC_ERR_TIMEOUT, KVC_ERR_STATE = range(10)
+    KVC_ERR_NOMEM, KVC_ERR_CUDA, KVC_ERR_WOULD_BLOCK, KVC_ERR_TIMEOUT, KVC_ERR_STATE, \
+    KVC_ERR_TOO_LARGE = range(11)
 KVC_VARIANT_AUTO, KVC_VARIANT_VEC, KVC_VARIANT_BULK = 0, 1, 2
 KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR = 0, 1, 2
 KVC_RING_DEVICE, KVC_RING_HOST_MAPPED = 0, 1
@@ -110,6 +111,7 @@ def lib() -> ctypes.CDLL:
         "kvc_unpack": (ci, [vp, vp, u64, vp, u32, ci, vp]),
         "kvc_pack_batch": (ci, [vp, vp, u32, ci, vp]),
         "kvc_unpack_batch": (ci, [vp, vp, u32, ci, vp]),
+        "kvc_pack_batch_static": (ci, [vp, vp, u32, vp]),
         "kvc_poll_device_status": (ci, [vp, vp, P(u32), P(u32)]),
         "kvc_layout_launch_count": (u64, [vp]),
         "kvc_staging_ring_create": (ci, [u64, u32, ci, vp, u64, P(vp)]),
@@ -356,6 +358,20 @@ def kvc_pack_batch(layout, ops: np.ndarray, ids_on_device: int = 0, stream=None)
 
 def kvc_unpack_batch(layout, ops: np.ndarray, ids_on_device: int = 0, stream=None) -> None:
     _batch("kvc_unpack_batch", layout, ops, ids_on_device, stream)
+
+
+KVC_STATIC_MAX_BLOCKS, KVC_STATIC_MAX_PLANES = 8192, 1024
+
+
+def kvc_pack_batch_static(layout, ops: np.ndarray, stream=None) -> None:
+    """kvc_pack_batch for callers that must not allocate device memory (an engine whose KV pool
+    already owns all of it, a thread that cannot tolerate an allocation's stall).  Host-resident
+    ids only, at most KVC_STATIC_MAX_BLOCKS blocks per call; calls share one fixed scratch area
+    inside the library, so keep them on one stream."""
+    if ops.dtype != CHUNK_OP_DTYPE or not ops.flags.c_contiguous:
+        raise TypeError("ops must be a contiguous array of CHUNK_OP_DTYPE")
+    _check(lib().kvc_pack_batch_static(layout.handle, ops.ctypes.data, len(ops), _stream(stream)),
+           "kvc_pack_batch_static")
 
 
 def kvc_poll_device_status(layout, stream=None) -> Tuple[int, int]:
