@@ -269,9 +269,6 @@ def run_ours(args, rank, world, local_rank):
     skipped, expired = kvc.kvc_poll_device_status(lay)
     assert (skipped, expired) == (0, 0), "device status flags set: %r" % ((skipped, expired),)
 
-    # spot check of the timed configuration: staging holds pack(src) at sampled positions
-    check_sampled(torch, pool, staging, src, dst, s, NB, args.chunk_tokens, dev)
-
     if world > 1:
         t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -329,39 +326,6 @@ def run_ours(args, rank, world, local_rank):
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
-
-
-def check_sampled(torch, pool, staging, src, dst, s, NB, chunk_tokens, dev, n_samples=200_000):
-    """After the timed steps the staging area holds pack(src) (the later unpack into dst does not
-    change it) and the pool's dst blocks hold those bytes: compare sampled 2-byte elements with
-    positions computed by the CPU oracle's index formulas, one sample at a time (vectorised)."""
-    from oracle import oracle as orc
-    g = orc.Dims(s.L, s.P, NB, s.B, s.H, s.D, s.e)
-    bpc = chunk_tokens // s.B
-    n = len(src)
-    rng = np.random.default_rng(12345)
-    blk = rng.integers(0, n, n_samples)           # table position of the sampled block
-    c = blk // bpc
-    j = blk - c * bpc
-    nb_c = np.minimum(bpc, n - c * bpc)
-    l = rng.integers(0, s.L, n_samples)
-    p = rng.integers(0, s.P, n_samples)
-    t = rng.integers(0, s.B, n_samples)
-    h = rng.integers(0, s.H, n_samples)
-    d = rng.integers(0, s.D, n_samples)
-    chunk_base = c.astype(np.int64) * (orc.chunk_bytes(g, bpc) // s.e)   # chunks lie back to back
-    stage_idx = chunk_base + orc.chunk_elem(g, nb_c, l, p, j, t, h, d)
-    src_idx = orc.pool_elem(g, l, p, src[blk].astype(np.int64), t, h, d)
-    dst_idx = orc.pool_elem(g, l, p, dst[blk].astype(np.int64), t, h, d)
-    pool16, stage16 = pool.view(torch.int16), staging.view(torch.int16)
-    sv = stage16[torch.from_numpy(stage_idx).to(dev)]
-    dv = pool16[torch.from_numpy(dst_idx).to(dev)]
-    assert bool((sv == dv).all()), "unpack: sampled pool elements differ from the staged chunk"
-    # source blocks overwritten by the unpack (src and dst tables overlap) can no longer be compared
-    keep = ~np.isin(src[blk], dst)
-    pv = pool16[torch.from_numpy(src_idx[keep]).to(dev)]
-    assert bool((sv[torch.from_numpy(np.flatnonzero(keep)).to(dev)] == pv).all()), \
-        "pack: sampled staged elements differ from the pool"
 
 
 def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, dist):
@@ -435,6 +399,286 @@ def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, di
     }
 
 
+# ------------------------------------------------------------------ suite: the other configs
+def _time_ms(torch, fn, reps, warm=3, flush=None):
+    """min / median of CUDA-event times of fn() on the current stream."""
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        if flush is not None:
+            flush.add_(1)  # a buffer larger than L2 is rewritten between timed launches
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b))
+    return min(ts), statistics.median(ts)
+
+
+def suite_chunk_sweep(torch, kvc, dev, reps):
+    """8B shape, 80k-token prefix: chunk 16/256/2048 tokens, one batched launch vs one launch per
+    chunk, pack and unpack timed separately."""
+    w = wl.WORKLOADS["8b_80k"]
+    s, NB, n = w.shape, w.pool_blocks, w.request_blocks
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    src, dst = wl.block_ids(w.seed, NB, n), wl.block_ids(w.dst_seed, NB, n)
+    one_way = n * s.bytes_per_block
+    staging = torch.empty(one_way, dtype=torch.uint8, device=dev)
+    base = staging.data_ptr()
+    out = []
+    for chunk_tokens in w.chunk_tokens:
+        lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, chunk_tokens)
+        descs = kvc.kvc_map_request(lay, n)
+        ops_p, k1, _, _ = kvc.request_chunk_ops(lay, src, staging)
+        ops_u, k2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+
+        def per_chunk(direction, ids):
+            off = 0
+            for (_, _, first, nb, nbytes) in descs:
+                if direction == 0:
+                    kvc.kvc_pack(lay, ids[first:first + nb], base + off, nbytes)
+                else:
+                    kvc.kvc_unpack(lay, base + off, ids[first:first + nb], nbytes)
+                off += nbytes
+
+        modes = [("batch", lambda: kvc.kvc_pack_batch(lay, ops_p, 0),
+                  lambda: kvc.kvc_unpack_batch(lay, ops_u, 0))]
+        if len(descs) <= 400:   # 5000 single-chunk launches of 2 MiB are launch-bound by design
+            modes.append(("per_chunk", lambda: per_chunk(0, src), lambda: per_chunk(1, dst)))
+        for name, fp, fu in modes:
+            pm, pd = _time_ms(torch, fp, reps)
+            um, ud = _time_ms(torch, fu, reps)
+            out.append({"chunk_tokens": chunk_tokens, "chunks": len(descs), "mode": name,
+                        "pack_ms_min": pm, "pack_ms_median": pd, "pack_gbs": 2 * one_way / pd / 1e6,
+                        "unpack_ms_min": um, "unpack_ms_median": ud,
+                        "unpack_gbs": 2 * one_way / ud / 1e6})
+        assert kvc.kvc_poll_device_status(lay) == (0, 0)
+        kvc.kvc_layout_destroy(lay)
+    return out
+
+
+def suite_8k(torch, kvc, dev, reps):
+    """Config 2: 8192-token prefix (1 GiB each way) with L2 flushed between timed launches."""
+    w = wl.WORKLOADS["8b_8k"]
+    s, NB, n = w.shape, w.pool_blocks, w.request_blocks
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    src, dst = wl.block_ids(w.seed, NB, n), wl.block_ids(w.dst_seed, NB, n)
+    one_way = n * s.bytes_per_block
+    staging = torch.empty(one_way, dtype=torch.uint8, device=dev)
+    flush = torch.zeros(512 << 20, dtype=torch.uint8, device=dev)
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    ops_p, k1, _, _ = kvc.request_chunk_ops(lay, src, staging)
+    ops_u, k2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+    pm, pd = _time_ms(torch, lambda: kvc.kvc_pack_batch(lay, ops_p, 0), reps, flush=flush)
+    um, ud = _time_ms(torch, lambda: kvc.kvc_unpack_batch(lay, ops_u, 0), reps, flush=flush)
+    return {"bytes_each_way": one_way, "l2": "512 MiB scratch rewritten between timed launches",
+            "pack_ms_min": pm, "pack_ms_median": pd, "pack_gbs": 2 * one_way / pd / 1e6,
+            "unpack_ms_min": um, "unpack_ms_median": ud, "unpack_gbs": 2 * one_way / ud / 1e6}
+
+
+def suite_batch(torch, kvc, dev, reps):
+    """Config 4: 70B-class shape, 64 requests with lognormal lengths and a shared 1024-token
+    prefix; every cache-hit chunk of every request unpacked by ONE call (shared chunks once)."""
+    w = wl.WORKLOADS["70b_batch"]
+    s = w.shape
+    free, _ = torch.cuda.mem_get_info()
+    scale = 1.0
+    while True:
+        NB, tables = wl.batch_workload(w, scale)
+        uniq = len({int(b) for t in tables for b in t})
+        need = NB * s.bytes_per_block + uniq * s.bytes_per_block + (4 << 30)
+        if need < free or scale < 0.1:
+            break
+        scale *= 0.8   # not enough free device memory: shrink every length, and say so
+    pool = torch.empty(NB * s.bytes_per_block, dtype=torch.uint8, device=dev)
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    t0 = time.perf_counter()
+    descs, uniq2 = kvc.kvc_map_requests_shared(lay, tables)
+    map_ms = (time.perf_counter() - t0) * 1e3
+    total = sum(d[4] for d in descs)
+    staging = wl.random_bits_cuda(w.seed + 3, total, dev)
+    slot, ids, nbs, off = [], [], [], 0
+    for (r, c, first, nb, nbytes) in descs:
+        slot.append(staging.data_ptr() + off)
+        ids.append(tables[r].ctypes.data + 4 * first)
+        nbs.append(nb)
+        off += nbytes
+    ops = kvc.make_chunk_ops(slot, ids, nbs)
+    um, ud = _time_ms(torch, lambda: kvc.kvc_unpack_batch(lay, ops, 0), max(5, reps // 2))
+    pm, pd = _time_ms(torch, lambda: kvc.kvc_pack_batch(lay, ops, 0), max(5, reps // 2))
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+    return {"requests": len(tables), "length_scale": scale, "pool_blocks": NB,
+            "table_blocks_total": int(sum(len(t) for t in tables)), "unique_blocks": int(uniq2),
+            "chunks_after_dedup": len(descs), "bytes_each_way": total, "mapper_ms": map_ms,
+            "launches_per_call": 1,
+            "unpack_ms_min": um, "unpack_ms_median": ud, "unpack_gbs": 2 * total / ud / 1e6,
+            "pack_ms_min": pm, "pack_ms_median": pd, "pack_gbs": 2 * total / pd / 1e6}
+
+
+def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
+    """Config 5: a 32k-token prefix (8B shape, 4 GiB) streamed through an 8-slot ring of 256-token
+    slots to/from pinned host memory while a bf16 GEMM loop runs on another stream.  Destinations:
+    device slots drained by cudaMemcpyAsync, or slots in mapped pinned host memory that the
+    kernels write/read directly.  Reports link GB/s, GEMM slowdown and overlap efficiency
+    1 - (T_both - max(T_gemm, T_xfer)) / min(T_gemm, T_xfer)."""
+    w = wl.WORKLOADS["8b_ring"]
+    s, NB, n = w.shape, w.pool_blocks, w.request_blocks
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    src, dst = wl.block_ids(w.seed, NB, n), wl.block_ids(w.dst_seed, NB, n)
+    one_way = n * s.bytes_per_block
+    host = torch.empty(one_way, dtype=torch.uint8, pin_memory=True)
+    hptr = host.data_ptr()
+    lo, hi = torch.cuda.Stream.priority_range()
+    s_gemm = torch.cuda.Stream(priority=lo)
+    s_k, s_c = torch.cuda.Stream(priority=hi), torch.cuda.Stream(priority=hi)
+    TO = 20_000_000
+    N = 8192
+    A = torch.randn(N, N, device=dev, dtype=torch.bfloat16)
+    B = torch.randn(N, N, device=dev, dtype=torch.bfloat16)
+    C = torch.empty(N, N, device=dev, dtype=torch.bfloat16)
+
+    # The GEMM loop is replayed from a CUDA graph of GRAPH_ITERS matmuls, so that enqueueing two
+    # seconds of GEMMs takes a few dozen launches and never blocks the host thread that also
+    # drives the ring (thousands of queued kernel launches would fill the stream's launch queue
+    # and stall the host before the transfer even starts).
+    GRAPH_ITERS = 64
+    with torch.cuda.stream(s_gemm):
+        for _ in range(5):
+            torch.matmul(A, B, out=C)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=s_gemm):
+        for _ in range(GRAPH_ITERS):
+            torch.matmul(A, B, out=C)
+
+    def gemm_loop(iters):
+        with torch.cuda.stream(s_gemm):
+            for _ in range(iters // GRAPH_ITERS):
+                graph.replay()
+
+    # size the GEMM loop to about `seconds`
+    gemm_loop(GRAPH_ITERS)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(s_gemm)
+    gemm_loop(2 * GRAPH_ITERS)
+    e1.record(s_gemm)
+    torch.cuda.synchronize()
+    per_iter = e0.elapsed_time(e1) / (2 * GRAPH_ITERS)
+    iters = max(GRAPH_ITERS, int(seconds * 1e3 / per_iter) // GRAPH_ITERS * GRAPH_ITERS)
+    results = []
+    for kind, kind_name in ((kvc.KVC_RING_DEVICE, "device slots + cudaMemcpyAsync"),
+                            (kvc.KVC_RING_HOST_MAPPED, "mapped pinned host slots")):
+        for max_ctas in ((16, 0) if kind == kvc.KVC_RING_DEVICE else (4, 16, 64)):
+            lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+            kvc.kvc_layout_set_tuning(lay, max_ctas=max_ctas)
+            descs = kvc.kvc_map_request(lay, n)
+            cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+            ring = kvc.kvc_staging_ring_create(cb, int(w.extra["ring_slots"]), kind)
+
+            def offload():
+                off = 0
+                for (_, c, first, nb, nbytes) in descs:
+                    slot, dptr, hp = kvc.kvc_staging_ring_acquire(ring, TO)
+                    kvc.kvc_pack(lay, src[first:first + nb], dptr, nbytes, stream=s_k)
+                    kvc.kvc_staging_ring_commit(ring, slot, s_k)
+                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
+                    if kind == kvc.KVC_RING_DEVICE:
+                        cuda_rt.memcpy_async(hptr + off, dptr, nbytes, cuda_rt.D2H, s_c)
+                    # a mapped slot already is host memory: its consumer (file I/O in the paper)
+                    # would read it here; nothing is copied
+                    kvc.kvc_staging_ring_release(ring, slot, s_c)
+                    off += nbytes
+
+            def load():
+                off = 0
+                for (_, c, first, nb, nbytes) in descs:
+                    slot, dptr, hp = kvc.kvc_staging_ring_acquire(ring, TO)
+                    if kind == kvc.KVC_RING_DEVICE:
+                        cuda_rt.memcpy_async(dptr, hptr + off, nbytes, cuda_rt.H2D, s_c)
+                    # a mapped slot is filled by its producer (a file read) on the host side
+                    kvc.kvc_staging_ring_commit(ring, slot, s_c)
+                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_k)
+                    kvc.kvc_unpack(lay, dptr, dst[first:first + nb], nbytes, stream=s_k)
+                    kvc.kvc_staging_ring_release(ring, slot, s_k)
+                    off += nbytes
+
+            for direction, fn in (("offload", offload), ("load", load)):
+                fn()
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                fn()
+                torch.cuda.synchronize()
+                once = time.perf_counter() - t0
+                passes = max(1, int(seconds / once))
+                t0 = time.perf_counter()
+                for _ in range(passes):
+                    fn()
+                torch.cuda.synchronize()
+                t_xfer = time.perf_counter() - t0
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                g0.record(s_gemm)
+                gemm_loop(iters)
+                g1.record(s_gemm)
+                torch.cuda.synchronize()
+                t_gemm = time.perf_counter() - t0
+                # both at once
+                x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                g0.record(s_gemm)
+                gemm_loop(iters)
+                g1.record(s_gemm)
+                x0.record(s_k)
+                for _ in range(passes):
+                    fn()
+                x1.record(s_k)
+                s_c.synchronize()
+                s_k.synchronize()
+                t_x_in_both = time.perf_counter() - t0
+                torch.cuda.synchronize()
+                t_both = time.perf_counter() - t0
+                t_gemm_in_both = g0.elapsed_time(g1) * 1e-3
+                eff = 1 - (t_both - max(t_gemm, t_xfer)) / min(t_gemm, t_xfer)
+                results.append({
+                    "destination": kind_name, "direction": direction, "max_ctas": max_ctas,
+                    "prefix_bytes": one_way, "passes": passes, "gemm_iters": iters,
+                    "once_ms": once * 1e3, "link_gbs_alone": passes * one_way / t_xfer / 1e9,
+                    "link_gbs_with_gemm": passes * one_way / t_x_in_both / 1e9,
+                    "t_xfer_s": t_xfer, "t_gemm_s": t_gemm, "t_both_s": t_both,
+                    "gemm_slowdown": t_gemm_in_both / t_gemm,
+                    "gemm_tflops_alone": 2 * N ** 3 * iters / t_gemm / 1e12,
+                    "overlap_efficiency": eff})
+            kvc.kvc_staging_ring_destroy(ring)
+            kvc.kvc_layout_destroy(lay)
+    return {"gemm": "bf16 %dx%dx%d torch.matmul loop" % (N, N, N), "ms_per_gemm": per_iter,
+            "ring_slots": int(w.extra["ring_slots"]), "slot_bytes": cb, "runs": results}
+
+
+def run_suite(args):
+    import torch
+    from paper_2609_11744_b200 import cuda_rt, kvc
+    torch.cuda.set_device(0)
+    dev = "cuda:0"
+    parts = args.suite.split(",")
+    out = {"suite": True, "peak_hbm_gbs": measured_peak()[0], "data": "synthetic"}
+    for name, fn in (("chunk_sweep", lambda: suite_chunk_sweep(torch, kvc, dev, args.steps)),
+                     ("prefix_8k", lambda: suite_8k(torch, kvc, dev, args.steps)),
+                     ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
+                     ("ring_overlap", lambda: suite_ring_overlap(torch, kvc, cuda_rt, dev,
+                                                                 args.overlap_seconds))):
+        if "all" in parts or name in parts:
+            out[name] = fn()
+            torch.cuda.synchronize()
+            torch.cuda.empty_cache()
+    print(json.dumps(out), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -457,6 +701,10 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--suite", default="",
+                    help="run the other configs instead of the bench step: all, or a comma list of "
+                         "chunk_sweep,prefix_8k,batch_70b,ring_overlap (1 GPU; prints one JSON line)")
+    ap.add_argument("--overlap-seconds", type=float, default=2.0)
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per launch from an ncu capture, copied into the roofline object")
     args = ap.parse_args()
@@ -466,6 +714,9 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.suite:
+        run_suite(args)
         return
     run_ours(args, rank, world, local_rank)
 

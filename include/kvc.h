@@ -118,6 +118,9 @@ typedef struct {
     uint32_t ctas_per_sm; /* BULK: resident thread blocks per SM, 1..4 (0 = default) */
     uint32_t l2_hint;    /* BULK: 0 = default, 1 = no L2 priority hint, 2 = evict-first on loads and stores */
     uint32_t lag;        /* BULK: loads issued ahead of the store they feed, 1..stages-2 (0 = default) */
+    uint32_t pdl;        /* 0 = default (= 2), 1 = plain launches, 2 = programmatic dependent launch:
+                            a kernel's blocks may be scheduled while the previous kernel of the
+                            stream drains; they wait for its completion before reading memory */
 } kvc_tuning;
 /* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */
 kvc_status kvc_layout_set_tuning(kvc_layout *layout, const kvc_tuning *tuning);

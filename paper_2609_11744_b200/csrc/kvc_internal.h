@@ -58,6 +58,7 @@ struct KvcLaunch {
     uint32_t stages;          // bulk kernels
     uint32_t lag;             // bulk kernels: loads issued ahead of the store they feed
     uint32_t l2_evict_first;  // bulk kernels: attach an evict-first L2 policy to the copies
+    uint32_t pdl;             // launch with programmatic stream serialisation
     int32_t ids[KVC_PARAM_IDS];
 };
 

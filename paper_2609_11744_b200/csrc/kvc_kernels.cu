@@ -17,6 +17,8 @@
 //          hand them to the issuing lane by shuffle.  Almost no registers or
 //          issue slots are used, which leaves the SM's math pipes to other work.
 // No cluster, no multicast: every byte is read exactly once by exactly one SM.
+#include <string.h>
+
 #include "kvc_internal.h"
 
 namespace {
@@ -81,6 +83,17 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
     return it;
 }
 
+// Programmatic dependent launch: when the launch carries the stream-serialisation attribute, the
+// grid may be scheduled while the previous kernel of the stream is still draining.  Nothing in
+// global memory may be read before grid_dependency_wait() returns (it waits for the previous
+// grid to complete and its writes to be visible); after it, the next kernel is let in early.
+// Without the attribute both instructions do nothing.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // ------------------------------------------------------------------------------------ VEC
 
 // A VB-byte vector held in registers.  VB = 32 uses the 256-bit global accesses of sm_100,
@@ -135,6 +148,7 @@ kvc_vec_kernel(const __grid_constant__ KvcLaunch a)
     const uint32_t tid = threadIdx.x;
     const uint32_t n_items = (uint32_t)a.n_items;
     uint32_t w = blockIdx.x;
+    grid_dependency_wait();
     if (w >= n_items)
         return;
     Item cur = decode<TABLE>(a, w, tid == 0);
@@ -283,8 +297,10 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
     const uint32_t lane = threadIdx.x;
     const uint32_t stages = a.stages, lag = a.lag, tile = a.g.tile_bytes;
     const uint32_t n_items = (uint32_t)a.n_items;
-    if (blockIdx.x >= n_items)
+    if (blockIdx.x >= n_items) {
+        grid_dependency_wait();
         return;
+    }
     const uint32_t K = (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x;  // my items
 
     if (lane == 0) {
@@ -293,6 +309,7 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    grid_dependency_wait();
     __syncwarp();
 
     const bool hint = a.l2_evict_first != 0;
@@ -369,6 +386,23 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
     }
 }
 
+template <typename K>
+cudaError_t launch_cfg(K kernel, const KvcLaunch &a, uint32_t grid, uint32_t block, uint32_t smem,
+                       cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = a.pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, a);
+}
+
 template <int DIR, bool TABLE>
 cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t smem,
                        cudaStream_t stream)
@@ -383,13 +417,11 @@ cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t 
                 return e;
             configured_smem[DIR][TABLE] = (int)smem;
         }
-        kvc_bulk_kernel<DIR, TABLE><<<grid, KVC_BULK_THREADS, smem, stream>>>(a);
-    } else if (variant == KVC_VARIANT_VEC32) {
-        kvc_vec_kernel<DIR, TABLE, 32><<<grid, KVC_VEC_THREADS, 0, stream>>>(a);
-    } else {
-        kvc_vec_kernel<DIR, TABLE, 16><<<grid, KVC_VEC_THREADS, 0, stream>>>(a);
+        return launch_cfg(kvc_bulk_kernel<DIR, TABLE>, a, grid, KVC_BULK_THREADS, smem, stream);
     }
-    return cudaGetLastError();
+    if (variant == KVC_VARIANT_VEC32)
+        return launch_cfg(kvc_vec_kernel<DIR, TABLE, 32>, a, grid, KVC_VEC_THREADS, 0, stream);
+    return launch_cfg(kvc_vec_kernel<DIR, TABLE, 16>, a, grid, KVC_VEC_THREADS, 0, stream);
 }
 
 }  // namespace

@@ -124,6 +124,7 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     a->stages = stages;
     a->lag = lag;
     a->l2_evict_first = t.l2_hint == 2;
+    a->pdl = t.pdl != 1;  // on unless switched off
     a->status = lay->d_status;
     uint64_t grid = variant == KVC_VARIANT_BULK
                         ? (uint64_t)lay->sm_count * (t.ctas_per_sm ? t.ctas_per_sm : 1u)
@@ -495,7 +496,7 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
         return KVC_ERR_INVALID_ARG;
     if (t->stages == 1 || t->stages > KVC_BULK_MAX_STAGES)
         return KVC_ERR_INVALID_ARG;
-    if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES)
+    if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2)
         return KVC_ERR_INVALID_ARG;
     lay->tuning = *t;
     return KVC_OK;

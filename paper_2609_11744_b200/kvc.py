@@ -51,7 +51,8 @@ class kvc_tuning(ctypes.Structure):
     _fields_ = [("variant", ctypes.c_uint32), ("order", ctypes.c_uint32),
                 ("max_ctas", ctypes.c_uint32), ("tile_bytes", ctypes.c_uint32),
                 ("stages", ctypes.c_uint32), ("ctas_per_sm", ctypes.c_uint32),
-                ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32)]
+                ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32),
+                ("pdl", ctypes.c_uint32)]
 
 
 class kvc_chunk_desc(ctypes.Structure):
@@ -268,8 +269,8 @@ def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
 
 
 def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
-                          ctas_per_sm=0, l2_hint=0, lag=0) -> None:
-    t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag)
+                          ctas_per_sm=0, l2_hint=0, lag=0, pdl=0) -> None:
+    t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag, pdl)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
 
 

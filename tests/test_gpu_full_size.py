@@ -1,0 +1,93 @@
+"""Full-size GPU checks in the launch configuration the benchmark times (one batched pack and
+one batched unpack of the whole prefix).  The pools are tens of GiB and live only on the device,
+so the oracle is applied to sampled outputs, one element at a time: for every sample the oracle's
+index formulas give the staging position and the pool positions, and the device values there must
+agree.  Properties that hold at any size are checked on everything: the staged bytes equal the
+gathered pool slabs, and pool blocks that were not named keep their contents."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import oracle as orc
+from paper_2609_11744_b200 import kvc
+import workloads as wl
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+N_SAMPLES = 300_000
+
+
+def _sampled_positions(g, src, dst, bpc, seed):
+    """Oracle positions (element indices) of N random chunk elements: in the staging area (chunks
+    back to back), in the pool at the source block and in the pool at the destination block."""
+    n = len(src)
+    rng = np.random.default_rng(seed)
+    blk = rng.integers(0, n, N_SAMPLES)
+    c = blk // bpc
+    j = blk - c * bpc
+    nb_c = np.minimum(bpc, n - c * bpc)
+    l, p = rng.integers(0, g.L, N_SAMPLES), rng.integers(0, g.P, N_SAMPLES)
+    t, h, d = (rng.integers(0, k, N_SAMPLES) for k in (g.B, g.H, g.D))
+    full_chunk_elems = orc.chunk_bytes(g, bpc) // g.e
+    stage = c.astype(np.int64) * full_chunk_elems + orc.chunk_elem(g, nb_c, l, p, j, t, h, d)
+    src_pos = orc.pool_elem(g, l, p, src[blk].astype(np.int64), t, h, d)
+    dst_pos = orc.pool_elem(g, l, p, dst[blk].astype(np.int64), t, h, d)
+    return blk, stage, src_pos, dst_pos
+
+
+def _full_size_case(w, chunk_tokens, n_free_check=64):
+    s = w.shape
+    NB, n = w.pool_blocks, w.request_blocks
+    free, _ = torch.cuda.mem_get_info()
+    need = NB * s.bytes_per_block + 3 * n * s.bytes_per_block + (2 << 30)
+    if free < need:
+        pytest.skip("needs %.1f GiB of free device memory" % (need / 2**30))
+    g = orc.Dims(s.L, s.P, NB, s.B, s.H, s.D, s.e)
+    bpc = chunk_tokens // s.B
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, DEV)
+    src = wl.block_ids(w.seed, NB, n)
+    dst = wl.block_ids(w.dst_seed, NB, n)
+    one_way = n * s.bytes_per_block
+    staging = torch.full((one_way + 4096,), 0x77, dtype=torch.uint8, device=DEV)
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, chunk_tokens)
+    assert kvc.kvc_layout_num_chunks(lay, n) == len(orc.chunk_ranges(n, bpc))
+    pool16, stage16 = pool.view(torch.int16), staging[:one_way].view(torch.int16)
+    blk, stage_pos, src_pos, dst_pos = _sampled_positions(g, src, dst, bpc, w.seed)
+    dev_idx = lambda a: torch.from_numpy(a).to(DEV)
+
+    # ---- pack: one launch
+    ops, keep, nbytes, on_dev = kvc.request_chunk_ops(lay, src, staging)
+    assert nbytes == one_way
+    kvc.kvc_pack_batch(lay, ops, on_dev)
+    torch.cuda.synchronize()
+    assert torch.equal(stage16[dev_idx(stage_pos)], pool16[dev_idx(src_pos)]), "pack: sampled elements"
+    assert bool((staging[one_way:] == 0x77).all()), "pack wrote past the last chunk"
+    # property at full size: every chunk equals the pool slabs gathered along the block axis
+    pool4 = pool.view(s.L * s.P, NB, s.slab_bytes)
+    off = 0
+    for first, nb in orc.chunk_ranges(n, bpc)[:: max(1, len(orc.chunk_ranges(n, bpc)) // 24)]:
+        off = first * s.bytes_per_block
+        ids_t = dev_idx(src[first:first + nb].astype(np.int64))
+        want = pool4[:, ids_t].reshape(-1)
+        assert torch.equal(staging[off:off + want.numel()], want), "pack: chunk at entry %d" % first
+
+    # ---- unpack: one launch into the second table
+    untouched = np.setdiff1d(np.arange(NB), dst)[:n_free_check]
+    before = pool4[:, dev_idx(untouched.astype(np.int64))].clone()
+    ops2, keep2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+    kvc.kvc_unpack_batch(lay, ops2, on_dev)
+    torch.cuda.synchronize()
+    assert torch.equal(pool16[dev_idx(dst_pos)], stage16[dev_idx(stage_pos)]), "unpack: sampled elements"
+    assert torch.equal(pool4[:, dev_idx(untouched.astype(np.int64))], before), "unpack touched other blocks"
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+    assert kvc.kvc_layout_launch_count(lay) == 2
+
+
+def test_config2_8b_8k_prefix():
+    _full_size_case(wl.WORKLOADS["8b_8k"], 256)
+
+
+@pytest.mark.parametrize("chunk_tokens", [256, 16, 2048])
+def test_config3_8b_80k_prefix(chunk_tokens):
+    _full_size_case(wl.WORKLOADS["8b_80k"], chunk_tokens)
