@@ -201,6 +201,22 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+# ------------------------------------------------------------------ multi-GPU bookkeeping
+def max_over_ranks(value: float, dist, world: int, device) -> float:
+    """The slowest rank's time (ranks are independent replicas; there is no data-path exchange)."""
+    if world <= 1:
+        return float(value)
+    import torch
+    t = torch.tensor([value], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_rank_per_step: int, steps: int, world: int, slowest_ms: float) -> float:
+    """Aggregate throughput of all replicas: bytes moved by every rank over the slowest rank's time."""
+    return world * bytes_per_rank_per_step * steps / (slowest_ms * 1e-3) / 1e9
+
+
 # ------------------------------------------------------------------ GPU arm
 def run_ours(args, rank, world, local_rank):
     import torch
@@ -269,12 +285,9 @@ def run_ours(args, rank, world, local_rank):
     skipped, expired = kvc.kvc_poll_device_status(lay)
     assert (skipped, expired) == (0, 0), "device status flags set: %r" % ((skipped, expired),)
 
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, dist, world, dev)
     bytes_step = 4 * one_way  # pack: read+write; unpack: read+write
-    value = world * bytes_step * args.steps / (total_ms * 1e-3) / 1e9
+    value = whole_job_gbs(bytes_step, args.steps, world, total_ms)
 
     e2e = None
     if not args.no_e2e:
@@ -380,10 +393,7 @@ def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, di
         t_off.append(t1 - t0)
         t_load.append(t2 - t1)
     step_s = statistics.mean(t_off) + statistics.mean(t_load)
-    if world > 1:
-        t = torch.tensor([step_s], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        step_s = float(t.item())
+    step_s = max_over_ranks(step_s, dist, world, dev)
     _, acquires, stalls = kvc.kvc_staging_ring_stats(ring)
     kvc.kvc_staging_ring_destroy(ring)
     return {
