@@ -150,6 +150,14 @@ class OracleSample:
                 f.result()
         return t1 - t0, time.perf_counter() - t1
 
+    def single_core(self):
+        """One chunk packed and unpacked by one thread: GB/s of bytes read + written."""
+        orc, g, bpc = self.orc, self.g, self.bpc
+        t0 = time.perf_counter()
+        orc.pack_chunk_into(g, self.pool, self.src[:bpc], self.bufs[0])
+        orc.unpack_chunk(g, self.pool, self.bufs[0], self.dst[:bpc])
+        return 4 * self.cb / (time.perf_counter() - t0) / 1e9
+
     def run(self, target_seconds: float):
         p1, u1 = self._pass(1)
         want = max(1, round(target_seconds / max(p1 + u1, 1e-6)))
@@ -293,11 +301,18 @@ def run_ours(args, rank, world, local_rank):
     if not args.no_e2e:
         e2e = run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, dist)
     peak, peak_kind = measured_peak()
+    traffic = args.traffic_bytes
+    if traffic is None and (args.workload, NB, n, args.chunk_tokens, args.variant) == \
+            ("8b_80k", 20000, 5000, 256, 0):
+        # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this exact workload, from a
+        # one-pass ncu capture (profiles/kvc_bulk_kernel_8b_80k_dram_traffic.md): mean of the
+        # pack launch (20,936,505,000) and the unpack launch (20,933,015,000)
+        traffic = 20_934_760_000.0
     launch_ms = statistics.mean(pack_ms + unpack_ms)
     achieved = 2 * one_way / (launch_ms * 1e-3) / 1e9
     roof = {
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "traffic": args.traffic_bytes, "peak_kind": peak_kind,
+        "traffic": traffic, "peak_kind": peak_kind,
         "kernel": "kvc_bulk_kernel (pack and unpack instantiations)" if args.variant != 1
                   else "kvc_vec_kernel (pack and unpack instantiations)",
         "algorithmic_bytes_per_launch": 2 * one_way,
@@ -316,7 +331,9 @@ def run_ours(args, rank, world, local_rank):
         return
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        cpu = OracleSample(s, args.chunk_tokens, w.seed + 50).run(12.0)
+        sample = OracleSample(s, args.chunk_tokens, w.seed + 50)
+        cpu = sample.run(15.0)
+        cpu["single_core_gbs"] = sample.single_core()
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
@@ -528,6 +545,53 @@ def suite_batch(torch, kvc, dev, reps):
             "pack_ms_min": pm, "pack_ms_median": pd, "pack_gbs": 2 * total / pd / 1e6}
 
 
+def _overlap_case(torch, fn, gemm_loop, s_gemm, s_k, s_c, iters, seconds, one_way, N, name,
+                  direction, max_ctas):
+    """Transfer alone, GEMM loop alone, both at once; see suite_ring_overlap."""
+    fn()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    fn()
+    torch.cuda.synchronize()
+    once = time.perf_counter() - t0
+    passes = max(1, int(seconds / once))
+    t0 = time.perf_counter()
+    for _ in range(passes):
+        fn()
+    torch.cuda.synchronize()
+    t_xfer = time.perf_counter() - t0
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    g0.record(s_gemm)
+    gemm_loop(iters)
+    g1.record(s_gemm)
+    torch.cuda.synchronize()
+    t_gemm = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    g0.record(s_gemm)
+    gemm_loop(iters)
+    g1.record(s_gemm)
+    for _ in range(passes):
+        fn()
+    s_c.synchronize()
+    s_k.synchronize()
+    t_x_in_both = time.perf_counter() - t0
+    torch.cuda.synchronize()
+    t_both = time.perf_counter() - t0
+    t_gemm_in_both = g0.elapsed_time(g1) * 1e-3
+    eff = 1 - (t_both - max(t_gemm, t_xfer)) / min(t_gemm, t_xfer)
+    return {"destination": name, "direction": direction, "max_ctas": max_ctas,
+            "prefix_bytes": one_way, "passes": passes, "gemm_iters": iters,
+            "once_ms": once * 1e3, "link_gbs_alone": passes * one_way / t_xfer / 1e9,
+            "link_gbs_with_gemm": passes * one_way / t_x_in_both / 1e9,
+            "t_xfer_s": t_xfer, "t_gemm_s": t_gemm, "t_both_s": t_both,
+            "gemm_slowdown": t_gemm_in_both / t_gemm,
+            "gemm_tflops_alone": 2 * N ** 3 * iters / t_gemm / 1e12,
+            "overlap_efficiency": eff}
+
+
 def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
     """Config 5: a 32k-token prefix (8B shape, 4 GiB) streamed through an 8-slot ring of 256-token
     slots to/from pinned host memory while a bf16 GEMM loop runs on another stream.  Destinations:
@@ -617,57 +681,95 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
                     off += nbytes
 
             for direction, fn in (("offload", offload), ("load", load)):
-                fn()
-                torch.cuda.synchronize()
-                t0 = time.perf_counter()
-                fn()
-                torch.cuda.synchronize()
-                once = time.perf_counter() - t0
-                passes = max(1, int(seconds / once))
-                t0 = time.perf_counter()
-                for _ in range(passes):
-                    fn()
-                torch.cuda.synchronize()
-                t_xfer = time.perf_counter() - t0
-                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                t0 = time.perf_counter()
-                g0.record(s_gemm)
-                gemm_loop(iters)
-                g1.record(s_gemm)
-                torch.cuda.synchronize()
-                t_gemm = time.perf_counter() - t0
-                # both at once
-                x0, x1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                torch.cuda.synchronize()
-                t0 = time.perf_counter()
-                g0.record(s_gemm)
-                gemm_loop(iters)
-                g1.record(s_gemm)
-                x0.record(s_k)
-                for _ in range(passes):
-                    fn()
-                x1.record(s_k)
-                s_c.synchronize()
-                s_k.synchronize()
-                t_x_in_both = time.perf_counter() - t0
-                torch.cuda.synchronize()
-                t_both = time.perf_counter() - t0
-                t_gemm_in_both = g0.elapsed_time(g1) * 1e-3
-                eff = 1 - (t_both - max(t_gemm, t_xfer)) / min(t_gemm, t_xfer)
-                results.append({
-                    "destination": kind_name, "direction": direction, "max_ctas": max_ctas,
-                    "prefix_bytes": one_way, "passes": passes, "gemm_iters": iters,
-                    "once_ms": once * 1e3, "link_gbs_alone": passes * one_way / t_xfer / 1e9,
-                    "link_gbs_with_gemm": passes * one_way / t_x_in_both / 1e9,
-                    "t_xfer_s": t_xfer, "t_gemm_s": t_gemm, "t_both_s": t_both,
-                    "gemm_slowdown": t_gemm_in_both / t_gemm,
-                    "gemm_tflops_alone": 2 * N ** 3 * iters / t_gemm / 1e12,
-                    "overlap_efficiency": eff})
+                results.append(_overlap_case(torch, fn, gemm_loop, s_gemm, s_k, s_c, iters, seconds,
+                                             one_way, N, kind_name, direction, max_ctas))
             kvc.kvc_staging_ring_destroy(ring)
             kvc.kvc_layout_destroy(lay)
+    # several ring slots per launch: one batched pack/unpack serves GROUP slots, so the compute
+    # stream is interrupted GROUP times less often
+    GROUP = 4
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    descs = kvc.kvc_map_request(lay, n)
+    cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+    ring = kvc.kvc_staging_ring_create(cb, int(w.extra["ring_slots"]), kvc.KVC_RING_DEVICE)
+
+    def grouped(direction):
+        off = 0
+        for g0 in range(0, len(descs), GROUP):
+            grp = descs[g0:g0 + GROUP]
+            slots = [kvc.kvc_staging_ring_acquire(ring, TO) for _ in grp]
+            ops = kvc.make_chunk_ops([sl[1] for sl in slots],
+                                     [(src if direction == 0 else dst).ctypes.data + 4 * d[2] for d in grp],
+                                     [d[3] for d in grp])
+            if direction == 0:
+                kvc.kvc_pack_batch(lay, ops, 0, stream=s_k)
+                for (slot, dptr, _), d in zip(slots, grp):
+                    kvc.kvc_staging_ring_commit(ring, slot, s_k)
+                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
+                    cuda_rt.memcpy_async(hptr + off, dptr, d[4], cuda_rt.D2H, s_c)
+                    kvc.kvc_staging_ring_release(ring, slot, s_c)
+                    off += d[4]
+            else:
+                for (slot, dptr, _), d in zip(slots, grp):
+                    cuda_rt.memcpy_async(dptr, hptr + off, d[4], cuda_rt.H2D, s_c)
+                    kvc.kvc_staging_ring_commit(ring, slot, s_c)
+                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_k)
+                    off += d[4]
+                kvc.kvc_unpack_batch(lay, ops, 0, stream=s_k)
+                for (slot, dptr, _) in slots:
+                    kvc.kvc_staging_ring_release(ring, slot, s_k)
+
+    for direction, name in ((0, "offload"), (1, "load")):
+        results.append(_overlap_case(torch, lambda: grouped(direction), gemm_loop, s_gemm, s_k, s_c,
+                                     iters, seconds, one_way, N,
+                                     "device slots + cudaMemcpyAsync, %d slots per launch" % GROUP,
+                                     name, 0))
+    kvc.kvc_staging_ring_destroy(ring)
+    kvc.kvc_layout_destroy(lay)
+    # the paper's mechanism for comparison: strided DMA copies straight between the pool and
+    # pinned host memory, no kernel, no staging slot
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    descs = kvc.kvc_map_request(lay, n)
+
+    def dma_offload():
+        off = 0
+        for (_, c, first, nb, nbytes) in descs:
+            kvc.kvc_pack_copy_engine(lay, src[first:first + nb], hptr + off, nbytes, stream=s_c)
+            off += nbytes
+
+    def dma_load():
+        off = 0
+        for (_, c, first, nb, nbytes) in descs:
+            kvc.kvc_unpack_copy_engine(lay, hptr + off, dst[first:first + nb], nbytes, stream=s_c)
+            off += nbytes
+
+    for direction, fn in (("offload", dma_offload), ("load", dma_load)):
+        results.append(_overlap_case(torch, fn, gemm_loop, s_gemm, s_c, s_c, iters, seconds, one_way, N,
+                                     "copy engines, pool <-> pinned host directly", direction, 0))
+    kvc.kvc_layout_destroy(lay)
     return {"gemm": "bf16 %dx%dx%d torch.matmul loop" % (N, N, N), "ms_per_gemm": per_iter,
             "ring_slots": int(w.extra["ring_slots"]), "slot_bytes": cb, "runs": results}
+
+
+def suite_host_link(torch, cuda_rt, dev):
+    """Host-link ceiling of this machine: cudaMemcpyAsync of 1 GiB of pinned memory, each direction,
+    best of 10."""
+    nbytes = 1 << 30
+    host = torch.empty(nbytes, dtype=torch.uint8, pin_memory=True)
+    devb = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+    st = torch.cuda.current_stream()
+    out = {}
+    for name, dst, src, kind in (("d2h_gbs", host, devb, cuda_rt.D2H), ("h2d_gbs", devb, host, cuda_rt.H2D)):
+        best = 1e9
+        for _ in range(10):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
+            cuda_rt.memcpy_async(dst.data_ptr(), src.data_ptr(), nbytes, kind, st)
+            b.record(st)
+            b.synchronize()
+            best = min(best, a.elapsed_time(b))
+        out[name] = nbytes / best / 1e6
+    return out
 
 
 def run_suite(args):
@@ -677,7 +779,8 @@ def run_suite(args):
     dev = "cuda:0"
     parts = args.suite.split(",")
     out = {"suite": True, "peak_hbm_gbs": measured_peak()[0], "data": "synthetic"}
-    for name, fn in (("chunk_sweep", lambda: suite_chunk_sweep(torch, kvc, dev, args.steps)),
+    for name, fn in (("host_link", lambda: suite_host_link(torch, cuda_rt, dev)),
+                     ("chunk_sweep", lambda: suite_chunk_sweep(torch, kvc, dev, args.steps)),
                      ("prefix_8k", lambda: suite_8k(torch, kvc, dev, args.steps)),
                      ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
                      ("ring_overlap", lambda: suite_ring_overlap(torch, kvc, cuda_rt, dev,
@@ -713,10 +816,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
-                         "chunk_sweep,prefix_8k,batch_70b,ring_overlap (1 GPU; prints one JSON line)")
+                         "host_link,chunk_sweep,prefix_8k,batch_70b,ring_overlap (1 GPU; prints one JSON line)")
     ap.add_argument("--overlap-seconds", type=float, default=2.0)
     ap.add_argument("--traffic-bytes", type=float, default=None,
-                    help="DRAM bytes per launch from an ncu capture, copied into the roofline object")
+                    help="DRAM bytes per launch from an ncu capture, copied into the roofline object "
+                         "(default: the committed capture of the default workload, else null)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
     rank = int(os.environ.get("RANK", "0"))

@@ -61,6 +61,12 @@ const char *kvc_status_str(kvc_status s);
 
 typedef struct kvc_layout kvc_layout;
 
+/* Byte order inside a chunk of n blocks.  The paper fixes only the file naming (Sec. 6.3), not
+ * the order inside a storage block.  LAYER_MAJOR [layer][K|V][n][token][head][dim] is the paged
+ * layout with the block axis gathered.  BLOCK_MAJOR [n][layer][K|V][token][head][dim] keeps all
+ * layers of one block together, so a shorter chunk is a prefix of a longer one. */
+typedef enum { KVC_CHUNK_LAYER_MAJOR = 0, KVC_CHUNK_BLOCK_MAJOR = 1 } kvc_chunk_order;
+
 typedef struct {
     uint32_t num_layers;
     uint32_t kv_planes;    /* planes per layer: 2 (K and V), or 1 for a fused cache */
@@ -72,12 +78,17 @@ typedef struct {
     uint32_t chunk_tokens; /* tokens per chunk; a positive multiple of block_size */
     /* Either plane_ptrs != NULL: HOST array of num_layers*kv_planes DEVICE pointers,
      * entry l*kv_planes+p is the base of plane (l,p) (the array is copied);
-     * or plane_ptrs == NULL: plane (l,p) starts at base + l*layer_stride + p*plane_stride. */
+     * or plane_ptrs == NULL: plane (l,p) starts at base + l*layer_stride + p*plane_stride.
+     * Planes must not overlap: either plane_stride >= the span of one plane (pool order
+     * [layer][K|V][block]..), or block_stride >= kv_planes*plane_stride >= kv_planes*slab_bytes
+     * (pool order [layer][block][K|V].., K and V of a block adjacent). */
     const void *const *plane_ptrs;
     const void *base;      /* device pointer */
     uint64_t layer_stride; /* bytes */
     uint64_t plane_stride; /* bytes */
     uint64_t block_stride; /* bytes between consecutive blocks of a plane; 0 means slab_bytes */
+    uint32_t chunk_order;  /* kvc_chunk_order: byte order inside a chunk */
+    uint32_t reserved;     /* must be 0 */
 } kvc_layout_desc;
 
 /* Validates and copies the descriptor.  Makes no CUDA call: the small device-side
@@ -215,6 +226,20 @@ kvc_status kvc_poll_device_status(kvc_layout *layout, void *stream, uint32_t *n_
 #define KVC_STATIC_MAX_PLANES 1024u
 kvc_status kvc_pack_batch_static(kvc_layout *layout, const kvc_chunk_op *ops, uint32_t n_ops,
                                  void *stream);
+
+/* Copy-engine variants (the paper's own mechanism, Sec. 6.2 / 6.4: a DMA-based batched block
+ * copy between the KV tensors and pinned staging slots; Sec. 5.1 contrasts it with kernel copies).
+ * Same result as kvc_pack / kvc_unpack for one chunk, but issued as strided asynchronous memory
+ * copies on `stream` -- one per block where the planes are equally spaced, else one per layer or
+ * per plane -- so no kernel runs and no SM is used.  `dst` / `src` may be DEVICE memory or PINNED
+ * HOST memory; with host memory the chunk crosses the host link directly and no staging slot is
+ * needed.  ids are HOST memory and are validated first (unpack rejects repeated ids).
+ * They allocate nothing and do not count as kernel launches.
+ * Errors: INVALID_ARG, ALIGNMENT, OUT_OF_RANGE, CONFLICT, CUDA. */
+kvc_status kvc_pack_copy_engine(kvc_layout *layout, const int32_t *ids, uint32_t n_blocks, void *dst,
+                                uint64_t dst_bytes, void *stream);
+kvc_status kvc_unpack_copy_engine(kvc_layout *layout, const void *src, uint64_t src_bytes,
+                                  const int32_t *ids, uint32_t n_blocks, void *stream);
 
 /* Number of kernel launches issued through this handle so far. */
 uint64_t kvc_layout_launch_count(const kvc_layout *layout);

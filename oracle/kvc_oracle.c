@@ -63,6 +63,17 @@ uint64_t kvc_oracle_chunk_elem(const kvc_oracle_dims *g, uint64_t nb_c, uint64_t
     return ((((l * g->P + p) * nb_c + j) * g->B + t) * g->H + h) * g->D + d;
 }
 
+/* Element index in a block-major chunk of nb_c blocks, [nb_c][L][P][B][H][D]: every block's
+ * data for all layers is one contiguous run (an alternative file layout; the paper does not fix
+ * the byte order inside a storage block). */
+uint64_t kvc_oracle_chunk_elem_block_major(const kvc_oracle_dims *g, uint64_t nb_c, uint64_t l,
+                                           uint64_t p, uint64_t j, uint64_t t, uint64_t h,
+                                           uint64_t d)
+{
+    (void)nb_c;
+    return ((((j * g->L + l) * g->P + p) * g->B + t) * g->H + h) * g->D + d;
+}
+
 static int ids_in_range(const kvc_oracle_dims *g, const int32_t *ids, uint32_t nb_c)
 {
     for (uint32_t j = 0; j < nb_c; ++j)
@@ -161,5 +172,50 @@ int kvc_oracle_unpack_chunk_planes(const kvc_oracle_dims *g, uint8_t *const *pla
                             plane[dst * g->e + k] = chunk[src * g->e + k];
                     }
     }
+    return 0;
+}
+
+/* pack / unpack with the block-major chunk order, separately allocated (or strided) planes. */
+int kvc_oracle_pack_chunk_planes_block_major(const kvc_oracle_dims *g, const uint8_t *const *planes,
+                                             uint64_t block_stride_elems, const int32_t *ids,
+                                             uint32_t nb_c, uint8_t *chunk)
+{
+    if (!ids_in_range(g, ids, nb_c))
+        return -1;
+    for (uint32_t j = 0; j < nb_c; ++j)
+        for (uint32_t l = 0; l < g->L; ++l)
+            for (uint32_t p = 0; p < g->P; ++p) {
+                const uint8_t *plane = planes[l * g->P + p];
+                for (uint32_t t = 0; t < g->B; ++t)
+                    for (uint32_t h = 0; h < g->H; ++h)
+                        for (uint32_t d = 0; d < g->D; ++d) {
+                            uint64_t src = plane_elem(g, block_stride_elems, (uint64_t)ids[j], t, h, d);
+                            uint64_t dst = kvc_oracle_chunk_elem_block_major(g, nb_c, l, p, j, t, h, d);
+                            for (uint32_t k = 0; k < g->e; ++k)
+                                chunk[dst * g->e + k] = plane[src * g->e + k];
+                        }
+            }
+    return 0;
+}
+
+int kvc_oracle_unpack_chunk_planes_block_major(const kvc_oracle_dims *g, uint8_t *const *planes,
+                                               uint64_t block_stride_elems, const int32_t *ids,
+                                               uint32_t nb_c, const uint8_t *chunk)
+{
+    if (!ids_in_range(g, ids, nb_c))
+        return -1;
+    for (uint32_t j = 0; j < nb_c; ++j)
+        for (uint32_t l = 0; l < g->L; ++l)
+            for (uint32_t p = 0; p < g->P; ++p) {
+                uint8_t *plane = planes[l * g->P + p];
+                for (uint32_t t = 0; t < g->B; ++t)
+                    for (uint32_t h = 0; h < g->H; ++h)
+                        for (uint32_t d = 0; d < g->D; ++d) {
+                            uint64_t dst = plane_elem(g, block_stride_elems, (uint64_t)ids[j], t, h, d);
+                            uint64_t src = kvc_oracle_chunk_elem_block_major(g, nb_c, l, p, j, t, h, d);
+                            for (uint32_t k = 0; k < g->e; ++k)
+                                plane[dst * g->e + k] = chunk[src * g->e + k];
+                        }
+            }
     return 0;
 }

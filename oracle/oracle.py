@@ -76,6 +76,11 @@ def chunk_elem(g: Dims, nb_c: int, l: int, p: int, j: int, t: int, h: int, d: in
     return ((((l * g.P + p) * nb_c + j) * g.B + t) * g.H + h) * g.D + d
 
 
+def chunk_elem_block_major(g: Dims, nb_c: int, l: int, p: int, j: int, t: int, h: int, d: int) -> int:
+    """Element index in a block-major chunk, [nb_c][L][P][B][H][D] (nb_c does not enter)."""
+    return ((((j * g.L + l) * g.P + p) * g.B + t) * g.H + h) * g.D + d
+
+
 def chunk_bytes(g: Dims, nb_c: int) -> int:
     """Exact size of a chunk of nb_c blocks: every byte is useful KV data."""
     return g.L * g.P * nb_c * g.slab_bytes
@@ -156,6 +161,13 @@ def _clib():
             f = getattr(lib, name)
             f.restype = ctypes.c_int
             f.argtypes = [dp, ctypes.c_void_p, u64, i32p, u32, u8p, u32, u32]
+        for name in ("kvc_oracle_pack_chunk_planes_block_major",
+                     "kvc_oracle_unpack_chunk_planes_block_major"):
+            f = getattr(lib, name)
+            f.restype = ctypes.c_int
+            f.argtypes = [dp, ctypes.c_void_p, u64, i32p, u32, u8p]
+        lib.kvc_oracle_chunk_elem_block_major.restype = u64
+        lib.kvc_oracle_chunk_elem_block_major.argtypes = [dp] + [u64] * 7
         _lib = lib
     return _lib
 
@@ -248,6 +260,40 @@ def unpack_chunk_planes(g: Dims, planes: Sequence[np.ndarray], chunk: np.ndarray
                                                 0, g.L * g.P)
     if rc:
         raise IndexError("block id out of range")
+
+
+def pack_chunk_planes_block_major(g: Dims, planes: Sequence[np.ndarray], ids,
+                                  block_stride_bytes: int | None = None) -> np.ndarray:
+    """Pack one chunk in block-major order [nb_c][L][P][B][H][D]."""
+    bs = block_stride_bytes or g.slab_bytes
+    arr = _plane_ptrs(g, planes, bs)
+    ids = _ids32(ids)
+    out = np.zeros(chunk_bytes(g, len(ids)), dtype=np.uint8)
+    rc = _clib().kvc_oracle_pack_chunk_planes_block_major(ctypes.byref(_cd(g)), arr, bs // g.e,
+                                                          ids.ctypes.data, len(ids), out.ctypes.data)
+    if rc:
+        raise IndexError("block id out of range")
+    return out
+
+
+def unpack_chunk_planes_block_major(g: Dims, planes: Sequence[np.ndarray], chunk: np.ndarray, ids,
+                                    block_stride_bytes: int | None = None) -> None:
+    bs = block_stride_bytes or g.slab_bytes
+    arr = _plane_ptrs(g, planes, bs)
+    chunk, ids = _bytes_view(chunk), _ids32(ids)
+    assert chunk.size == chunk_bytes(g, len(ids))
+    rc = _clib().kvc_oracle_unpack_chunk_planes_block_major(ctypes.byref(_cd(g)), arr, bs // g.e,
+                                                            ids.ctypes.data, len(ids),
+                                                            chunk.ctypes.data)
+    if rc:
+        raise IndexError("block id out of range")
+
+
+def dense_planes(g: Dims, pool: np.ndarray) -> List[np.ndarray]:
+    """The L*P planes of a dense pool [L][P][NB][B][H][D] as views (plane l*P+p)."""
+    pool = _bytes_view(pool)
+    pb = g.NB * g.slab_bytes
+    return [pool[i * pb:(i + 1) * pb] for i in range(g.L * g.P)]
 
 
 def pack_request(g: Dims, pool: np.ndarray, ids, chunk_tokens: int) -> List[np.ndarray]:

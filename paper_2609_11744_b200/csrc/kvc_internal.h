@@ -39,9 +39,9 @@ struct KvcGeom {
 struct KvcEnt {
     uint64_t slot_addr;   // chunk base + j*S : where block j of the chunk starts in plane 0
     uint64_t id_or_ptr;   // the pool block id, or the device address of it
-    uint32_t nb_c;        // blocks in this chunk (plane stride inside the chunk = nb_c*S)
+    uint32_t nb_c;        // blocks in this chunk
     uint32_t id_is_ptr;
-    uint64_t pad;
+    uint64_t plane_step;  // bytes between consecutive planes of this block inside the chunk
 };
 static_assert(sizeof(KvcEnt) == 32, "KvcEnt is loaded as two 16-byte vectors");
 
@@ -50,6 +50,8 @@ struct KvcLaunch {
     KvcGeom g;
     const KvcEnt *table;      // batched launch: n_ent entries in device memory; else nullptr
     uint64_t slot;            // single-chunk launch: chunk base
+    uint64_t ent_step;        // single-chunk launch: bytes between consecutive blocks of a plane
+    uint64_t plane_step;      // single-chunk launch: bytes between consecutive planes of a block
     const int32_t *dev_ids;   // single-chunk launch with device-resident ids; else nullptr
     uint32_t *status;         // [0] blocks skipped (bad device id), [1] waits that gave up
     uint64_t n_items;         // n_ent * LP * parts
@@ -104,6 +106,20 @@ struct kvc_layout {
     uint32_t seen_stamp;
 };
 
+
+// Where block j, plane lp of a chunk of nb blocks starts, relative to the chunk base:
+// j * ent_step + lp * plane_step.  Layer-major chunks [L][P][nb][..]: (S, nb*S);
+// block-major chunks [nb][L][P][..]: (L*P*S, S).
+inline void kvc_chunk_steps(const kvc_layout *lay, uint32_t nb, uint64_t *ent_step, uint64_t *plane_step)
+{
+    if (lay->d.chunk_order == KVC_CHUNK_BLOCK_MAJOR) {
+        *ent_step = (uint64_t)lay->planes_total * lay->slab_bytes;
+        *plane_step = lay->slab_bytes;
+    } else {
+        *ent_step = lay->slab_bytes;
+        *plane_step = (uint64_t)nb * lay->slab_bytes;
+    }
+}
 
 // Launch shape chosen by the host for one call.
 struct KvcPlan {

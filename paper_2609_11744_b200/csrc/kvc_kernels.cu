@@ -3,7 +3,8 @@
 // A launch moves n_ent blocks x LP planes x `parts` tiles.  Work item w names one
 // tile of one slab (the contiguous bytes of one block in one (layer, K|V) plane):
 //     pool side : plane(lp) + id*block_stride + part*tile
-//     slot side : chunk + (lp*nb_c + j)*S    + part*tile        (Sec. 6.4 chunk layout)
+//     slot side : chunk + j*ent_step + lp*plane_step + part*tile
+//                 (layer-major chunk: ent_step = S, plane_step = nb_c*S)
 // pack copies pool -> slot, unpack slot -> pool.  Nothing is a contraction: the
 // kernels are bound by HBM bandwidth, so they only keep many full-line requests
 // in flight and touch every byte once.
@@ -53,19 +54,18 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
         ent = r / g.planes_total;
         lp = r - ent * g.planes_total;
     }
-    uint64_t slot_j;
-    uint32_t nb_c;
+    uint64_t slot_j, plane_step;
     int64_t id;
     if (TABLE) {
         const uint4 *e = reinterpret_cast<const uint4 *>(a.table + ent);
         uint4 lo = __ldg(e), hi = __ldg(e + 1);
         slot_j = ((uint64_t)lo.y << 32) | lo.x;
         uint64_t idp = ((uint64_t)lo.w << 32) | lo.z;
-        nb_c = hi.x;
+        plane_step = ((uint64_t)hi.w << 32) | hi.z;
         id = hi.y ? (int64_t)__ldg(reinterpret_cast<const int32_t *>(idp)) : (int64_t)(int32_t)lo.z;
     } else {
-        slot_j = a.slot + (uint64_t)ent * g.slab_bytes;
-        nb_c = a.n_ent;
+        slot_j = a.slot + (uint64_t)ent * a.ent_step;
+        plane_step = a.plane_step;
         id = a.dev_ids ? (int64_t)__ldg(a.dev_ids + ent) : (int64_t)a.ids[ent];
     }
     Item it;
@@ -79,7 +79,7 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
         id = 0;
     }
     it.pool = plane_base(g, lp) + (uint64_t)id * g.block_stride + off;
-    it.slot = slot_j + (uint64_t)lp * nb_c * g.slab_bytes + off;
+    it.slot = slot_j + (uint64_t)lp * plane_step + off;
     return it;
 }
 

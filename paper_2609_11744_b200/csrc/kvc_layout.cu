@@ -212,6 +212,7 @@ kvc_status copy_one(kvc_layout *lay, int dir, const int32_t *ids, uint32_t n_blo
     if (s != KVC_OK)
         return s;
     a.slot = (uint64_t)(uintptr_t)slot;
+    kvc_chunk_steps(lay, n_blocks, &a.ent_step, &a.plane_step);
     if (ids_on_device)
         a.dev_ids = ids;
     else
@@ -311,11 +312,13 @@ kvc_status copy_batch(kvc_layout *lay, int dir, const kvc_chunk_op *ops, uint32_
         return s;
     uint64_t k = 0;
     for (uint32_t i = 0; i < n_ops; ++i) {
+        uint64_t ent_step, plane_step;
+        kvc_chunk_steps(lay, ops[i].n_blocks, &ent_step, &plane_step);
         for (uint32_t j = 0; j < ops[i].n_blocks; ++j, ++k) {
             KvcEnt &e = ar->host[k];
-            e.slot_addr = (uint64_t)(uintptr_t)ops[i].slot + (uint64_t)j * lay->slab_bytes;
+            e.slot_addr = (uint64_t)(uintptr_t)ops[i].slot + (uint64_t)j * ent_step;
             e.nb_c = ops[i].n_blocks;
-            e.pad = 0;
+            e.plane_step = plane_step;
             if (ids_on_device) {
                 e.id_or_ptr = (uint64_t)(uintptr_t)(ops[i].ids + j);
                 e.id_is_ptr = 1;
@@ -377,6 +380,9 @@ kvc_status kvc_layout_create(const kvc_layout_desc *d, kvc_layout **out)
         return KVC_ERR_INVALID_ARG;
     if (d->chunk_tokens % d->block_size)
         return KVC_ERR_INVALID_ARG;
+    if ((d->chunk_order != KVC_CHUNK_LAYER_MAJOR && d->chunk_order != KVC_CHUNK_BLOCK_MAJOR) ||
+        d->reserved != 0)
+        return KVC_ERR_INVALID_ARG;
     if (!d->plane_ptrs && !d->base)
         return KVC_ERR_INVALID_ARG;
     const uint64_t row = (uint64_t)d->num_kv_heads * d->head_dim * d->elem_bytes;
@@ -399,10 +405,18 @@ kvc_status kvc_layout_create(const kvc_layout_desc *d, kvc_layout **out)
     } else {
         if (!mult16((uintptr_t)d->base) || !mult16(d->layer_stride) || !mult16(d->plane_stride))
             return KVC_ERR_ALIGNMENT;
+        // Two ways to keep planes from overlapping: every plane is its own range
+        // ([L][P][NB][..], plane stride >= one plane), or the planes of a layer interleave inside
+        // the block axis ([L][NB][P][..], block stride >= planes * plane stride >= planes * slab).
         const uint64_t plane_span = (uint64_t)(d->num_blocks - 1) * bstride + slab;
-        if (d->kv_planes > 1 && d->plane_stride < plane_span)
+        const bool disjoint = d->kv_planes == 1 || d->plane_stride >= plane_span;
+        const bool interleaved = d->plane_stride >= slab && bstride >= d->kv_planes * d->plane_stride;
+        if (!disjoint && !interleaved)
             return KVC_ERR_INVALID_ARG;
-        if (d->num_layers > 1 && d->layer_stride < plane_span)
+        const uint64_t layer_span =
+            disjoint ? (uint64_t)(d->kv_planes - 1) * d->plane_stride + plane_span
+                     : (uint64_t)(d->num_blocks - 1) * bstride + (uint64_t)d->kv_planes * d->plane_stride;
+        if (d->num_layers > 1 && d->layer_stride < layer_span)
             return KVC_ERR_INVALID_ARG;
     }
     kvc_layout *lay = new (std::nothrow) kvc_layout();

@@ -26,6 +26,7 @@ KVC_OK, KVC_ERR_INVALID_ARG, KVC_ERR_OUT_OF_RANGE, KVC_ERR_ALIGNMENT, KVC_ERR_CO
 KVC_VARIANT_AUTO, KVC_VARIANT_VEC, KVC_VARIANT_BULK = 0, 1, 2
 KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR = 0, 1, 2
 KVC_RING_DEVICE, KVC_RING_HOST_MAPPED = 0, 1
+KVC_CHUNK_LAYER_MAJOR, KVC_CHUNK_BLOCK_MAJOR = 0, 1
 KVC_MAP_FULL_CHUNKS_ONLY = 1
 
 
@@ -44,7 +45,8 @@ class kvc_layout_desc(ctypes.Structure):
                 ("elem_bytes", ctypes.c_uint32), ("chunk_tokens", ctypes.c_uint32),
                 ("plane_ptrs", ctypes.POINTER(ctypes.c_void_p)), ("base", ctypes.c_void_p),
                 ("layer_stride", ctypes.c_uint64), ("plane_stride", ctypes.c_uint64),
-                ("block_stride", ctypes.c_uint64)]
+                ("block_stride", ctypes.c_uint64), ("chunk_order", ctypes.c_uint32),
+                ("reserved", ctypes.c_uint32)]
 
 
 class kvc_tuning(ctypes.Structure):
@@ -113,6 +115,8 @@ def lib() -> ctypes.CDLL:
         "kvc_pack_batch": (ci, [vp, vp, u32, ci, vp]),
         "kvc_unpack_batch": (ci, [vp, vp, u32, ci, vp]),
         "kvc_pack_batch_static": (ci, [vp, vp, u32, vp]),
+        "kvc_pack_copy_engine": (ci, [vp, vp, u32, vp, u64, vp]),
+        "kvc_unpack_copy_engine": (ci, [vp, vp, u64, vp, u32, vp]),
         "kvc_poll_device_status": (ci, [vp, vp, P(u32), P(u32)]),
         "kvc_layout_launch_count": (u64, [vp]),
         "kvc_staging_ring_create": (ci, [u64, u32, ci, vp, u64, P(vp)]),
@@ -214,7 +218,8 @@ class LayoutHandle:
 def kvc_layout_create(num_layers: int, kv_planes: int, num_blocks: int, block_size: int,
                       num_kv_heads: int, head_dim: int, elem_bytes: int, chunk_tokens: int,
                       base=None, layer_stride: int = 0, plane_stride: int = 0,
-                      block_stride: int = 0, plane_ptrs: Optional[Sequence] = None) -> LayoutHandle:
+                      block_stride: int = 0, plane_ptrs: Optional[Sequence] = None,
+                      chunk_order: int = 0) -> LayoutHandle:
     d = kvc_layout_desc(num_layers, kv_planes, num_blocks, block_size, num_kv_heads, head_dim,
                         elem_bytes, chunk_tokens)
     keep = [base, plane_ptrs]
@@ -227,19 +232,20 @@ def kvc_layout_create(num_layers: int, kv_planes: int, num_blocks: int, block_si
         d.base = _ptr(base)
         d.layer_stride, d.plane_stride = layer_stride, plane_stride
     d.block_stride = block_stride
+    d.chunk_order = chunk_order
     out = ctypes.c_void_p()
     _check(lib().kvc_layout_create(ctypes.byref(d), ctypes.byref(out)), "kvc_layout_create")
     return LayoutHandle(out.value, keep)
 
 
 def kvc_layout_create_dense(pool, num_layers, kv_planes, num_blocks, block_size, num_kv_heads,
-                            head_dim, elem_bytes, chunk_tokens) -> LayoutHandle:
+                            head_dim, elem_bytes, chunk_tokens, chunk_order: int = 0) -> LayoutHandle:
     """Layout over one dense allocation [L][P][NB][B][H][D] (a tensor or a device address)."""
     slab = block_size * num_kv_heads * head_dim * elem_bytes
     plane = slab * num_blocks
     return kvc_layout_create(num_layers, kv_planes, num_blocks, block_size, num_kv_heads, head_dim,
                              elem_bytes, chunk_tokens, base=pool, layer_stride=plane * kv_planes,
-                             plane_stride=plane)
+                             plane_stride=plane, chunk_order=chunk_order)
 
 
 def kvc_layout_destroy(layout: LayoutHandle) -> None:
@@ -322,6 +328,25 @@ def kvc_unpack(layout, src_slot, ids, slot_bytes: Optional[int] = None, stream=N
     nb = _nbytes(src_slot) if slot_bytes is None else slot_bytes
     _check(lib().kvc_unpack(layout.handle, _ptr(src_slot), nb, p, n, dev, _stream(stream)),
            "kvc_unpack")
+
+
+def kvc_pack_copy_engine(layout, ids, dst, dst_bytes: Optional[int] = None, stream=None) -> None:
+    """kvc_pack done by the DMA engines (strided async copies); dst may be pinned host memory."""
+    keep, p, n, dev = _ids(ids)
+    if dev:
+        raise TypeError("the copy-engine variants take host-resident ids")
+    nb = _nbytes(dst) if dst_bytes is None else dst_bytes
+    _check(lib().kvc_pack_copy_engine(layout.handle, p, n, _ptr(dst), nb, _stream(stream)),
+           "kvc_pack_copy_engine")
+
+
+def kvc_unpack_copy_engine(layout, src, ids, src_bytes: Optional[int] = None, stream=None) -> None:
+    keep, p, n, dev = _ids(ids)
+    if dev:
+        raise TypeError("the copy-engine variants take host-resident ids")
+    nb = _nbytes(src) if src_bytes is None else src_bytes
+    _check(lib().kvc_unpack_copy_engine(layout.handle, _ptr(src), nb, p, n, _stream(stream)),
+           "kvc_unpack_copy_engine")
 
 
 def make_chunk_ops(slot_addrs, ids_addrs, n_blocks) -> np.ndarray:

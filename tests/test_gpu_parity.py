@@ -395,3 +395,190 @@ def test_prefix_streamed_through_ring_equals_one_shot_pack(kind):
     assert np.array_equal(pool_t.cpu().numpy(), want_pool)
     kvc.kvc_staging_ring_destroy(ring)
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+# ------------------------------------------------------------------ copy-engine variants (DMA, no kernel)
+@pytest.mark.parametrize("pool_kind", ["dense", "layer_gap", "separate_planes"])
+@pytest.mark.parametrize("host_side", [False, True])
+def test_copy_engine_variants_match_oracle(pool_kind, host_side):
+    """kvc_pack_copy_engine / kvc_unpack_copy_engine move the same bytes with strided DMA copies:
+    one per block (dense pool), one per layer (layers not equally spaced) or one per plane
+    (separate allocations); the chunk may live in device memory or in pinned host memory."""
+    g = orc.Dims(3, 2, 40, 16, 4, 64, 2)
+    plane_bytes = g.NB * g.slab_bytes
+    planes_np = [wl.random_bits(300 + i, plane_bytes) for i in range(g.L * g.P)]
+    if pool_kind == "separate_planes":
+        planes_t = [to_dev(p) for p in planes_np]
+        lay = kvc.kvc_layout_create(g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 64, plane_ptrs=planes_t)
+        views = planes_t
+    else:
+        gap = 4096 if pool_kind == "layer_gap" else 0
+        layer_stride = g.P * plane_bytes + gap
+        buf = torch.full((g.L * layer_stride,), 0xEE, dtype=torch.uint8, device=DEV)
+        views = []
+        for l in range(g.L):
+            for p in range(g.P):
+                v = buf[l * layer_stride + p * plane_bytes:][:plane_bytes]
+                v.copy_(to_dev(planes_np[l * g.P + p]))
+                views.append(v)
+        lay = kvc.kvc_layout_create(g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 64, base=buf,
+                                    layer_stride=layer_stride, plane_stride=plane_bytes)
+    src, dst = wl.block_ids(31, g.NB, 11), wl.block_ids(32, g.NB, 11)
+    total = 11 * g.bytes_per_block
+    if host_side:
+        staging = torch.full((total + 4096,), 0x44, dtype=torch.uint8).pin_memory()
+    else:
+        staging = torch.full((total + 4096,), 0x44, dtype=torch.uint8, device=DEV)
+    launches0 = kvc.kvc_layout_launch_count(lay)
+    off = 0
+    want_chunks = []
+    for f, nb in orc.chunk_ranges(11, 4):
+        nbytes = kvc.kvc_layout_chunk_bytes(lay, nb)
+        kvc.kvc_pack_copy_engine(lay, src[f:f + nb], staging.data_ptr() + off, nbytes)
+        want_chunks.append(orc.pack_chunk_planes(g, planes_np, src[f:f + nb]))
+        off += nbytes
+    torch.cuda.synchronize()
+    host = staging.cpu().numpy()
+    assert np.array_equal(host[:total], np.concatenate(want_chunks))
+    assert (host[total:] == 0x44).all()
+    off = 0
+    want_planes = [p.copy() for p in planes_np]
+    for (f, nb), ch in zip(orc.chunk_ranges(11, 4), want_chunks):
+        kvc.kvc_unpack_copy_engine(lay, staging.data_ptr() + off, dst[f:f + nb], ch.size)
+        orc.unpack_chunk_planes(g, want_planes, ch, dst[f:f + nb])
+        off += ch.size
+    torch.cuda.synchronize()
+    for v, wnt in zip(views, want_planes):
+        assert np.array_equal(v.cpu().numpy(), wnt)
+    if pool_kind == "layer_gap":
+        b2 = buf.cpu().numpy().reshape(g.L, -1)
+        assert (b2[:, g.P * plane_bytes:] == 0xEE).all()      # the gap between layers is untouched
+    assert kvc.kvc_layout_launch_count(lay) == launches0      # no kernel ran
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_unpack_copy_engine(lay, staging.data_ptr(), np.array([1, 2, 1], np.int32), total)
+    assert e.value.status == kvc.KVC_ERR_CONFLICT
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_pack_copy_engine(lay, np.array([g.NB], np.int32), staging.data_ptr(), total)
+    assert e.value.status == kvc.KVC_ERR_OUT_OF_RANGE
+
+
+# ------------------------------------------------------------------ random tiny layouts
+def test_random_tiny_layouts():
+    """Seeded random geometries (any element size, planes per layer, block size; slab bytes a
+    multiple of 16), random tables, chunk sizes, kernels, tiles and traversal orders; host and
+    device ids; per-chunk and batched calls.  Every case byte for byte against the oracle."""
+    rng = np.random.default_rng(20260911)
+    done = 0
+    while done < 40:
+        e = int(rng.choice([1, 2, 4]))
+        L, P = int(rng.integers(1, 5)), int(rng.integers(1, 3))
+        B, H = int(rng.integers(1, 9)), int(rng.integers(1, 5))
+        D = int(rng.choice([8, 16, 24, 32, 40, 64, 128]))
+        S = B * H * D * e
+        if S % 16:
+            continue
+        NB = int(rng.integers(2, 60))
+        g = orc.Dims(L, P, NB, B, H, D, e)
+        n = int(rng.integers(1, NB + 1))
+        bpc = int(rng.integers(1, n + 2))
+        pool = wl.random_bits(int(rng.integers(1 << 30)), g.pool_bytes + (g.pool_bytes & 1))[:g.pool_bytes]
+        src = rng.permutation(NB)[:n].astype(np.int32)
+        dst = rng.permutation(NB)[:n].astype(np.int32)
+        variant = int(rng.choice(VARIANTS))
+        order = int(rng.choice([1, 2]))
+        tile = int(rng.choice([0, 16, 48, 256, 4096]))
+        mode = str(rng.choice(["chunk", "chunk_dev", "batch", "batch_dev"]))
+        run_pack_unpack(g, pool, src, dst, bpc * B, variant, order, mode, tile)
+        done += 1
+
+
+# ------------------------------------------------------------------ layout variants
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("mode", ["chunk", "batch_dev", "copy_engine", "static"])
+def test_block_major_chunk_order(variant, mode):
+    """Chunks in block-major order [n][L][P][B][H][D] through every entry point."""
+    g = orc.Dims(4, 2, 48, 16, 4, 64, 2)
+    pool = wl.random_bits(500, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 64,
+                                      chunk_order=kvc.KVC_CHUNK_BLOCK_MAJOR)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    src, dst = wl.block_ids(51, g.NB, 14), wl.block_ids(52, g.NB, 14)
+    total = 14 * g.bytes_per_block
+    staging = torch.full((total + 4096,), 0x66, dtype=torch.uint8, device=DEV)
+    ranges = orc.chunk_ranges(14, 4)
+    planes = orc.dense_planes(g, pool)
+    want_chunks = [orc.pack_chunk_planes_block_major(g, planes, src[f:f + nb]) for f, nb in ranges]
+
+    def run(direction, ids):
+        if mode == "batch_dev" or (mode == "static" and direction == 1):
+            ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, to_dev(ids), staging)
+            (kvc.kvc_pack_batch if direction == 0 else kvc.kvc_unpack_batch)(lay, ops, dev)
+        elif mode == "static":
+            ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, ids, staging)
+            kvc.kvc_pack_batch_static(lay, ops)
+        else:
+            off = 0
+            for f, nb in ranges:
+                nbytes = kvc.kvc_layout_chunk_bytes(lay, nb)
+                slot = staging[off:off + nbytes]
+                if mode == "chunk":
+                    (kvc.kvc_pack(lay, ids[f:f + nb], slot) if direction == 0
+                     else kvc.kvc_unpack(lay, slot, ids[f:f + nb]))
+                else:
+                    (kvc.kvc_pack_copy_engine(lay, ids[f:f + nb], slot) if direction == 0
+                     else kvc.kvc_unpack_copy_engine(lay, slot, ids[f:f + nb]))
+                off += nbytes
+        torch.cuda.synchronize()
+
+    run(0, src)
+    host = staging.cpu().numpy()
+    assert np.array_equal(host[:total], np.concatenate(want_chunks))
+    assert (host[total:] == 0x66).all()
+    # the short last chunk is a prefix of what a full chunk starting there would be
+    run(1, dst)
+    want_pool = pool.copy()
+    for (f, nb), ch in zip(ranges, want_chunks):
+        orc.unpack_chunk_planes_block_major(g, orc.dense_planes(g, want_pool), ch, dst[f:f + nb])
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+@pytest.mark.parametrize("variant", VARIANTS)
+@pytest.mark.parametrize("chunk_order", [kvc.KVC_CHUNK_LAYER_MAJOR, kvc.KVC_CHUNK_BLOCK_MAJOR])
+def test_pool_with_kv_inside_the_block_axis(variant, chunk_order):
+    """Pool order [L][NB][P][B][H][D] (K and V of a block adjacent): described by plane stride S and
+    block stride P*S.  Chunks equal those of the same data in the dense order."""
+    g = orc.Dims(3, 2, 30, 16, 4, 64, 2)
+    S = g.slab_bytes
+    dense = wl.random_bits(600, g.pool_bytes)
+    inter = np.ascontiguousarray(dense.reshape(g.L, g.P, g.NB, S).transpose(0, 2, 1, 3)).reshape(-1)
+    pool_t = to_dev(inter)
+    lay = kvc.kvc_layout_create(g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 64, base=pool_t,
+                                layer_stride=g.NB * g.P * S, plane_stride=S, block_stride=g.P * S,
+                                chunk_order=chunk_order)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    src, dst = wl.block_ids(61, g.NB, 9), wl.block_ids(62, g.NB, 9)
+    staging = torch.zeros(9 * g.bytes_per_block, dtype=torch.uint8, device=DEV)
+    ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, src, staging)
+    kvc.kvc_pack_batch(lay, ops, dev)
+    torch.cuda.synchronize()
+    planes = orc.dense_planes(g, dense)
+    packer = (orc.pack_chunk_planes if chunk_order == kvc.KVC_CHUNK_LAYER_MAJOR
+              else orc.pack_chunk_planes_block_major)
+    unpacker = (orc.unpack_chunk_planes if chunk_order == kvc.KVC_CHUNK_LAYER_MAJOR
+                else orc.unpack_chunk_planes_block_major)
+    chunks = [packer(g, planes, src[f:f + nb]) for f, nb in orc.chunk_ranges(9, 4)]
+    assert np.array_equal(staging.cpu().numpy(), np.concatenate(chunks))
+    # copy-engine pack of the first chunk gives the same bytes
+    again = torch.zeros(chunks[0].size, dtype=torch.uint8, device=DEV)
+    kvc.kvc_pack_copy_engine(lay, src[:4], again)
+    ops2, keep2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+    kvc.kvc_unpack_batch(lay, ops2, dev)
+    torch.cuda.synchronize()
+    assert np.array_equal(again.cpu().numpy(), chunks[0])
+    want = dense.copy()
+    for (f, nb), ch in zip(orc.chunk_ranges(9, 4), chunks):
+        unpacker(g, orc.dense_planes(g, want), ch, dst[f:f + nb])
+    want_inter = np.ascontiguousarray(want.reshape(g.L, g.P, g.NB, S).transpose(0, 2, 1, 3)).reshape(-1)
+    assert np.array_equal(pool_t.cpu().numpy(), want_inter)

@@ -298,3 +298,53 @@ def test_dedup_ops_small_cases():
     assert len(kept2) == 4
     # a shorter tail chunk that is a prefix of a longer one is dropped
     assert orc.dedup_ops([[1, 2, 3], [1, 2, 3, 4]], 2) == [(0, 0, 0, 2), (1, 1, 2, 2)]
+
+
+# ---------------------------------------------------------------- block-major chunk order
+def test_block_major_chunk_order_pins():
+    g = Dims(L=3, P=2, NB=11, B=2, H=3, D=4, e=4)
+    pool = _tag_pool(g)                       # value = own dense pool index
+    planes = orc.dense_planes(g, pool)
+    rng = np.random.default_rng(21)
+    for n in (1, 4, 7):
+        ids = rng.permutation(g.NB)[:n].astype(np.int32)
+        ch = orc.pack_chunk_planes_block_major(g, planes, ids).view(np.uint32)
+        # decode each chunk position with numpy over the block-major shape
+        j, l, p, t, h, d = np.unravel_index(np.arange(ch.size), (n, g.L, g.P, g.B, g.H, g.D))
+        want = np.ravel_multi_index((l, p, ids[j], t, h, d), (g.L, g.P, g.NB, g.B, g.H, g.D))
+        assert np.array_equal(ch, want.astype(np.uint32))
+        # it is the layer-major chunk with the block axis moved to the front (library routine)
+        lm = orc.pack_chunk(g, pool, ids).view(np.uint32).reshape(g.L, g.P, n, -1)
+        assert np.array_equal(ch, np.moveaxis(lm, 2, 0).reshape(-1))
+        # a shorter chunk is a prefix of a longer one (what makes the order attractive for files)
+        if n > 1:
+            shorter = orc.pack_chunk_planes_block_major(g, planes, ids[:n - 1])
+            assert np.array_equal(shorter, ch.view(np.uint8)[:shorter.size])
+        # formula against numpy
+        for _ in range(50):
+            c = tuple(int(rng.integers(0, s)) for s in (g.L, g.P, n, g.B, g.H, g.D))
+            assert orc.chunk_elem_block_major(g, n, *c) == np.ravel_multi_index(
+                (c[2], c[0], c[1], c[3], c[4], c[5]), (n, g.L, g.P, g.B, g.H, g.D))
+        # round trip into a sentinel pool
+        fresh = np.full(g.pool_bytes, 0xEE, dtype=np.uint8)
+        orc.unpack_chunk_planes_block_major(g, orc.dense_planes(g, fresh), ch.view(np.uint8), ids)
+        a, b = pool.reshape(g.L, g.P, g.NB, -1), fresh.reshape(g.L, g.P, g.NB, -1)
+        assert np.array_equal(a[:, :, ids], b[:, :, ids])
+        rest = np.setdiff1d(np.arange(g.NB), ids)
+        assert (b[:, :, rest] == 0xEE).all()
+
+
+def test_interleaved_kv_pool_order_is_a_strided_plane_view():
+    """A pool laid out [L][NB][P][B][H][D] (K|V inside the block axis) is the same data seen as
+    planes with plane stride S and block stride P*S: its chunks equal those of the dense pool."""
+    g = Dims(L=2, P=2, NB=9, B=4, H=2, D=8, e=2)
+    rng = np.random.default_rng(23)
+    dense = rng.integers(0, 256, g.pool_bytes, dtype=np.uint8)
+    S = g.slab_bytes
+    inter = np.ascontiguousarray(
+        dense.reshape(g.L, g.P, g.NB, S).transpose(0, 2, 1, 3)).reshape(-1)   # [L][NB][P][S]
+    layer = g.NB * g.P * S
+    planes = [inter[l * layer + p * S:] for l in range(g.L) for p in range(g.P)]
+    planes = [pl[:(g.NB - 1) * g.P * S + S] for pl in planes]
+    ids = rng.permutation(g.NB)[:5].astype(np.int32)
+    assert np.array_equal(orc.pack_chunk_planes(g, planes, ids, g.P * S), orc.pack_chunk(g, dense, ids))
