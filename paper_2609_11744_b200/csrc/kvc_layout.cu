@@ -128,7 +128,8 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     a->status = lay->d_status;
     uint64_t grid = variant == KVC_VARIANT_BULK
                         ? (uint64_t)lay->sm_count * (t.ctas_per_sm ? t.ctas_per_sm : 1u)
-                        : (uint64_t)lay->sm_count * (uint64_t)lay->vec_blocks_per_sm;
+                        : (uint64_t)lay->sm_count *
+                              std::min<uint64_t>(lay->vec_blocks_per_sm, KVC_VEC_DEFAULT_BLOCKS_PER_SM);
     if (t.max_ctas)
         grid = std::min<uint64_t>(grid, t.max_ctas);
     grid = std::min<uint64_t>(grid, n_items);
