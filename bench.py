@@ -772,6 +772,52 @@ def suite_host_link(torch, cuda_rt, dev):
     return out
 
 
+def suite_file_pipeline(torch, kvc, dev, root):
+    """f1: a 32k-token prefix (8B shape, 4 GiB) offloaded to chunk files and loaded back through an
+    8-slot mapped-host ring, with 4 I/O threads, kernel copies and copy-engine copies.  `root` is
+    where the files go (the box's scratch disk, or /dev/shm as the memory-backed upper bound)."""
+    import shutil
+    import tempfile
+    w = wl.WORKLOADS["8b_ring"]
+    s, NB, n = w.shape, w.pool_blocks, w.request_blocks
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    src, dst = wl.block_ids(w.seed, NB, n), wl.block_ids(w.dst_seed, NB, n)
+    out = []
+    for base in root.split(","):
+        if not os.path.isdir(base):
+            continue
+        for use_ce in (False, True):
+            d = tempfile.mkdtemp(prefix="kvc_suite_", dir=base)
+            try:
+                lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+                kvc.kvc_layout_set_tuning(lay, max_ctas=16)
+                cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+                ring = kvc.kvc_staging_ring_create(cb, 8, kvc.KVC_RING_HOST_MAPPED)
+                store = kvc.kvc_store_open(d, "8b", direct_io=True)
+                hashes = [kvc.kvc_fnv1a64(b"chunk%d" % c) for c in range(kvc.kvc_layout_num_chunks(lay, n))]
+                st = kvc.kvc_pipeline_store(lay, ring, store, src, hashes, io_threads=4,
+                                            use_copy_engine=use_ce)
+                torch.cuda.synchronize()
+                t0 = time.perf_counter()
+                ld = kvc.kvc_pipeline_load(lay, ring, store, dst, hashes, io_threads=4,
+                                           use_copy_engine=use_ce)
+                torch.cuda.synchronize()
+                load_s = time.perf_counter() - t0
+                out.append({"root": base, "copies": "copy engines" if use_ce else "kernels (16 CTAs)",
+                            "bytes": st["bytes"], "store_s": st["seconds"],
+                            "store_gbs": st["bytes"] / st["seconds"] / 1e9,
+                            "load_s": load_s, "load_gbs": ld["bytes"] / load_s / 1e9,
+                            "chunks": st["chunks"], "published": st["published"],
+                            "direct_io_refused": kvc.kvc_store_direct_io_refused(store),
+                            "ring_stalls_store": st["ring_stalls"]})
+                kvc.kvc_store_close(store)
+                kvc.kvc_staging_ring_destroy(ring)
+                kvc.kvc_layout_destroy(lay)
+            finally:
+                shutil.rmtree(d, ignore_errors=True)
+    return out
+
+
 def run_suite(args):
     import torch
     from paper_2609_11744_b200 import cuda_rt, kvc
@@ -784,7 +830,8 @@ def run_suite(args):
                      ("prefix_8k", lambda: suite_8k(torch, kvc, dev, args.steps)),
                      ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
                      ("ring_overlap", lambda: suite_ring_overlap(torch, kvc, cuda_rt, dev,
-                                                                 args.overlap_seconds))):
+                                                                 args.overlap_seconds)),
+                     ("file_pipeline", lambda: suite_file_pipeline(torch, kvc, dev, args.file_roots))):
         if "all" in parts or name in parts:
             out[name] = fn()
             torch.cuda.synchronize()
@@ -816,8 +863,10 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
-                         "host_link,chunk_sweep,prefix_8k,batch_70b,ring_overlap (1 GPU; prints one JSON line)")
+                         "host_link,chunk_sweep,prefix_8k,batch_70b,ring_overlap,file_pipeline (1 GPU; prints one JSON line)")
     ap.add_argument("--overlap-seconds", type=float, default=2.0)
+    ap.add_argument("--file-roots", default="/tmp,/dev/shm",
+                    help="comma list of directories for the file_pipeline suite part")
     ap.add_argument("--traffic-bytes", type=float, default=None,
                     help="DRAM bytes per launch from an ncu capture, copied into the roofline object "
                          "(default: the committed capture of the default workload, else null)")

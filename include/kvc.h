@@ -52,7 +52,10 @@ typedef enum {
     KVC_ERR_WOULD_BLOCK = 7,  /* ring: no free slot and timeout_us == 0 */
     KVC_ERR_TIMEOUT = 8,      /* ring: no free slot before the deadline */
     KVC_ERR_STATE = 9,        /* ring: call does not fit the slot's state */
-    KVC_ERR_TOO_LARGE = 10    /* more work than a fixed-capacity entry point can take in one call */
+    KVC_ERR_TOO_LARGE = 10,   /* more work than a fixed-capacity entry point can take in one call */
+    KVC_ERR_EXISTS = 11,      /* store: the entry is already published (first writer wins) */
+    KVC_ERR_NOT_FOUND = 12,   /* store: no entry for this hash */
+    KVC_ERR_IO = 13           /* store: a file-system call failed, or an entry has the wrong size */
 } kvc_status;
 
 const char *kvc_status_str(kvc_status s);
@@ -279,12 +282,90 @@ kvc_status kvc_staging_ring_wait_filled(kvc_ring *ring, uint32_t slot, void *con
 /* Records the slot's "drained" event on the consumer stream; the slot becomes free when that
  * event completes.  STATE unless committed. */
 kvc_status kvc_staging_ring_release(kvc_ring *ring, uint32_t slot, void *consumer_stream);
+/* Host-side producers and consumers (file reads and writes on mapped pinned slots):
+ * commit_host marks an acquired slot filled by the host (no event; wait_filled then adds no
+ * dependency), sync_filled blocks the calling host thread until the slot's "filled" event has
+ * completed (may be called from a worker thread, for distinct slots concurrently with other ring
+ * calls), release_host frees a filled slot at once because its consumer was the host and is done.
+ * STATE unless the slot is acquired (commit_host) or filled (the other two). */
+kvc_status kvc_staging_ring_commit_host(kvc_ring *ring, uint32_t slot);
+kvc_status kvc_staging_ring_sync_filled(kvc_ring *ring, uint32_t slot);
+kvc_status kvc_staging_ring_release_host(kvc_ring *ring, uint32_t slot);
 /* in_flight = slots acquired and not yet observed free; stalls = acquire polls that found the
  * next slot still busy.  Any pointer may be NULL. */
 kvc_status kvc_staging_ring_stats(const kvc_ring *ring, uint32_t *in_flight, uint64_t *acquires,
                                   uint64_t *stalls);
 uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *ring);
 uint32_t kvc_staging_ring_num_slots(const kvc_ring *ring);
+
+/* ------------------------------------------------------------------ chunk files (Sec. 6.3) */
+
+/* The step behind the ring: one file per chunk in a hash-addressed directory tree that several
+ * engine instances can share (Sec. 6.3).  Host only; every pointer is HOST memory.
+ * Path of an entry: <root>/<model_tag>/<hh>/<hh>/<16 hex digits of the hash>.kv, the two
+ * directory levels taken from the top two bytes of the hash.
+ * Publication is first-writer-wins: the data goes to a uniquely named temporary file in the
+ * target directory, a hard link creates the final name atomically (KVC_ERR_EXISTS if another
+ * writer was first; the existing entry is kept), the temporary name is removed.  Readers open
+ * final names only, so an entry is either absent or complete.
+ * direct_io != 0: files are opened with O_DIRECT when the buffer is 4096-byte aligned and the
+ * size a multiple of 4096 (ring slots are); where the file system refuses the flag the call
+ * falls back to buffered I/O and counts it (kvc_store_direct_io_refused).
+ * A store handle may be used from several threads at once. */
+typedef struct kvc_store kvc_store;
+kvc_status kvc_store_open(const char *root, const char *model_tag, int direct_io, kvc_store **out);
+kvc_status kvc_store_close(kvc_store *store);
+/* Writes the entry's path (NUL-terminated) into buf.  INVALID_ARG if cap is too small. */
+kvc_status kvc_store_path(const kvc_store *store, uint64_t hash, char *buf, uint32_t cap);
+/* KVC_OK and the file size, or KVC_ERR_NOT_FOUND (size 0). */
+kvc_status kvc_store_lookup(const kvc_store *store, uint64_t hash, uint64_t *bytes);
+/* Errors: INVALID_ARG, EXISTS, IO. */
+kvc_status kvc_store_publish(kvc_store *store, uint64_t hash, const void *host_buf, uint64_t bytes);
+/* Reads exactly `bytes`; INVALID_ARG if the entry has another size.  Errors: NOT_FOUND, IO. */
+kvc_status kvc_store_read(kvc_store *store, uint64_t hash, void *host_buf, uint64_t bytes);
+int kvc_store_direct_io_refused(const kvc_store *store);
+
+/* Prefix-hash chaining (Sec. 2.1): the hash of a block covers its tokens and the hash of the
+ * block before it, so two requests share an entry only if they agree from the first token on.
+ * 64-bit FNV-1a over the 8 bytes of `prev` (little endian) followed by the tokens' bytes;
+ * prev = 0 starts a chain.  kvc_fnv1a64 is the plain hash of a byte string. */
+uint64_t kvc_chain_hash(uint64_t prev, const int32_t *tokens, uint32_t n_tokens);
+uint64_t kvc_fnv1a64(const void *data, uint64_t n);
+
+/* ------------------------------------------------------------------ store / load pipelines (Sec. 6.4) */
+
+typedef struct {
+    uint64_t bytes;           /* chunk bytes written to / read from files */
+    double seconds;           /* wall time of the call */
+    uint32_t chunks;          /* chunks processed (load: length of the prefix that was present) */
+    uint32_t published;       /* store: files this call created */
+    uint32_t already_present; /* store: chunks another writer had published already */
+    uint32_t ring_stalls;     /* polls that found no free slot */
+} kvc_pipeline_stats;
+
+/* Offload one request to chunk files: for every chunk (kvc_map_request order) acquire a ring slot,
+ * pack the chunk's blocks into it on `stream`, and let one of `io_threads` (0 = 4) host threads
+ * publish the slot as the file named by hashes[c] once its copy has completed; the slot returns
+ * to the ring when the file is written.  `ring` must be a KVC_RING_HOST_MAPPED ring whose slots
+ * hold a full chunk; the request may be far larger than the ring.  use_copy_engine != 0 packs
+ * with the DMA engines (kvc_pack_copy_engine) instead of a kernel.  ids and hashes are HOST
+ * arrays; n_hashes >= number of chunks.  Returns when every file is published.
+ * kvc_pipeline_load is the reverse: it looks up the chunks in order, stops at the first one that
+ * is missing or has the wrong size (only a contiguous prefix is usable, Sec. 2.1), reads the rest
+ * into ring slots with the host threads and unpacks each slot into ids on `stream` as it arrives.
+ * It returns when all files are read and all unpacks are ENQUEUED: synchronise `stream` before
+ * using the blocks.  stats->chunks * blocks_per_chunk (capped by n_blocks) blocks were loaded.
+ * Neither call is re-entrant on the same ring.
+ * Errors: INVALID_ARG (no host-visible slots, slot too small, too few hashes), TIMEOUT, and
+ * whatever pack / unpack / the store report. */
+kvc_status kvc_pipeline_store(kvc_layout *layout, kvc_ring *ring, kvc_store *store, const int32_t *ids,
+                              uint32_t n_blocks, const uint64_t *hashes, uint32_t n_hashes,
+                              uint32_t io_threads, int use_copy_engine, void *stream,
+                              kvc_pipeline_stats *stats);
+kvc_status kvc_pipeline_load(kvc_layout *layout, kvc_ring *ring, kvc_store *store, const int32_t *ids,
+                             uint32_t n_blocks, const uint64_t *hashes, uint32_t n_hashes,
+                             uint32_t io_threads, int use_copy_engine, void *stream,
+                             kvc_pipeline_stats *stats);
 
 /* Event provider used by a ring.  The default one wraps CUDA events.  Tests replace it to
  * drive the slot state machine on a machine without a GPU (events that complete on command);

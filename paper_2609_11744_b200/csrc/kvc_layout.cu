@@ -365,6 +365,9 @@ const char *kvc_status_str(kvc_status s)
     case KVC_ERR_TIMEOUT: return "timed out waiting for a staging slot";
     case KVC_ERR_STATE: return "call does not fit the slot's state";
     case KVC_ERR_TOO_LARGE: return "more blocks or planes than this fixed-capacity entry point takes per call";
+    case KVC_ERR_EXISTS: return "entry already published";
+    case KVC_ERR_NOT_FOUND: return "no such entry";
+    case KVC_ERR_IO: return "file-system call failed or entry has the wrong size";
     }
     return "unknown status";
 }

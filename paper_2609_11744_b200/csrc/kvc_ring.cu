@@ -57,6 +57,7 @@ struct Slot {
     SlotState state = SLOT_FREE;
     void *filled = nullptr;
     void *drained = nullptr;
+    bool filled_by_host = false;  // committed by kvc_staging_ring_commit_host: no event to wait for
 };
 
 }  // namespace
@@ -268,6 +269,7 @@ kvc_status kvc_staging_ring_commit(kvc_ring *r, uint32_t slot, void *producer_st
         return KVC_ERR_STATE;
     if (r->ev.record(r->ev.ctx, s.filled, producer_stream) != 0)
         return KVC_ERR_CUDA;
+    s.filled_by_host = false;
     s.state = SLOT_FILLED;
     return KVC_OK;
 }
@@ -279,7 +281,7 @@ kvc_status kvc_staging_ring_wait_filled(kvc_ring *r, uint32_t slot, void *consum
     Slot &s = r->slots[slot];
     if (s.state != SLOT_FILLED)
         return KVC_ERR_STATE;
-    if (r->ev.stream_wait(r->ev.ctx, consumer_stream, s.filled) != 0)
+    if (!s.filled_by_host && r->ev.stream_wait(r->ev.ctx, consumer_stream, s.filled) != 0)
         return KVC_ERR_CUDA;
     return KVC_OK;
 }
@@ -294,6 +296,41 @@ kvc_status kvc_staging_ring_release(kvc_ring *r, uint32_t slot, void *consumer_s
     if (r->ev.record(r->ev.ctx, s.drained, consumer_stream) != 0)
         return KVC_ERR_CUDA;
     s.state = SLOT_DRAINING;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_commit_host(kvc_ring *r, uint32_t slot)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[slot];
+    if (s.state != SLOT_ACQUIRED)
+        return KVC_ERR_STATE;
+    s.filled_by_host = true;
+    s.state = SLOT_FILLED;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_sync_filled(kvc_ring *r, uint32_t slot)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[slot];
+    if (s.state != SLOT_FILLED)
+        return KVC_ERR_STATE;
+    if (!s.filled_by_host && r->ev.synchronize(r->ev.ctx, s.filled) != 0)
+        return KVC_ERR_CUDA;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_release_host(kvc_ring *r, uint32_t slot)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[slot];
+    if (s.state != SLOT_FILLED)
+        return KVC_ERR_STATE;
+    s.state = SLOT_FREE;
     return KVC_OK;
 }
 

@@ -22,7 +22,7 @@ LIB_PATH = os.path.join(_HERE, "libkvc.so")
 
 KVC_OK, KVC_ERR_INVALID_ARG, KVC_ERR_OUT_OF_RANGE, KVC_ERR_ALIGNMENT, KVC_ERR_CONFLICT, \
     KVC_ERR_NOMEM, KVC_ERR_CUDA, KVC_ERR_WOULD_BLOCK, KVC_ERR_TIMEOUT, KVC_ERR_STATE, \
-    KVC_ERR_TOO_LARGE = range(11)
+    KVC_ERR_TOO_LARGE, KVC_ERR_EXISTS, KVC_ERR_NOT_FOUND, KVC_ERR_IO = range(14)
 KVC_VARIANT_AUTO, KVC_VARIANT_VEC, KVC_VARIANT_BULK = 0, 1, 2
 KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR = 0, 1, 2
 KVC_RING_DEVICE, KVC_RING_HOST_MAPPED = 0, 1
@@ -61,6 +61,12 @@ class kvc_chunk_desc(ctypes.Structure):
     _fields_ = [("request", ctypes.c_uint32), ("chunk", ctypes.c_uint32),
                 ("first", ctypes.c_uint32), ("n_blocks", ctypes.c_uint32),
                 ("bytes", ctypes.c_uint64)]
+
+
+class kvc_pipeline_stats(ctypes.Structure):
+    _fields_ = [("bytes", ctypes.c_uint64), ("seconds", ctypes.c_double), ("chunks", ctypes.c_uint32),
+                ("published", ctypes.c_uint32), ("already_present", ctypes.c_uint32),
+                ("ring_stalls", ctypes.c_uint32)]
 
 
 # kvc_chunk_op as a numpy record so that thousands of ops can be filled without a Python loop
@@ -129,6 +135,20 @@ def lib() -> ctypes.CDLL:
         "kvc_staging_ring_slot_bytes": (u64, [vp]),
         "kvc_staging_ring_num_slots": (u32, [vp]),
         "kvc_staging_ring_set_event_provider": (ci, [P(kvc_event_provider)]),
+        "kvc_staging_ring_commit_host": (ci, [vp, u32]),
+        "kvc_staging_ring_sync_filled": (ci, [vp, u32]),
+        "kvc_staging_ring_release_host": (ci, [vp, u32]),
+        "kvc_pipeline_store": (ci, [vp, vp, vp, vp, u32, vp, u32, u32, ci, vp, P(kvc_pipeline_stats)]),
+        "kvc_pipeline_load": (ci, [vp, vp, vp, vp, u32, vp, u32, u32, ci, vp, P(kvc_pipeline_stats)]),
+        "kvc_store_open": (ci, [ctypes.c_char_p, ctypes.c_char_p, ci, P(vp)]),
+        "kvc_store_close": (ci, [vp]),
+        "kvc_store_path": (ci, [vp, u64, ctypes.c_char_p, u32]),
+        "kvc_store_lookup": (ci, [vp, u64, P(u64)]),
+        "kvc_store_publish": (ci, [vp, u64, vp, u64]),
+        "kvc_store_read": (ci, [vp, u64, vp, u64]),
+        "kvc_store_direct_io_refused": (ci, [vp]),
+        "kvc_chain_hash": (u64, [u64, vp, u32]),
+        "kvc_fnv1a64": (u64, [vp, u64]),
     }
     for name, (res, args) in sig.items():
         f = getattr(L, name)
@@ -500,3 +520,115 @@ def kvc_staging_ring_set_event_provider(provider: Optional[dict]) -> None:
     _check(lib().kvc_staging_ring_set_event_provider(ctypes.byref(p)),
            "kvc_staging_ring_set_event_provider")
     _provider_keep = (p, fns)
+
+
+# ------------------------------------------------------------------ chunk files
+class StoreHandle:
+    """Owns a ``kvc_store*``."""
+
+    def __init__(self, handle: int):
+        self.handle = handle
+
+    def __del__(self):
+        try:
+            if self.handle and _lib is not None:
+                _lib.kvc_store_close(self.handle)
+        except Exception:
+            pass
+        self.handle = 0
+
+
+def kvc_store_open(root: str, model_tag: str, direct_io: bool = True) -> StoreHandle:
+    out = ctypes.c_void_p()
+    _check(lib().kvc_store_open(root.encode(), model_tag.encode(), int(direct_io), ctypes.byref(out)),
+           "kvc_store_open")
+    return StoreHandle(out.value)
+
+
+def kvc_store_close(store: StoreHandle) -> None:
+    h, store.handle = store.handle, 0
+    if h:
+        _check(lib().kvc_store_close(h), "kvc_store_close")
+
+
+def kvc_store_path(store, hash64: int) -> str:
+    buf = ctypes.create_string_buffer(4096)
+    _check(lib().kvc_store_path(store.handle, hash64, buf, 4096), "kvc_store_path")
+    return buf.value.decode()
+
+
+def kvc_store_lookup(store, hash64: int) -> Optional[int]:
+    """Size of the entry in bytes, or None if it is not published."""
+    n = ctypes.c_uint64()
+    st = lib().kvc_store_lookup(store.handle, hash64, ctypes.byref(n))
+    if st == KVC_ERR_NOT_FOUND:
+        return None
+    _check(st, "kvc_store_lookup")
+    return n.value
+
+
+def kvc_store_publish(store, hash64: int, host_buf, nbytes: Optional[int] = None) -> bool:
+    """True if this call published the entry, False if another writer already had."""
+    nb = _nbytes(host_buf) if nbytes is None else nbytes
+    st = lib().kvc_store_publish(store.handle, hash64, _ptr(host_buf), nb)
+    if st == KVC_ERR_EXISTS:
+        return False
+    _check(st, "kvc_store_publish")
+    return True
+
+
+def kvc_store_read(store, hash64: int, host_buf, nbytes: Optional[int] = None) -> None:
+    nb = _nbytes(host_buf) if nbytes is None else nbytes
+    _check(lib().kvc_store_read(store.handle, hash64, _ptr(host_buf), nb), "kvc_store_read")
+
+
+def kvc_store_direct_io_refused(store) -> int:
+    return lib().kvc_store_direct_io_refused(store.handle)
+
+
+def kvc_chain_hash(prev: int, tokens) -> int:
+    t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+    return lib().kvc_chain_hash(prev, t.ctypes.data, t.size)
+
+
+def kvc_fnv1a64(data: bytes) -> int:
+    return lib().kvc_fnv1a64(ctypes.c_char_p(data), len(data))
+
+
+def kvc_staging_ring_commit_host(ring, slot: int) -> None:
+    _check(lib().kvc_staging_ring_commit_host(ring.handle, slot), "kvc_staging_ring_commit_host")
+
+
+def kvc_staging_ring_sync_filled(ring, slot: int) -> None:
+    _check(lib().kvc_staging_ring_sync_filled(ring.handle, slot), "kvc_staging_ring_sync_filled")
+
+
+def kvc_staging_ring_release_host(ring, slot: int) -> None:
+    _check(lib().kvc_staging_ring_release_host(ring.handle, slot), "kvc_staging_ring_release_host")
+
+
+def _pipeline(fn_name, layout, ring, store, ids, hashes, io_threads, use_copy_engine, stream):
+    keep, p, n, dev = _ids(ids)
+    if dev:
+        raise TypeError("the pipelines take host-resident ids")
+    hs = np.ascontiguousarray(np.asarray(hashes, dtype=np.uint64))
+    stats = kvc_pipeline_stats()
+    st = getattr(lib(), fn_name)(layout.handle, ring.handle, store.handle, p, n, hs.ctypes.data,
+                                 hs.size, io_threads, int(use_copy_engine), _stream(stream),
+                                 ctypes.byref(stats))
+    _check(st, fn_name)
+    return {k: getattr(stats, k) for k, _ in kvc_pipeline_stats._fields_}
+
+
+def kvc_pipeline_store(layout, ring, store, ids, hashes, io_threads: int = 0,
+                       use_copy_engine: bool = False, stream=None) -> dict:
+    """Offload a request to chunk files through a mapped-host ring; returns the stats as a dict."""
+    return _pipeline("kvc_pipeline_store", layout, ring, store, ids, hashes, io_threads,
+                     use_copy_engine, stream)
+
+
+def kvc_pipeline_load(layout, ring, store, ids, hashes, io_threads: int = 0,
+                      use_copy_engine: bool = False, stream=None) -> dict:
+    """Load the present prefix of a request's chunks from files; synchronise the stream afterwards."""
+    return _pipeline("kvc_pipeline_load", layout, ring, store, ids, hashes, io_threads,
+                     use_copy_engine, stream)

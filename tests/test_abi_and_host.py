@@ -300,3 +300,33 @@ def test_ring_create_validation(fake_events):
         with pytest.raises(kvc.KvcError) as e:
             kvc.kvc_staging_ring_create(*args)
         assert e.value.status == want, args
+
+
+def test_ring_host_side_transitions(fake_events):
+    """Slots filled or drained by the host (file reads and writes) need no event."""
+    n, sb = 2, 4096
+    mem = np.zeros(n * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    ring = kvc.kvc_staging_ring_create(sb, n, kvc.KVC_RING_DEVICE, base, n * sb)
+    for fn in (kvc.kvc_staging_ring_commit_host, kvc.kvc_staging_ring_sync_filled,
+               kvc.kvc_staging_ring_release_host):
+        with pytest.raises(kvc.KvcError) as e:       # nothing acquired yet
+            fn(ring, 0)
+        assert e.value.status == kvc.KVC_ERR_STATE
+    slot, _, _ = kvc.kvc_staging_ring_acquire(ring)
+    kvc.kvc_staging_ring_commit_host(ring, slot)      # host filled it: no event recorded
+    assert fake_events.recorded == []
+    kvc.kvc_staging_ring_sync_filled(ring, slot)      # returns at once
+    kvc.kvc_staging_ring_wait_filled(ring, slot, 5)   # adds no dependency
+    kvc.kvc_staging_ring_release_host(ring, slot)     # host consumer done: free immediately
+    assert kvc.kvc_staging_ring_stats(ring)[0] == 0
+    # GPU producer, host consumer: sync_filled waits on the recorded event
+    slot2, _, _ = kvc.kvc_staging_ring_acquire(ring)
+    kvc.kvc_staging_ring_commit(ring, slot2, 9)
+    ev = fake_events.recorded[-1][0]
+    assert fake_events.done[ev] is False
+    kvc.kvc_staging_ring_sync_filled(ring, slot2)     # the fake "synchronize" completes it
+    assert fake_events.done[ev] is True
+    kvc.kvc_staging_ring_release_host(ring, slot2)
+    assert [kvc.kvc_staging_ring_acquire(ring)[0] for _ in range(2)] == [0, 1]
+    kvc.kvc_staging_ring_destroy(ring)
