@@ -367,6 +367,48 @@ kvc_status kvc_pipeline_load(kvc_layout *layout, kvc_ring *ring, kvc_store *stor
                              uint32_t io_threads, int use_copy_engine, void *stream,
                              kvc_pipeline_stats *stats);
 
+/* ------------------------------------------------------------------ slot policy (Sec. 6.5) */
+
+/* Who gets a staging slot when demand loads, stores and speculative preloads share one pool.
+ * Host bookkeeping only (no CUDA call); slot indices name regions of the caller's staging memory.
+ * Rules (Sec. 6.4, 6.5): `foreground_reserve` slots (the I/O depth) are kept for demand loads and
+ * stores -- a preload gets a slot only while more than that many are free and fewer than
+ * `max_speculative` preloads are in flight (0 = no limit); requests for a key (chunk hash) that
+ * already holds a slot join it (reference count) instead of reading again, and a demand request
+ * joining a preload claims it; with no free slot, foreground work takes over the least recently
+ * used retained slot, else a staged preload nobody claimed; an unclaimed preload in flight can be
+ * cancelled; with retain_completed != 0 released staged slots stay as a cache until taken over.
+ * Not thread-safe. */
+typedef struct kvc_slot_pool kvc_slot_pool;
+typedef enum { KVC_CLASS_DEMAND_LOAD = 0, KVC_CLASS_STORE = 1, KVC_CLASS_PRELOAD = 2 } kvc_slot_class;
+typedef struct {
+    uint32_t n_free, n_in_flight, n_staged, n_retained; /* slots by state, now */
+    uint64_t acquires;            /* slots handed out for a new operation */
+    uint64_t joins;               /* requests that joined a slot already holding their key */
+    uint64_t claims;              /* preloads taken over by a demand request for the same key */
+    uint64_t reclaims;            /* retained or unclaimed staged slots taken over by foreground work */
+    uint64_t cancels;             /* preloads cancelled in flight */
+    uint64_t preload_refusals;    /* preloads refused by the reserve or the in-flight limit */
+    uint64_t foreground_refusals; /* foreground requests that found nothing to take */
+} kvc_slot_pool_counters;
+kvc_status kvc_slot_pool_create(uint32_t n_slots, uint32_t foreground_reserve, uint32_t max_speculative,
+                                int retain_completed, kvc_slot_pool **out);
+kvc_status kvc_slot_pool_destroy(kvc_slot_pool *pool);
+/* A slot for `key`.  *joined = 1: the key already has a slot (in flight, staged or retained); the
+ * caller shares it and must not start another read.  *joined = 0: a slot was taken for a new
+ * operation (state "in flight").  WOULD_BLOCK: nothing available for this class right now. */
+kvc_status kvc_slot_pool_acquire(kvc_slot_pool *pool, kvc_slot_class cls, uint64_t key, uint32_t *slot,
+                                 int *joined);
+/* The slot's I/O has completed: the chunk is staged.  STATE unless in flight. */
+kvc_status kvc_slot_pool_mark_staged(kvc_slot_pool *pool, uint32_t slot);
+/* Drops one reference.  At zero the slot is freed -- or, if staged, kept: as a cache entry when
+ * retention is on, or as a finished preload waiting to be claimed. */
+kvc_status kvc_slot_pool_release(kvc_slot_pool *pool, uint32_t slot);
+/* Gives up an unclaimed preload that is still in flight (its read is abandoned and requeued by the
+ * caller).  STATE for anything else. */
+kvc_status kvc_slot_pool_cancel(kvc_slot_pool *pool, uint32_t slot);
+kvc_status kvc_slot_pool_get_counters(const kvc_slot_pool *pool, kvc_slot_pool_counters *out);
+
 /* Event provider used by a ring.  The default one wraps CUDA events.  Tests replace it to
  * drive the slot state machine on a machine without a GPU (events that complete on command);
  * it must be installed before the ring is created and applies to rings created afterwards.

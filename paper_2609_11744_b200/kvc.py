@@ -69,6 +69,15 @@ class kvc_pipeline_stats(ctypes.Structure):
                 ("ring_stalls", ctypes.c_uint32)]
 
 
+class kvc_slot_pool_counters(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_uint32) for k in ("n_free", "n_in_flight", "n_staged", "n_retained")] + \
+               [(k, ctypes.c_uint64) for k in ("acquires", "joins", "claims", "reclaims", "cancels",
+                                               "preload_refusals", "foreground_refusals")]
+
+
+KVC_CLASS_DEMAND_LOAD, KVC_CLASS_STORE, KVC_CLASS_PRELOAD = 0, 1, 2
+
+
 # kvc_chunk_op as a numpy record so that thousands of ops can be filled without a Python loop
 CHUNK_OP_DTYPE = np.dtype([("slot", np.uint64), ("ids", np.uint64), ("n_blocks", np.uint32),
                            ("reserved", np.uint32)])
@@ -140,6 +149,13 @@ def lib() -> ctypes.CDLL:
         "kvc_staging_ring_release_host": (ci, [vp, u32]),
         "kvc_pipeline_store": (ci, [vp, vp, vp, vp, u32, vp, u32, u32, ci, vp, P(kvc_pipeline_stats)]),
         "kvc_pipeline_load": (ci, [vp, vp, vp, vp, u32, vp, u32, u32, ci, vp, P(kvc_pipeline_stats)]),
+        "kvc_slot_pool_create": (ci, [u32, u32, u32, ci, P(vp)]),
+        "kvc_slot_pool_destroy": (ci, [vp]),
+        "kvc_slot_pool_acquire": (ci, [vp, ci, u64, P(u32), P(ci)]),
+        "kvc_slot_pool_mark_staged": (ci, [vp, u32]),
+        "kvc_slot_pool_release": (ci, [vp, u32]),
+        "kvc_slot_pool_cancel": (ci, [vp, u32]),
+        "kvc_slot_pool_get_counters": (ci, [vp, P(kvc_slot_pool_counters)]),
         "kvc_store_open": (ci, [ctypes.c_char_p, ctypes.c_char_p, ci, P(vp)]),
         "kvc_store_close": (ci, [vp]),
         "kvc_store_path": (ci, [vp, u64, ctypes.c_char_p, u32]),
@@ -632,3 +648,61 @@ def kvc_pipeline_load(layout, ring, store, ids, hashes, io_threads: int = 0,
     """Load the present prefix of a request's chunks from files; synchronise the stream afterwards."""
     return _pipeline("kvc_pipeline_load", layout, ring, store, ids, hashes, io_threads,
                      use_copy_engine, stream)
+
+
+# ------------------------------------------------------------------ slot policy
+class SlotPoolHandle:
+    """Owns a ``kvc_slot_pool*``."""
+
+    def __init__(self, handle: int):
+        self.handle = handle
+
+    def __del__(self):
+        try:
+            if self.handle and _lib is not None:
+                _lib.kvc_slot_pool_destroy(self.handle)
+        except Exception:
+            pass
+        self.handle = 0
+
+
+def kvc_slot_pool_create(n_slots: int, foreground_reserve: int, max_speculative: int = 1,
+                         retain_completed: bool = False) -> SlotPoolHandle:
+    out = ctypes.c_void_p()
+    _check(lib().kvc_slot_pool_create(n_slots, foreground_reserve, max_speculative,
+                                      int(retain_completed), ctypes.byref(out)), "kvc_slot_pool_create")
+    return SlotPoolHandle(out.value)
+
+
+def kvc_slot_pool_destroy(pool: SlotPoolHandle) -> None:
+    h, pool.handle = pool.handle, 0
+    if h:
+        _check(lib().kvc_slot_pool_destroy(h), "kvc_slot_pool_destroy")
+
+
+def kvc_slot_pool_acquire(pool, cls: int, key: int) -> Optional[Tuple[int, bool]]:
+    """(slot, joined), or None when nothing is available for this class right now."""
+    slot, joined = ctypes.c_uint32(), ctypes.c_int()
+    st = lib().kvc_slot_pool_acquire(pool.handle, cls, key, ctypes.byref(slot), ctypes.byref(joined))
+    if st == KVC_ERR_WOULD_BLOCK:
+        return None
+    _check(st, "kvc_slot_pool_acquire")
+    return slot.value, bool(joined.value)
+
+
+def kvc_slot_pool_mark_staged(pool, slot: int) -> None:
+    _check(lib().kvc_slot_pool_mark_staged(pool.handle, slot), "kvc_slot_pool_mark_staged")
+
+
+def kvc_slot_pool_release(pool, slot: int) -> None:
+    _check(lib().kvc_slot_pool_release(pool.handle, slot), "kvc_slot_pool_release")
+
+
+def kvc_slot_pool_cancel(pool, slot: int) -> None:
+    _check(lib().kvc_slot_pool_cancel(pool.handle, slot), "kvc_slot_pool_cancel")
+
+
+def kvc_slot_pool_get_counters(pool) -> dict:
+    c = kvc_slot_pool_counters()
+    _check(lib().kvc_slot_pool_get_counters(pool.handle, ctypes.byref(c)), "kvc_slot_pool_get_counters")
+    return {k: getattr(c, k) for k, _ in kvc_slot_pool_counters._fields_}
