@@ -97,7 +97,8 @@ typedef struct {
 /* Validates and copies the descriptor.  Makes no CUDA call: the small device-side
  * state a launch needs (plane-pointer table, status words, id-table arenas) is
  * allocated by the first pack/unpack call on the handle, which therefore must not
- * happen during stream capture.
+ * happen during stream capture.  From then on the handle belongs to the device that was
+ * current at that call (INVALID_ARG if another device is current later); use one handle per GPU.
  * Errors: INVALID_ARG (NULL, zero dimension, chunk_tokens not a multiple of
  * block_size, elem_bytes not 1/2/4, block_stride < slab_bytes), ALIGNMENT (slab
  * bytes, a base pointer or a stride not a multiple of 16), NOMEM. */

@@ -408,14 +408,20 @@ cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t 
                        cudaStream_t stream)
 {
     if (variant == KVC_VARIANT_BULK) {
-        static int configured_smem[2][2] = {{0, 0}, {0, 0}};
-        if ((int)smem > configured_smem[DIR][TABLE]) {
-            cudaError_t e = cudaFuncSetAttribute(kvc_bulk_kernel<DIR, TABLE>,
-                                                 cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)smem);
+        // the opt-in shared-memory size is a per-device attribute of the kernel
+        static int configured_smem[64][2][2];
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess)
+            return e;
+        if (dev < 0 || dev >= 64)
+            return cudaErrorInvalidDevice;
+        if ((int)smem > configured_smem[dev][DIR][TABLE]) {
+            e = cudaFuncSetAttribute(kvc_bulk_kernel<DIR, TABLE>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e != cudaSuccess)
                 return e;
-            configured_smem[DIR][TABLE] = (int)smem;
+            configured_smem[dev][DIR][TABLE] = (int)smem;
         }
         return launch_cfg(kvc_bulk_kernel<DIR, TABLE>, a, grid, KVC_BULK_THREADS, smem, stream);
     }

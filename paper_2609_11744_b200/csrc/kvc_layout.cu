@@ -16,8 +16,13 @@ inline bool mult16(uint64_t v) { return (v & 15u) == 0; }
 
 kvc_status ensure_device(kvc_layout *lay)
 {
-    if (lay->dev_ready)
-        return KVC_OK;
+    if (lay->dev_ready) {
+        // a handle belongs to the device that was current at its first launch
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess)
+            return KVC_ERR_CUDA;
+        return dev == lay->device ? KVC_OK : KVC_ERR_INVALID_ARG;
+    }
     if (cudaGetDevice(&lay->device) != cudaSuccess)
         return KVC_ERR_CUDA;
     if (kvc_kernel_limits(&lay->sm_count, &lay->vec_blocks_per_sm, &lay->max_smem_optin) !=
