@@ -305,7 +305,7 @@ def run_ours(args, rank, world, local_rank):
     if traffic is None and (args.workload, NB, n, args.chunk_tokens, args.variant) == \
             ("8b_80k", 20000, 5000, 256, 0):
         # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this exact workload, from a
-        # one-pass ncu capture (profiles/kvc_bulk_kernel_8b_80k_dram_traffic.md): mean of the
+        # one-pass ncu capture (its summary is kept under profiles/): mean of the
         # pack launch (20,936,505,000) and the unpack launch (20,933,015,000)
         traffic = 20_934_760_000.0
     launch_ms = statistics.mean(pack_ms + unpack_ms)

@@ -582,3 +582,37 @@ def test_pool_with_kv_inside_the_block_axis(variant, chunk_order):
         unpacker(g, orc.dense_planes(g, want), ch, dst[f:f + nb])
     want_inter = np.ascontiguousarray(want.reshape(g.L, g.P, g.NB, S).transpose(0, 2, 1, 3)).reshape(-1)
     assert np.array_equal(pool_t.cpu().numpy(), want_inter)
+
+
+# ------------------------------------------------------------------ many launches in flight, two streams
+def test_many_batched_launches_on_two_streams_share_one_handle():
+    """More batched launches than the handle has id-table buffers, issued back to back on two
+    streams without synchronising: every launch must read its own table.  Some ops are empty."""
+    g = orc.Dims(2, 2, 64, 16, 4, 64, 2)
+    pool = wl.random_bits(800, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 64)
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    n_launch, per = 24, 10
+    staging = torch.zeros(n_launch * per * g.bytes_per_block, dtype=torch.uint8, device=DEV)
+    tables, keep = [], []
+    for k in range(n_launch):
+        ids = wl.block_ids(900 + k, g.NB, per)
+        tables.append(ids)
+        base = staging.data_ptr() + k * per * g.bytes_per_block
+        sizes = [kvc.kvc_layout_chunk_bytes(lay, nb) for _, nb in orc.chunk_ranges(per, 4)]
+        offs = np.concatenate([[0], np.cumsum(sizes)[:-1]])
+        slot_addrs = [base + int(o) for o in offs] + [base]            # last op is empty
+        id_addrs = [ids.ctypes.data + 4 * f for f, _ in orc.chunk_ranges(per, 4)] + [ids.ctypes.data]
+        nbs = [nb for _, nb in orc.chunk_ranges(per, 4)] + [0]
+        ops = kvc.make_chunk_ops(slot_addrs, id_addrs, nbs)
+        keep.append(ops)
+        kvc.kvc_pack_batch(lay, ops, 0, stream=streams[k % 2])
+    torch.cuda.synchronize()
+    host = staging.cpu().numpy()
+    for k in range(n_launch):
+        want = np.concatenate(orc.pack_request(g, pool, tables[k], 64))
+        got = host[k * per * g.bytes_per_block:(k + 1) * per * g.bytes_per_block]
+        assert np.array_equal(got, want), "launch %d" % k
+    assert kvc.kvc_layout_launch_count(lay) == n_launch
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
