@@ -296,6 +296,18 @@ kvc_status kvc_staging_ring_release_host(kvc_ring *ring, uint32_t slot);
  * next slot still busy.  Any pointer may be NULL. */
 kvc_status kvc_staging_ring_stats(const kvc_ring *ring, uint32_t *in_flight, uint64_t *acquires,
                                   uint64_t *stalls);
+/* Slot transitions with host timestamps, for timelines of a transfer (the paper traces its
+ * pipeline the same way, Sec. 4.1).  `buf` is a HOST array of `cap` entries owned by the caller and
+ * must outlive the ring or be detached with buf = NULL; entries past `cap` are dropped but still
+ * counted.  A stall is logged once per acquire call that had to wait or was refused. */
+typedef enum { KVC_TRACE_ACQUIRE = 0, KVC_TRACE_COMMIT = 1, KVC_TRACE_RELEASE = 2, KVC_TRACE_STALL = 3 } kvc_ring_trace_kind;
+typedef struct {
+    uint64_t t_ns; /* steady-clock nanoseconds */
+    uint32_t slot;
+    uint32_t what; /* kvc_ring_trace_kind */
+} kvc_ring_trace_entry;
+kvc_status kvc_staging_ring_set_trace(kvc_ring *ring, kvc_ring_trace_entry *buf, uint32_t cap);
+uint32_t kvc_staging_ring_trace_count(const kvc_ring *ring);
 uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *ring);
 uint32_t kvc_staging_ring_num_slots(const kvc_ring *ring);
 

@@ -74,9 +74,26 @@ struct kvc_ring {
     std::vector<Slot> slots;
     uint32_t head;             // next slot to hand out
     uint64_t acquires, stalls;
+    kvc_ring_trace_entry *trace;  // caller's buffer, or nullptr
+    uint32_t trace_cap, trace_n;
 };
 
 namespace {
+
+void trace(kvc_ring *r, uint32_t slot, kvc_ring_trace_kind what)
+{
+    if (!r->trace)
+        return;
+    if (r->trace_n < r->trace_cap) {
+        kvc_ring_trace_entry &e = r->trace[r->trace_n];
+        e.t_ns = (uint64_t)std::chrono::duration_cast<std::chrono::nanoseconds>(
+                     std::chrono::steady_clock::now().time_since_epoch())
+                     .count();
+        e.slot = slot;
+        e.what = (uint32_t)what;
+    }
+    ++r->trace_n;  // keeps counting past the capacity so that the caller can see what was dropped
+}
 
 // FREE, or DRAINING whose event has completed.  Returns 0 free, 1 busy, <0 error.
 int slot_is_free(kvc_ring *r, Slot &s)
@@ -140,6 +157,8 @@ kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ri
     r->owns_mem = false;
     r->head = 0;
     r->acquires = r->stalls = 0;
+    r->trace = nullptr;
+    r->trace_cap = r->trace_n = 0;
     try {
         r->slots.resize(n_slots);
     } catch (const std::bad_alloc &) {
@@ -232,6 +251,7 @@ kvc_status kvc_staging_ring_acquire(kvc_ring *r, int64_t timeout_us, uint32_t *s
     Slot &s = r->slots[r->head];
     const auto deadline =
         std::chrono::steady_clock::now() + std::chrono::microseconds(timeout_us);
+    bool stall_logged = false;
     for (;;) {
         int q = slot_is_free(r, s);
         if (q < 0)
@@ -239,6 +259,10 @@ kvc_status kvc_staging_ring_acquire(kvc_ring *r, int64_t timeout_us, uint32_t *s
         if (q == 0)
             break;
         ++r->stalls;
+        if (!stall_logged) {
+            trace(r, r->head, KVC_TRACE_STALL);
+            stall_logged = true;
+        }
         if (timeout_us == 0)
             return KVC_ERR_WOULD_BLOCK;
         if (std::chrono::steady_clock::now() >= deadline)
@@ -255,6 +279,7 @@ kvc_status kvc_staging_ring_acquire(kvc_ring *r, int64_t timeout_us, uint32_t *s
         *dev_ptr = r->dev_base + (uint64_t)r->head * r->slot_bytes;
     if (host_ptr)
         *host_ptr = r->host_base ? r->host_base + (uint64_t)r->head * r->slot_bytes : nullptr;
+    trace(r, r->head, KVC_TRACE_ACQUIRE);
     r->head = (r->head + 1) % r->n_slots;
     ++r->acquires;
     return KVC_OK;
@@ -271,6 +296,7 @@ kvc_status kvc_staging_ring_commit(kvc_ring *r, uint32_t slot, void *producer_st
         return KVC_ERR_CUDA;
     s.filled_by_host = false;
     s.state = SLOT_FILLED;
+    trace(r, slot, KVC_TRACE_COMMIT);
     return KVC_OK;
 }
 
@@ -296,6 +322,7 @@ kvc_status kvc_staging_ring_release(kvc_ring *r, uint32_t slot, void *consumer_s
     if (r->ev.record(r->ev.ctx, s.drained, consumer_stream) != 0)
         return KVC_ERR_CUDA;
     s.state = SLOT_DRAINING;
+    trace(r, slot, KVC_TRACE_RELEASE);
     return KVC_OK;
 }
 
@@ -308,6 +335,7 @@ kvc_status kvc_staging_ring_commit_host(kvc_ring *r, uint32_t slot)
         return KVC_ERR_STATE;
     s.filled_by_host = true;
     s.state = SLOT_FILLED;
+    trace(r, slot, KVC_TRACE_COMMIT);
     return KVC_OK;
 }
 
@@ -331,6 +359,7 @@ kvc_status kvc_staging_ring_release_host(kvc_ring *r, uint32_t slot)
     if (s.state != SLOT_FILLED)
         return KVC_ERR_STATE;
     s.state = SLOT_FREE;
+    trace(r, slot, KVC_TRACE_RELEASE);
     return KVC_OK;
 }
 
@@ -351,6 +380,18 @@ kvc_status kvc_staging_ring_stats(const kvc_ring *r, uint32_t *in_flight, uint64
         *stalls = r->stalls;
     return KVC_OK;
 }
+
+kvc_status kvc_staging_ring_set_trace(kvc_ring *r, kvc_ring_trace_entry *buf, uint32_t cap)
+{
+    if (!r || (buf && cap == 0))
+        return KVC_ERR_INVALID_ARG;
+    r->trace = buf;
+    r->trace_cap = buf ? cap : 0;
+    r->trace_n = 0;
+    return KVC_OK;
+}
+
+uint32_t kvc_staging_ring_trace_count(const kvc_ring *r) { return r ? r->trace_n : 0; }
 
 uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *r) { return r ? r->slot_bytes : 0; }
 uint32_t kvc_staging_ring_num_slots(const kvc_ring *r) { return r ? r->n_slots : 0; }

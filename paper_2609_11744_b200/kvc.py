@@ -144,6 +144,8 @@ def lib() -> ctypes.CDLL:
         "kvc_staging_ring_slot_bytes": (u64, [vp]),
         "kvc_staging_ring_num_slots": (u32, [vp]),
         "kvc_staging_ring_set_event_provider": (ci, [P(kvc_event_provider)]),
+        "kvc_staging_ring_set_trace": (ci, [vp, vp, u32]),
+        "kvc_staging_ring_trace_count": (u32, [vp]),
         "kvc_staging_ring_commit_host": (ci, [vp, u32]),
         "kvc_staging_ring_sync_filled": (ci, [vp, u32]),
         "kvc_staging_ring_release_host": (ci, [vp, u32]),
@@ -706,3 +708,25 @@ def kvc_slot_pool_get_counters(pool) -> dict:
     c = kvc_slot_pool_counters()
     _check(lib().kvc_slot_pool_get_counters(pool.handle, ctypes.byref(c)), "kvc_slot_pool_get_counters")
     return {k: getattr(c, k) for k, _ in kvc_slot_pool_counters._fields_}
+
+
+RING_TRACE_DTYPE = np.dtype([("t_ns", np.uint64), ("slot", np.uint32), ("what", np.uint32)])
+KVC_TRACE_ACQUIRE, KVC_TRACE_COMMIT, KVC_TRACE_RELEASE, KVC_TRACE_STALL = 0, 1, 2, 3
+
+
+def kvc_staging_ring_set_trace(ring, capacity: int) -> Optional[np.ndarray]:
+    """Start logging slot transitions into a new array of RING_TRACE_DTYPE (returned; it is kept
+    alive by the ring handle), or stop logging with capacity 0."""
+    if capacity <= 0:
+        _check(lib().kvc_staging_ring_set_trace(ring.handle, None, 0), "kvc_staging_ring_set_trace")
+        ring._trace = None
+        return None
+    buf = np.zeros(capacity, dtype=RING_TRACE_DTYPE)
+    _check(lib().kvc_staging_ring_set_trace(ring.handle, buf.ctypes.data, capacity),
+           "kvc_staging_ring_set_trace")
+    ring._trace = buf
+    return buf
+
+
+def kvc_staging_ring_trace_count(ring) -> int:
+    return lib().kvc_staging_ring_trace_count(ring.handle)

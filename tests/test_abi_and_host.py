@@ -330,3 +330,26 @@ def test_ring_host_side_transitions(fake_events):
     kvc.kvc_staging_ring_release_host(ring, slot2)
     assert [kvc.kvc_staging_ring_acquire(ring)[0] for _ in range(2)] == [0, 1]
     kvc.kvc_staging_ring_destroy(ring)
+
+
+def test_ring_trace_records_transitions_in_order(fake_events):
+    n, sb = 2, 4096
+    mem = np.zeros(n * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    ring = kvc.kvc_staging_ring_create(sb, n, kvc.KVC_RING_DEVICE, base, n * sb)
+    tr = kvc.kvc_staging_ring_set_trace(ring, 6)
+    for _ in range(2):
+        slot, _, _ = kvc.kvc_staging_ring_acquire(ring)
+        kvc.kvc_staging_ring_commit(ring, slot, 1)
+        kvc.kvc_staging_ring_release(ring, slot, 2)
+    with pytest.raises(kvc.KvcError):
+        kvc.kvc_staging_ring_acquire(ring)            # both slots wait for their events: a stall
+    assert kvc.kvc_staging_ring_trace_count(ring) == 7        # one more than the buffer holds
+    A, C, R = kvc.KVC_TRACE_ACQUIRE, kvc.KVC_TRACE_COMMIT, kvc.KVC_TRACE_RELEASE
+    assert list(zip(tr["slot"].tolist(), tr["what"].tolist())) == [(0, A), (0, C), (0, R), (1, A), (1, C), (1, R)]
+    assert (np.diff(tr["t_ns"].astype(np.int64)) >= 0).all() and tr["t_ns"][0] > 0
+    kvc.kvc_staging_ring_set_trace(ring, 0)
+    fake_events.complete_all()
+    kvc.kvc_staging_ring_acquire(ring)
+    assert kvc.kvc_staging_ring_trace_count(ring) == 0
+    kvc.kvc_staging_ring_destroy(ring)
