@@ -181,6 +181,10 @@ kvc_status kvc_map_requests_shared(const kvc_layout *layout, const int32_t *cons
  * repeated id).  Device ids are range-checked in the kernel: a bad id skips its block and
  * is counted (see kvc_poll_device_status); repeated device ids in unpack are undefined.
  * n_blocks == 0 is a no-op returning KVC_OK.
+ * With device ids, or with at most 128 host ids (they travel in the kernel parameters), a call
+ * enqueues exactly one kernel and nothing else, so once the handle has made its first launch such
+ * calls can be captured into a CUDA graph.  Longer host id lists, and the batched calls, also
+ * upload an id table on a second stream and are not meant for capture.
  * Errors: INVALID_ARG, OUT_OF_RANGE, CONFLICT, ALIGNMENT, NOMEM, CUDA. */
 kvc_status kvc_pack(kvc_layout *layout, const int32_t *ids, uint32_t n_blocks, int ids_on_device,
                     void *dst_slot, uint64_t slot_bytes, void *stream);

@@ -15,6 +15,7 @@
 // Measured on B200: the vector kernels peak with three resident blocks per SM and 16 KiB tiles
 // (6.37 TB/s); four blocks per SM (the occupancy limit) put more loads in flight and lose 3 %.
 #define KVC_VEC_DEFAULT_BLOCKS_PER_SM 3u
+#define KVC_HOST_SLOT_DEFAULT_CTAS 16u
 #define KVC_BULK_THREADS 32u    // one warp drives the bulk-copy pipeline
 #define KVC_BULK_MAX_STAGES 16u
 // Measured on B200 (80k-token prefix, 32 KiB slabs): HBM throughput peaks when each SM keeps one

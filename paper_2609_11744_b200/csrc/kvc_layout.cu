@@ -72,6 +72,7 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     g.num_blocks = lay->d.num_blocks;
 
     int variant = t.variant ? (int)t.variant : KVC_VARIANT_BULK;
+    bool host_slot = false;
     if (variant == KVC_VARIANT_BULK) {
         // Bulk copies are used for device memory only; a slot in mapped host memory is
         // written with ordinary vector stores.
@@ -80,8 +81,10 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
             (void)cudaGetLastError();
             return KVC_ERR_CUDA;
         }
-        if (attr.type != cudaMemoryTypeDevice)
+        if (attr.type != cudaMemoryTypeDevice) {
             variant = KVC_VARIANT_VEC;
+            host_slot = true;
+        }
     }
     uint32_t tile = t.tile_bytes;
     if (tile == 0)
@@ -137,6 +140,10 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
                               std::min<uint64_t>(lay->vec_blocks_per_sm, KVC_VEC_DEFAULT_BLOCKS_PER_SM);
     if (t.max_ctas)
         grid = std::min<uint64_t>(grid, t.max_ctas);
+    else if (host_slot)
+        // a slot in host memory is bound by the host link: 16 blocks saturate it (measured), more
+        // would only hold SMs while they wait for the link
+        grid = std::min<uint64_t>(grid, KVC_HOST_SLOT_DEFAULT_CTAS);
     grid = std::min<uint64_t>(grid, n_items);
     plan->variant = variant;
     plan->grid = (uint32_t)grid;

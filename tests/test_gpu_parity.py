@@ -616,3 +616,40 @@ def test_many_batched_launches_on_two_streams_share_one_handle():
         assert np.array_equal(got, want), "launch %d" % k
     assert kvc.kvc_layout_launch_count(lay) == n_launch
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+# ------------------------------------------------------------------ CUDA graph capture of per-chunk calls
+def test_per_chunk_calls_replay_from_a_cuda_graph():
+    """kvc_pack / kvc_unpack with at most 128 host ids (they travel in the kernel parameters) or
+    with device ids enqueue exactly one kernel and nothing else, so a sequence of them can be
+    captured into a CUDA graph once the handle has made its first launch, and replayed."""
+    g = orc.Dims(4, 2, 64, 16, 8, 128, 2)
+    pool = wl.random_bits(950, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 64)
+    src, dst = wl.block_ids(95, g.NB, 16), wl.block_ids(96, g.NB, 16)
+    dst_dev = to_dev(dst)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 4)
+    staging = torch.zeros(4 * cb, dtype=torch.uint8, device=DEV)
+    kvc.kvc_pack(lay, src[:4], staging[:cb])          # first launch: allocates the handle's device state
+    torch.cuda.synchronize()
+    staging.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for c in range(4):
+            kvc.kvc_pack(lay, src[4 * c:4 * c + 4], staging[c * cb:(c + 1) * cb])
+        for c in range(4):
+            kvc.kvc_unpack(lay, staging[c * cb:(c + 1) * cb], dst_dev[4 * c:4 * c + 4].contiguous())
+    torch.cuda.synchronize()
+    assert bool((staging == 0).all())                 # capture enqueued nothing
+    want_chunks = orc.pack_request(g, pool, src, 64)
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, want_chunks, dst, 64)
+    for _ in range(2):
+        pool_t.copy_(to_dev(pool))
+        staging.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert np.array_equal(staging.cpu().numpy(), np.concatenate(want_chunks))
+        assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
