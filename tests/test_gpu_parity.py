@@ -186,6 +186,8 @@ def test_single_call_with_more_ids_than_fit_in_parameters():
     dst = wl.block_ids(6, g.NB, 136)
     # one chunk of 136 blocks: more ids than the kernel parameters hold (128) -> id-table path
     run_pack_unpack(g, pool, src, dst, 136 * 16, kvc.KVC_VARIANT_AUTO, 0, "chunk")
+    # the same with device-resident ids: read straight from the caller's array, any length
+    run_pack_unpack(g, pool, src, dst, 136 * 16, kvc.KVC_VARIANT_AUTO, 0, "chunk_dev")
 
 
 # ------------------------------------------------------------------ odd geometries
