@@ -655,3 +655,37 @@ def test_per_chunk_calls_replay_from_a_cuda_graph():
         assert np.array_equal(staging.cpu().numpy(), np.concatenate(want_chunks))
         assert np.array_equal(pool_t.cpu().numpy(), want_pool)
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+# ------------------------------------------------------------------ every tuning knob keeps the bytes right
+@pytest.mark.parametrize("tuning", [
+    dict(variant=2, stages=2), dict(variant=2, stages=3, lag=1), dict(variant=2, stages=7, lag=5),
+    dict(variant=2, stages=16, tile_bytes=8192, lag=3), dict(variant=2, stages=6, lag=2, max_ctas=5),
+    dict(variant=2, ctas_per_sm=2, stages=3), dict(variant=2, ctas_per_sm=4, tile_bytes=16384),
+    dict(variant=2, l2_hint=2), dict(variant=2, pdl=1), dict(variant=1, pdl=1, tile_bytes=32768),
+    dict(variant=1, max_ctas=1), dict(variant=2, max_ctas=1, stages=2),
+])
+def test_tuning_knobs_do_not_change_results(tuning):
+    g = orc.Dims(8, 2, 96, 16, 8, 128, 2)
+    key = "tuning_pool"
+    if key not in _POOL_CACHE:
+        _POOL_CACHE[key] = wl.random_bits(1234, g.pool_bytes)
+    pool = _POOL_CACHE[key]
+    src, dst = wl.block_ids(12, g.NB, 37), wl.block_ids(13, g.NB, 37)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 256)
+    kvc.kvc_layout_set_tuning(lay, **tuning)
+    want_chunks, want_pool = _oracle_results(g, pool, src, dst, 256)
+    total = 37 * g.bytes_per_block
+    staging = torch.zeros(total, dtype=torch.uint8, device=DEV)
+    off = 0
+    for f, nb in orc.chunk_ranges(37, 16):            # per-chunk calls, back to back
+        nbytes = kvc.kvc_layout_chunk_bytes(lay, nb)
+        kvc.kvc_pack(lay, src[f:f + nb], staging[off:off + nbytes])
+        off += nbytes
+    ops, keep, _, dev = kvc.request_chunk_ops(lay, dst, staging)
+    kvc.kvc_unpack_batch(lay, ops, dev)
+    torch.cuda.synchronize()
+    assert np.array_equal(staging.cpu().numpy(), np.concatenate(want_chunks))
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
