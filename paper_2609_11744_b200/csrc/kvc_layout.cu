@@ -3,7 +3,6 @@
 #include <string.h>
 
 #include <algorithm>
-#include <chrono>
 #include <map>
 #include <new>
 #include <utility>
