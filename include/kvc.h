@@ -121,18 +121,26 @@ typedef enum {
 typedef enum {
     KVC_ORDER_AUTO = 0,
     KVC_ORDER_PLANE_MAJOR = 1, /* walk all blocks of one (layer,K|V) plane, then the next plane */
-    KVC_ORDER_BLOCK_MAJOR = 2  /* walk all planes of one block, then the next block */
+    KVC_ORDER_BLOCK_MAJOR = 2, /* walk all planes of one block, then the next block */
+    KVC_ORDER_CHUNK_MAJOR = 3  /* walk the chunks one after another, each in the order its bytes
+                                  lie in the slot: the staging side is accessed sequentially */
 } kvc_order;
 typedef struct {
     uint32_t variant;    /* kvc_variant */
     uint32_t order;      /* kvc_order */
-    uint32_t max_ctas;   /* cap on thread blocks per launch (0 = fill the GPU); a small cap
-                            leaves SMs to a concurrent compute stream */
+    uint32_t max_ctas;   /* 0 = default launch shape: many short-lived blocks of a few work items
+                            each, scheduled by the hardware.  N > 0: exactly N persistent blocks
+                            that stride over all items; a small N leaves SMs to a concurrent
+                            compute stream */
     uint32_t tile_bytes; /* bytes of one slab moved per work item (0 = default); multiple of 16 */
     uint32_t stages;     /* BULK: shared-memory stages per thread block (0 = default) */
     uint32_t ctas_per_sm; /* BULK: resident thread blocks per SM, 1..4 (0 = default) */
     uint32_t l2_hint;    /* BULK: 0 = default, 1 = no L2 priority hint, 2 = evict-first on loads and stores */
     uint32_t lag;        /* BULK: loads issued ahead of the store they feed, 1..stages-2 (0 = default) */
+    uint32_t items_per_cta; /* default launch shape: work items per block (0 = about 64 KiB for
+                            BULK, 32 KiB for VEC) */
+    uint32_t interleave; /* 0/1 = off; K > 1: the sequence of slabs is cut into K equal ranges that
+                            are walked side by side (K sequential streams open at a time) */
     uint32_t pdl;        /* 0 = default (= 2), 1 = plain launches, 2 = programmatic dependent launch:
                             a kernel's blocks may be scheduled while the previous kernel of the
                             stream drains; they wait for its completion before reading memory */

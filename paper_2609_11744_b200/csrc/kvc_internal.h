@@ -12,9 +12,6 @@
 #define KVC_PARAM_IDS 128u      // block ids that travel inside the kernel parameters
 #define KVC_VEC_THREADS 256u    // threads per block of the vector kernels
 #define KVC_VEC_UNROLL 4u       // 16-byte vectors in flight per thread
-// Measured on B200: the vector kernels peak with three resident blocks per SM and 16 KiB tiles
-// (6.37 TB/s); four blocks per SM (the occupancy limit) put more loads in flight and lose 3 %.
-#define KVC_VEC_DEFAULT_BLOCKS_PER_SM 3u
 #define KVC_HOST_SLOT_DEFAULT_CTAS 16u
 #define KVC_BULK_THREADS 32u    // one warp drives the bulk-copy pipeline
 #define KVC_BULK_MAX_STAGES 16u
@@ -22,6 +19,12 @@
 // to two 32 KiB loads in flight (about 5-9 MB over the GPU); deeper prefetch lowers it by 3-4 %.
 #define KVC_BULK_DEFAULT_STAGES 4u
 #define KVC_BULK_DEFAULT_LAG 1u
+// Streaming launch shape (measured on B200 against the persistent one in the same process, all
+// workloads): two resident blocks per SM, each with two 32 KiB stages (load, then store, no
+// prefetch) and about 64 KiB of work, in chunk-major order: 6.68-6.78 TB/s pack, 6.77-6.88 TB/s
+// unpack where the persistent grid reaches 6.54-6.60 TB/s.
+#define KVC_BULK_STREAMING_BLOCKS_PER_SM 2u
+#define KVC_BULK_STREAMING_STAGES 2u
 #define KVC_BULK_SMEM_HEADER 1024u  // mbarriers + per-stage bookkeeping ahead of the data stages
 #define KVC_WAIT_LIMIT (1u << 22)   // polls of an mbarrier before a kernel gives up
 
@@ -39,14 +42,15 @@ struct KvcGeom {
     uint32_t parts;                         // ceil(S / tile_bytes)
 };
 
-// One block of one chunk in a batched launch.
+// One block of one chunk in a batched launch.  Entries are ordered by chunk, then by block.
 struct KvcEnt {
-    uint64_t slot_addr;   // chunk base + j*S : where block j of the chunk starts in plane 0
+    uint64_t slot_addr;   // chunk base + j*ent_step : where block j of the chunk starts in plane 0
     uint64_t id_or_ptr;   // the pool block id, or the device address of it
-    uint32_t nb_c;        // blocks in this chunk
-    uint32_t id_is_ptr;
     uint64_t plane_step;  // bytes between consecutive planes of this block inside the chunk
+    uint32_t nb_c;        // blocks in this chunk; bit 31 set: id_or_ptr is an address
+    uint32_t first_ent;   // index of the chunk's first entry
 };
+#define KVC_ENT_ID_IS_PTR 0x80000000u
 static_assert(sizeof(KvcEnt) == 32, "KvcEnt is loaded as two 16-byte vectors");
 
 // Kernel parameters.
@@ -61,6 +65,8 @@ struct KvcLaunch {
     uint64_t n_items;         // n_ent * LP * parts
     uint32_t n_ent;
     uint32_t order;           // kvc_order (never AUTO here)
+    uint32_t block_major_chunks;  // chunk layout is [n][L][P].. (else [L][P][n]..)
+    uint32_t interleave;      // >1: that many ranges of the slab sequence are walked side by side
     uint32_t stages;          // bulk kernels
     uint32_t lag;             // bulk kernels: loads issued ahead of the store they feed
     uint32_t l2_evict_first;  // bulk kernels: attach an evict-first L2 policy to the copies

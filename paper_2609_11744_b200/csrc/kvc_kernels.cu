@@ -46,13 +46,44 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
     const KvcGeom &g = a.g;
     uint32_t part = w % g.parts;
     uint32_t r = w / g.parts;
+    bool beyond = false;
+    if (a.interleave > 1) {
+        // K equal ranges of the slab sequence are walked side by side: consecutive work items
+        // come from different ranges, so K sequential streams are open at any time
+        const uint32_t total = a.n_ent * g.planes_total;
+        const uint32_t per = (total + a.interleave - 1) / a.interleave;
+        r = (r % a.interleave) * per + r / a.interleave;
+        beyond = r >= total;
+        if (beyond)
+            r = 0;
+    }
     uint32_t ent, lp;
     if (a.order == KVC_ORDER_PLANE_MAJOR) {
         lp = r / a.n_ent;
         ent = r - lp * a.n_ent;
-    } else {
+    } else if (a.order == KVC_ORDER_BLOCK_MAJOR) {
         ent = r / g.planes_total;
         lp = r - ent * g.planes_total;
+    } else {
+        // chunk-major: slabs in the order they lie in staging memory, chunk after chunk.  Slab r
+        // belongs to the chunk that owns entry r / LP (a chunk of nb blocks owns nb*LP slabs
+        // starting at slab first_ent*LP); inside the chunk, q walks the chunk linearly.
+        uint32_t first = 0, nb = a.n_ent;
+        if (TABLE) {
+            const uint4 probe = __ldg(reinterpret_cast<const uint4 *>(a.table + r / g.planes_total) + 1);
+            nb = probe.z & ~KVC_ENT_ID_IS_PTR;
+            first = probe.w;
+        }
+        const uint32_t q = r - first * g.planes_total;
+        uint32_t j;
+        if (a.block_major_chunks) {
+            j = q / g.planes_total;
+            lp = q - j * g.planes_total;
+        } else {
+            lp = q / nb;
+            j = q - lp * nb;
+        }
+        ent = first + j;
     }
     uint64_t slot_j, plane_step;
     int64_t id;
@@ -61,8 +92,9 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
         uint4 lo = __ldg(e), hi = __ldg(e + 1);
         slot_j = ((uint64_t)lo.y << 32) | lo.x;
         uint64_t idp = ((uint64_t)lo.w << 32) | lo.z;
-        plane_step = ((uint64_t)hi.w << 32) | hi.z;
-        id = hi.y ? (int64_t)__ldg(reinterpret_cast<const int32_t *>(idp)) : (int64_t)(int32_t)lo.z;
+        plane_step = ((uint64_t)hi.y << 32) | hi.x;
+        id = (hi.z & KVC_ENT_ID_IS_PTR) ? (int64_t)__ldg(reinterpret_cast<const int32_t *>(idp))
+                                        : (int64_t)(int32_t)lo.z;
     } else {
         slot_j = a.slot + (uint64_t)ent * a.ent_step;
         plane_step = a.plane_step;
@@ -70,10 +102,10 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
     }
     Item it;
     uint32_t off = part * g.tile_bytes;
-    it.len = min(g.tile_bytes, g.slab_bytes - off);
+    it.len = beyond ? 0u : min(g.tile_bytes, g.slab_bytes - off);
     if (id < 0 || id >= (int64_t)g.num_blocks) {
         // never touch memory for a bad id: count the block once and skip it
-        if (count_bad && part == 0 && lp == 0)
+        if (count_bad && part == 0 && lp == 0 && !beyond)
             atomicAdd(a.status, 1u);
         it.len = 0;
         id = 0;

@@ -85,18 +85,25 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
             host_slot = true;
         }
     }
+    // Two launch shapes.  Streaming (the default): many short-lived blocks, each taking a few
+    // consecutive work items, handed out by the hardware scheduler as SMs free up -- measured
+    // 2-4 % faster than a persistent grid because it balances itself and throttles the bytes in
+    // flight.  Persistent: a fixed, small number of blocks that stride over all items, used when
+    // the caller caps the blocks (to leave SMs to a compute stream) or the slot is host memory.
+    const bool persistent = t.max_ctas != 0 || host_slot;
     uint32_t tile = t.tile_bytes;
     if (tile == 0)
-        tile = variant == KVC_VARIANT_BULK ? 32768u : 16384u;
+        tile = (variant == KVC_VARIANT_BULK || !persistent) ? 32768u : 16384u;
     tile = (uint32_t)std::min<uint64_t>(tile, lay->slab_bytes);
     uint32_t stages = 0, lag = 0, smem = 0;
     if (variant == KVC_VARIANT_BULK) {
-        const uint32_t per_sm = t.ctas_per_sm ? t.ctas_per_sm : 1u;
+        const uint32_t per_sm = t.ctas_per_sm ? t.ctas_per_sm
+                                              : (persistent ? 1u : KVC_BULK_STREAMING_BLOCKS_PER_SM);
         // every resident block also costs 1 KiB of system-reserved shared memory
         const uint32_t room = ((uint32_t)lay->max_smem_optin + 1024u) / per_sm - 1024u - KVC_BULK_SMEM_HEADER;
         if (tile > room / 2)
             tile = (room / 2) & ~15u;
-        stages = t.stages ? t.stages : KVC_BULK_DEFAULT_STAGES;
+        stages = t.stages ? t.stages : (persistent ? KVC_BULK_DEFAULT_STAGES : KVC_BULK_STREAMING_STAGES);
         stages = std::min<uint32_t>(std::min<uint32_t>(stages, room / tile), KVC_BULK_MAX_STAGES);
         if (stages < 2)
             return KVC_ERR_INVALID_ARG;
@@ -122,28 +129,39 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     }
     g.tile_bytes = tile;
     g.parts = (uint32_t)((lay->slab_bytes + tile - 1) / tile);
-    const uint64_t n_items = n_ent * lay->planes_total * g.parts;
+    uint64_t n_slabs = n_ent * lay->planes_total;
+    if (t.interleave > 1)  // rounded up so that the K ranges are equally long; the excess is skipped
+        n_slabs = (n_slabs + t.interleave - 1) / t.interleave * t.interleave;
+    const uint64_t n_items = n_slabs * g.parts;
     if (n_items == 0 || n_items > 0xFFFFFFFFull)
         return KVC_ERR_INVALID_ARG;
     a->n_items = n_items;
     a->n_ent = (uint32_t)n_ent;
-    a->order = t.order ? t.order : KVC_ORDER_PLANE_MAJOR;
+    a->order = t.order ? t.order : KVC_ORDER_CHUNK_MAJOR;
+    a->block_major_chunks = lay->d.chunk_order == KVC_CHUNK_BLOCK_MAJOR;
+    a->interleave = t.interleave;
     a->stages = stages;
     a->lag = lag;
     a->l2_evict_first = t.l2_hint == 2;
     a->pdl = t.pdl != 1;  // on unless switched off
     a->status = lay->d_status;
-    uint64_t grid = variant == KVC_VARIANT_BULK
-                        ? (uint64_t)lay->sm_count * (t.ctas_per_sm ? t.ctas_per_sm : 1u)
-                        : (uint64_t)lay->sm_count *
-                              std::min<uint64_t>(lay->vec_blocks_per_sm, KVC_VEC_DEFAULT_BLOCKS_PER_SM);
-    if (t.max_ctas)
-        grid = std::min<uint64_t>(grid, t.max_ctas);
-    else if (host_slot)
+    uint64_t grid;
+    if (t.max_ctas) {
+        grid = t.max_ctas;
+    } else if (host_slot) {
         // a slot in host memory is bound by the host link: 16 blocks saturate it (measured), more
         // would only hold SMs while they wait for the link
-        grid = std::min<uint64_t>(grid, KVC_HOST_SLOT_DEFAULT_CTAS);
-    grid = std::min<uint64_t>(grid, n_items);
+        grid = KVC_HOST_SLOT_DEFAULT_CTAS;
+    } else {
+        // streaming: about 64 KiB (bulk) or 32 KiB (vector) of items per block
+        uint32_t per_block = t.items_per_cta;
+        if (per_block == 0) {
+            const uint32_t bytes = variant == KVC_VARIANT_BULK ? 65536u : 32768u;
+            per_block = std::max<uint32_t>(variant == KVC_VARIANT_BULK ? 2u : 1u, bytes / tile);
+        }
+        grid = (n_items + per_block - 1) / per_block;
+    }
+    grid = std::min<uint64_t>(std::min<uint64_t>(grid, n_items), 0x7FFFFFFFull);
     plan->variant = variant;
     plan->grid = (uint32_t)grid;
     plan->smem = smem;
@@ -324,19 +342,22 @@ kvc_status copy_batch(kvc_layout *lay, int dir, const kvc_chunk_op *ops, uint32_
         return s;
     uint64_t k = 0;
     for (uint32_t i = 0; i < n_ops; ++i) {
+        if (ops[i].n_blocks >= KVC_ENT_ID_IS_PTR)
+            return KVC_ERR_INVALID_ARG;
         uint64_t ent_step, plane_step;
         kvc_chunk_steps(lay, ops[i].n_blocks, &ent_step, &plane_step);
+        const uint32_t first = (uint32_t)k;
         for (uint32_t j = 0; j < ops[i].n_blocks; ++j, ++k) {
             KvcEnt &e = ar->host[k];
             e.slot_addr = (uint64_t)(uintptr_t)ops[i].slot + (uint64_t)j * ent_step;
-            e.nb_c = ops[i].n_blocks;
             e.plane_step = plane_step;
+            e.first_ent = first;
             if (ids_on_device) {
                 e.id_or_ptr = (uint64_t)(uintptr_t)(ops[i].ids + j);
-                e.id_is_ptr = 1;
+                e.nb_c = ops[i].n_blocks | KVC_ENT_ID_IS_PTR;
             } else {
                 e.id_or_ptr = (uint64_t)(uint32_t)ops[i].ids[j];
-                e.id_is_ptr = 0;
+                e.nb_c = ops[i].n_blocks;
             }
         }
     }
@@ -519,13 +540,13 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
 {
     if (!lay || !t)
         return KVC_ERR_INVALID_ARG;
-    if (t->variant > KVC_VARIANT_BULK || t->order > KVC_ORDER_BLOCK_MAJOR)
+    if (t->variant > KVC_VARIANT_BULK || t->order > KVC_ORDER_CHUNK_MAJOR)
         return KVC_ERR_INVALID_ARG;
     if (t->tile_bytes % 16)
         return KVC_ERR_INVALID_ARG;
     if (t->stages == 1 || t->stages > KVC_BULK_MAX_STAGES)
         return KVC_ERR_INVALID_ARG;
-    if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2)
+    if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2 || t->interleave > 1024 || t->items_per_cta > (1u << 20))
         return KVC_ERR_INVALID_ARG;
     lay->tuning = *t;
     return KVC_OK;

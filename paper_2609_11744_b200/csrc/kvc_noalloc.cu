@@ -125,13 +125,14 @@ extern "C" kvc_status kvc_pack_batch_static(kvc_layout *lay, const kvc_chunk_op 
     for (uint32_t i = 0; i < n_ops; ++i) {
         uint64_t ent_step, plane_step;
         kvc_chunk_steps(lay, ops[i].n_blocks, &ent_step, &plane_step);
+        const uint32_t first = (uint32_t)k;
         for (uint32_t j = 0; j < ops[i].n_blocks; ++j, ++k) {
             KvcEnt &e = g_host_table[k];
             e.slot_addr = (uint64_t)(uintptr_t)ops[i].slot + (uint64_t)j * ent_step;
             e.id_or_ptr = (uint64_t)(uint32_t)ops[i].ids[j];
-            e.nb_c = ops[i].n_blocks;
-            e.id_is_ptr = 0;
             e.plane_step = plane_step;
+            e.nb_c = ops[i].n_blocks;
+            e.first_ent = first;
         }
     }
     cudaStream_t st = (cudaStream_t)stream;

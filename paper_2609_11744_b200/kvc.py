@@ -24,7 +24,7 @@ KVC_OK, KVC_ERR_INVALID_ARG, KVC_ERR_OUT_OF_RANGE, KVC_ERR_ALIGNMENT, KVC_ERR_CO
     KVC_ERR_NOMEM, KVC_ERR_CUDA, KVC_ERR_WOULD_BLOCK, KVC_ERR_TIMEOUT, KVC_ERR_STATE, \
     KVC_ERR_TOO_LARGE, KVC_ERR_EXISTS, KVC_ERR_NOT_FOUND, KVC_ERR_IO = range(14)
 KVC_VARIANT_AUTO, KVC_VARIANT_VEC, KVC_VARIANT_BULK = 0, 1, 2
-KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR = 0, 1, 2
+KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR, KVC_ORDER_CHUNK_MAJOR = 0, 1, 2, 3
 KVC_RING_DEVICE, KVC_RING_HOST_MAPPED = 0, 1
 KVC_CHUNK_LAYER_MAJOR, KVC_CHUNK_BLOCK_MAJOR = 0, 1
 KVC_MAP_FULL_CHUNKS_ONLY = 1
@@ -54,6 +54,7 @@ class kvc_tuning(ctypes.Structure):
                 ("max_ctas", ctypes.c_uint32), ("tile_bytes", ctypes.c_uint32),
                 ("stages", ctypes.c_uint32), ("ctas_per_sm", ctypes.c_uint32),
                 ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32),
+                ("items_per_cta", ctypes.c_uint32), ("interleave", ctypes.c_uint32),
                 ("pdl", ctypes.c_uint32)]
 
 
@@ -313,8 +314,10 @@ def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
 
 
 def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
-                          ctas_per_sm=0, l2_hint=0, lag=0, pdl=0) -> None:
-    t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag, pdl)
+                          ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, interleave=0,
+                          pdl=0) -> None:
+    t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag,
+                   items_per_cta, interleave, pdl)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
 
 

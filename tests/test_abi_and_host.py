@@ -156,7 +156,7 @@ def test_pack_unpack_validate_before_any_launch():
 def test_set_tuning_validation():
     lay = _layout()
     kvc.kvc_layout_set_tuning(lay, variant=kvc.KVC_VARIANT_VEC, max_ctas=8, tile_bytes=8192)
-    for bad in (dict(variant=3), dict(order=3), dict(tile_bytes=24), dict(stages=1), dict(stages=99)):
+    for bad in (dict(variant=3), dict(order=4), dict(tile_bytes=24), dict(stages=1), dict(stages=99)):
         with pytest.raises(kvc.KvcError):
             kvc.kvc_layout_set_tuning(lay, **bad)
 

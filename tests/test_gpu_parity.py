@@ -154,7 +154,8 @@ def test_tiny_separate_planes(variant, mode):
 
 # ------------------------------------------------------------------ 8B shape, several tiles + ragged tail
 @pytest.mark.parametrize("variant", VARIANTS)
-@pytest.mark.parametrize("order", [kvc.KVC_ORDER_PLANE_MAJOR, kvc.KVC_ORDER_BLOCK_MAJOR])
+@pytest.mark.parametrize("order", [kvc.KVC_ORDER_PLANE_MAJOR, kvc.KVC_ORDER_BLOCK_MAJOR,
+                                   kvc.KVC_ORDER_CHUNK_MAJOR])
 @pytest.mark.parametrize("mode,chunk_tokens", [("chunk", 256), ("batch", 256), ("batch", 16),
                                                ("batch_dev", 2048), ("chunk", 2048)])
 def test_8b_shape_reduced_pool(variant, order, mode, chunk_tokens):
@@ -487,7 +488,7 @@ def test_random_tiny_layouts():
         src = rng.permutation(NB)[:n].astype(np.int32)
         dst = rng.permutation(NB)[:n].astype(np.int32)
         variant = int(rng.choice(VARIANTS))
-        order = int(rng.choice([1, 2]))
+        order = int(rng.choice([1, 2, 3]))
         tile = int(rng.choice([0, 16, 48, 256, 4096]))
         mode = str(rng.choice(["chunk", "chunk_dev", "batch", "batch_dev"]))
         run_pack_unpack(g, pool, src, dst, bpc * B, variant, order, mode, tile)
@@ -504,7 +505,8 @@ def test_block_major_chunk_order(variant, mode):
     pool_t = to_dev(pool)
     lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 64,
                                       chunk_order=kvc.KVC_CHUNK_BLOCK_MAJOR)
-    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    kvc.kvc_layout_set_tuning(lay, variant=variant, order=kvc.KVC_ORDER_CHUNK_MAJOR if variant == 2
+                              else kvc.KVC_ORDER_PLANE_MAJOR)
     src, dst = wl.block_ids(51, g.NB, 14), wl.block_ids(52, g.NB, 14)
     total = 14 * g.bytes_per_block
     staging = torch.full((total + 4096,), 0x66, dtype=torch.uint8, device=DEV)
