@@ -306,8 +306,8 @@ def run_ours(args, rank, world, local_rank):
             ("8b_80k", 20000, 5000, 256, 0):
         # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this exact workload, from a
         # one-pass ncu capture (its summary is kept under profiles/): mean of the
-        # pack launch (20,936,505,000) and the unpack launch (20,933,015,000)
-        traffic = 20_934_760_000.0
+        # pack launch (20,919,990,000) and the unpack launch (20,920,350,000)
+        traffic = 20_920_170_000.0
     launch_ms = statistics.mean(pack_ms + unpack_ms)
     achieved = 2 * one_way / (launch_ms * 1e-3) / 1e9
     roof = {
