@@ -139,8 +139,6 @@ typedef struct {
     uint32_t lag;        /* BULK: loads issued ahead of the store they feed, 1..stages-2 (0 = default) */
     uint32_t items_per_cta; /* default launch shape: work items per block (0 = about 64 KiB for
                             BULK, 32 KiB for VEC) */
-    uint32_t interleave; /* 0/1 = off; K > 1: the sequence of slabs is cut into K equal ranges that
-                            are walked side by side (K sequential streams open at a time) */
     uint32_t pdl;        /* 0 = default (= 2), 1 = plain launches, 2 = programmatic dependent launch:
                             a kernel's blocks may be scheduled while the previous kernel of the
                             stream drains; they wait for its completion before reading memory */

@@ -67,7 +67,6 @@ struct KvcLaunch {
     uint32_t n_ent;
     uint32_t order;           // kvc_order (never AUTO here)
     uint32_t block_major_chunks;  // chunk layout is [n][L][P].. (else [L][P][n]..)
-    uint32_t interleave;      // >1: that many ranges of the slab sequence are walked side by side
     uint32_t stages;          // bulk kernels
     uint32_t lag;             // bulk kernels: loads issued ahead of the store they feed
     uint32_t l2_evict_first;  // bulk kernels: attach an evict-first L2 policy to the copies

@@ -46,17 +46,6 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
     const KvcGeom &g = a.g;
     uint32_t part = w % g.parts;
     uint32_t r = w / g.parts;
-    bool beyond = false;
-    if (a.interleave > 1) {
-        // K equal ranges of the slab sequence are walked side by side: consecutive work items
-        // come from different ranges, so K sequential streams are open at any time
-        const uint32_t total = a.n_ent * g.planes_total;
-        const uint32_t per = (total + a.interleave - 1) / a.interleave;
-        r = (r % a.interleave) * per + r / a.interleave;
-        beyond = r >= total;
-        if (beyond)
-            r = 0;
-    }
     uint32_t ent, lp;
     if (a.order == KVC_ORDER_PLANE_MAJOR) {
         lp = r / a.n_ent;
@@ -102,10 +91,10 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
     }
     Item it;
     uint32_t off = part * g.tile_bytes;
-    it.len = beyond ? 0u : min(g.tile_bytes, g.slab_bytes - off);
+    it.len = min(g.tile_bytes, g.slab_bytes - off);
     if (id < 0 || id >= (int64_t)g.num_blocks) {
         // never touch memory for a bad id: count the block once and skip it
-        if (count_bad && part == 0 && lp == 0 && !beyond)
+        if (count_bad && part == 0 && lp == 0)
             atomicAdd(a.status, 1u);
         it.len = 0;
         id = 0;

@@ -133,17 +133,13 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     }
     g.tile_bytes = tile;
     g.parts = (uint32_t)((lay->slab_bytes + tile - 1) / tile);
-    uint64_t n_slabs = n_ent * lay->planes_total;
-    if (t.interleave > 1)  // rounded up so that the K ranges are equally long; the excess is skipped
-        n_slabs = (n_slabs + t.interleave - 1) / t.interleave * t.interleave;
-    const uint64_t n_items = n_slabs * g.parts;
+    const uint64_t n_items = n_ent * lay->planes_total * g.parts;
     if (n_items == 0 || n_items > 0xFFFFFFFFull)
         return KVC_ERR_INVALID_ARG;
     a->n_items = n_items;
     a->n_ent = (uint32_t)n_ent;
     a->order = t.order ? t.order : KVC_ORDER_CHUNK_MAJOR;
     a->block_major_chunks = lay->d.chunk_order == KVC_CHUNK_BLOCK_MAJOR;
-    a->interleave = t.interleave;
     a->stages = stages;
     a->lag = lag;
     a->l2_evict_first = t.l2_hint == 2;
@@ -552,7 +548,7 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
         return KVC_ERR_INVALID_ARG;
     if (t->stages == 1 || t->stages > KVC_BULK_MAX_STAGES)
         return KVC_ERR_INVALID_ARG;
-    if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2 || t->interleave > 1024 || t->items_per_cta > (1u << 20))
+    if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2 || t->items_per_cta > (1u << 20))
         return KVC_ERR_INVALID_ARG;
     lay->tuning = *t;
     return KVC_OK;

@@ -54,8 +54,7 @@ class kvc_tuning(ctypes.Structure):
                 ("max_ctas", ctypes.c_uint32), ("tile_bytes", ctypes.c_uint32),
                 ("stages", ctypes.c_uint32), ("ctas_per_sm", ctypes.c_uint32),
                 ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32),
-                ("items_per_cta", ctypes.c_uint32), ("interleave", ctypes.c_uint32),
-                ("pdl", ctypes.c_uint32)]
+                ("items_per_cta", ctypes.c_uint32), ("pdl", ctypes.c_uint32)]
 
 
 class kvc_chunk_desc(ctypes.Structure):
@@ -314,10 +313,9 @@ def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
 
 
 def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
-                          ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, interleave=0,
-                          pdl=0) -> None:
+                          ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, pdl=0) -> None:
     t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag,
-                   items_per_cta, interleave, pdl)
+                   items_per_cta, pdl)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
 
 
