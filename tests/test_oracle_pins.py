@@ -348,3 +348,36 @@ def test_interleaved_kv_pool_order_is_a_strided_plane_view():
     planes = [pl[:(g.NB - 1) * g.P * S + S] for pl in planes]
     ids = rng.permutation(g.NB)[:5].astype(np.int32)
     assert np.array_equal(orc.pack_chunk_planes(g, planes, ids, g.P * S), orc.pack_chunk(g, dense, ids))
+
+
+# ---------------------------------------------------------------- random layouts (hypothesis)
+from hypothesis import given, settings, strategies as st
+
+
+@settings(max_examples=60, deadline=None)
+@given(L=st.integers(1, 4), P=st.integers(1, 3), NB=st.integers(1, 12), B=st.integers(1, 5),
+       H=st.integers(1, 4), D=st.integers(1, 9), e=st.sampled_from([1, 2, 4]),
+       data=st.data())
+def test_random_layouts_against_numpy_and_round_trip(L, P, NB, B, H, D, e, data):
+    g = Dims(L, P, NB, B, H, D, e)
+    n = data.draw(st.integers(1, NB))
+    ids = np.array(data.draw(st.permutations(list(range(NB))))[:n], dtype=np.int32)
+    seed = data.draw(st.integers(0, 2**31))
+    pool = np.random.default_rng(seed).integers(0, 256, g.pool_bytes, dtype=np.uint8)
+    # layer-major chunk = take along the block axis; block-major = the same with that axis first
+    lm = orc.pack_chunk(g, pool, ids)
+    want = np.take(pool.reshape(L, P, NB, -1), ids, axis=2)
+    assert np.array_equal(lm, want.reshape(-1))
+    bm = orc.pack_chunk_planes_block_major(g, orc.dense_planes(g, pool), ids)
+    assert np.array_equal(bm, np.moveaxis(want, 2, 0).reshape(-1))
+    assert np.array_equal(orc.pack_chunk_planes(g, orc.dense_planes(g, pool), ids), lm)
+    # unpack into a sentinel pool restores exactly the named blocks
+    fresh = np.full(g.pool_bytes, 0xA7, dtype=np.uint8)
+    orc.unpack_chunk(g, fresh, lm, ids)
+    f4, p4 = fresh.reshape(L, P, NB, -1), pool.reshape(L, P, NB, -1)
+    assert np.array_equal(f4[:, :, ids], p4[:, :, ids])
+    rest = np.setdiff1d(np.arange(NB), ids)
+    assert (f4[:, :, rest] == 0xA7).all()
+    fresh2 = np.full(g.pool_bytes, 0xA7, dtype=np.uint8)
+    orc.unpack_chunk_planes_block_major(g, orc.dense_planes(g, fresh2), bm, ids)
+    assert np.array_equal(fresh2, fresh)
