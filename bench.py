@@ -471,10 +471,36 @@ def suite_chunk_sweep(torch, kvc, dev, reps):
                     kvc.kvc_unpack(lay, base + off, ids[first:first + nb], nbytes)
                 off += nbytes
 
+        streams = [torch.cuda.Stream() for _ in range(4)]
+        done = [torch.cuda.Event() for _ in streams]
+
+        def per_chunk_streams(direction, ids):
+            # the paper's store pipeline gives every staging slot its own stream (Sec. 6.4): here
+            # the per-chunk launches rotate over four streams, so one kernel's tail overlaps the
+            # next kernel's start
+            cur = torch.cuda.current_stream()
+            start = torch.cuda.Event()
+            start.record(cur)
+            for st in streams:
+                st.wait_event(start)
+            off = 0
+            for i, (_, _, first, nb, nbytes) in enumerate(descs):
+                st = streams[i % len(streams)]
+                if direction == 0:
+                    kvc.kvc_pack(lay, ids[first:first + nb], base + off, nbytes, stream=st)
+                else:
+                    kvc.kvc_unpack(lay, base + off, ids[first:first + nb], nbytes, stream=st)
+                off += nbytes
+            for st, ev in zip(streams, done):
+                ev.record(st)
+                cur.wait_event(ev)
+
         modes = [("batch", lambda: kvc.kvc_pack_batch(lay, ops_p, 0),
                   lambda: kvc.kvc_unpack_batch(lay, ops_u, 0))]
         if len(descs) <= 400:   # 5000 single-chunk launches of 2 MiB are launch-bound by design
             modes.append(("per_chunk", lambda: per_chunk(0, src), lambda: per_chunk(1, dst)))
+            modes.append(("per_chunk_4_streams", lambda: per_chunk_streams(0, src),
+                          lambda: per_chunk_streams(1, dst)))
         for name, fp, fu in modes:
             pm, pd = _time_ms(torch, fp, reps)
             um, ud = _time_ms(torch, fu, reps)

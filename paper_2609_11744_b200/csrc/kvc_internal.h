@@ -23,7 +23,6 @@
 // workloads): two resident blocks per SM, each with two 32 KiB stages (load, then store, no
 // prefetch) and about 64 KiB of work, in chunk-major order: 6.68-6.78 TB/s pack, 6.77-6.88 TB/s
 // unpack where the persistent grid reaches 6.54-6.60 TB/s.
-#define KVC_STREAMING_MIN_BYTES (64ull << 20)
 #define KVC_BULK_STREAMING_BLOCKS_PER_SM 2u
 #define KVC_BULK_STREAMING_STAGES 2u
 #define KVC_BULK_SMEM_HEADER 1024u  // mbarriers + per-stage bookkeeping ahead of the data stages

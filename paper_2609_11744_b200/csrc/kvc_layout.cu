@@ -88,13 +88,11 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     // Two launch shapes.  Streaming (the default): many short-lived blocks, each taking a few
     // consecutive work items, handed out by the hardware scheduler as SMs free up -- measured
     // 2-4 % faster than a persistent grid because it balances itself and throttles the bytes in
-    // flight.  Persistent: a fixed, small number of blocks that stride over all items, used when
+    // flight, and several such launches on different streams share the SMs well (per-chunk
+    // launches rotated over 4 streams reach the batched rate; with persistent grids they lose
+    // 10 %).  Persistent: a fixed, small number of blocks that stride over all items, used when
     // the caller caps the blocks (to leave SMs to a compute stream) or the slot is host memory.
-    // A launch of less than 64 MiB (one 256-token chunk of an 8B-class model) has too few items
-    // for the streaming shape to pay off: measured 4 % slower than a persistent grid there.
-    const uint64_t launch_bytes = n_ent * lay->planes_total * lay->slab_bytes;
-    const bool persistent = t.max_ctas != 0 || host_slot ||
-                            (t.items_per_cta == 0 && launch_bytes < KVC_STREAMING_MIN_BYTES);
+    const bool persistent = t.max_ctas != 0 || host_slot;
     uint32_t tile = t.tile_bytes;
     if (tile == 0)
         tile = (variant == KVC_VARIANT_BULK || !persistent) ? 32768u : 16384u;
@@ -152,8 +150,6 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
         // a slot in host memory is bound by the host link: 16 blocks saturate it (measured), more
         // would only hold SMs while they wait for the link
         grid = KVC_HOST_SLOT_DEFAULT_CTAS;
-    } else if (persistent) {
-        grid = variant == KVC_VARIANT_BULK ? (uint64_t)lay->sm_count : 3ull * lay->sm_count;
     } else {
         // streaming: about 64 KiB (bulk) or 32 KiB (vector) of items per block
         uint32_t per_block = t.items_per_cta;
