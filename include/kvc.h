@@ -116,7 +116,7 @@ uint32_t kvc_layout_num_chunks(const kvc_layout *layout, uint32_t n_blocks);  /*
 typedef enum {
     KVC_VARIANT_AUTO = 0,
     KVC_VARIANT_VEC = 1,  /* 16-byte vector loads/stores through registers */
-    KVC_VARIANT_BULK = 2  /* bulk async copies global->shared->global driven by one warp per SM */
+    KVC_VARIANT_BULK = 2  /* bulk async copies global->shared->global, one warp per thread block */
 } kvc_variant;
 typedef enum {
     KVC_ORDER_AUTO = 0,

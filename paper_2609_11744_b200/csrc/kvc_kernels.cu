@@ -10,13 +10,16 @@
 // in flight and touch every byte once.
 //
 // Two ways to move a tile:
-//   VEC  : every thread keeps KVC_VEC_UNROLL 16-byte loads in flight, then stores
-//          them; streaming cache hints; many resident blocks per SM.
-//   BULK : one warp per SM drives a ring of shared-memory stages with bulk async
+//   VEC  : every thread keeps KVC_VEC_UNROLL 16- or 32-byte loads in flight, then
+//          stores them; streaming cache hints.
+//   BULK : a one-warp block drives a few shared-memory stages with bulk async
 //          copies (global -> shared, completion on an mbarrier; shared -> global,
-//          completion by bulk group).  Lanes decode 32 work items at a time and
-//          hand them to the issuing lane by shuffle.  Almost no registers or
+//          completion by bulk group).  Lanes decode up to 32 work items at a time
+//          and hand them to the issuing lane by shuffle.  Almost no registers or
 //          issue slots are used, which leaves the SM's math pipes to other work.
+// A block handles items blockIdx.x, blockIdx.x + gridDim.x, ...: with a large grid
+// every block takes a couple of items and retires (the default), with a small one
+// the blocks persist and stride over everything.
 // No cluster, no multicast: every byte is read exactly once by exactly one SM.
 #include <string.h>
 
