@@ -2,6 +2,7 @@
 steps are a barrier and a max over ranks of the measured time.  Run as two gloo processes."""
 import json
 import os
+import socket
 import subprocess
 import sys
 
@@ -27,11 +28,17 @@ dist.destroy_process_group()
 """
 
 
+def _free_port() -> int:
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def _torchrun(args, timeout):
     env = dict(os.environ, MASTER_ADDR="127.0.0.1", OMP_NUM_THREADS="1")
     return subprocess.run([sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
                            "--nproc-per-node", "2", "--master-addr", "127.0.0.1",
-                           "--master-port", "29431"] + args,
+                           "--master-port", str(_free_port())] + args,
                           cwd=ROOT, env=env, capture_output=True, text=True, timeout=timeout)
 
 
