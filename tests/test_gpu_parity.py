@@ -666,6 +666,8 @@ def test_per_chunk_calls_replay_from_a_cuda_graph():
     dict(variant=2, ctas_per_sm=2, stages=3), dict(variant=2, ctas_per_sm=4, tile_bytes=16384),
     dict(variant=2, l2_hint=2), dict(variant=2, pdl=1), dict(variant=1, pdl=1, tile_bytes=32768),
     dict(variant=1, max_ctas=1), dict(variant=2, max_ctas=1, stages=2),
+    dict(items_per_cta=1), dict(items_per_cta=7, stages=3), dict(variant=1, items_per_cta=3),
+    dict(variant=2, order=1, items_per_cta=5), dict(variant=1, order=2, tile_bytes=4096),
 ])
 def test_tuning_knobs_do_not_change_results(tuning):
     g = orc.Dims(8, 2, 96, 16, 8, 128, 2)
