@@ -91,3 +91,96 @@ def test_config2_8b_8k_prefix():
 @pytest.mark.parametrize("chunk_tokens", [256, 16, 2048])
 def test_config3_8b_80k_prefix(chunk_tokens):
     _full_size_case(wl.WORKLOADS["8b_80k"], chunk_tokens)
+
+
+def test_config4_70b_batch_one_call_unpack():
+    """64 requests (lognormal lengths, shared 1024-token prefix), 70B-class shape, every kept chunk
+    unpacked by ONE kvc_unpack_batch call, at full size; sampled elements against the oracle's
+    index formulas, plus whole-block equality for a few hundred blocks."""
+    w = wl.WORKLOADS["70b_batch"]
+    s = w.shape
+    NB, tables = wl.batch_workload(w, 1.0)
+    lay_probe = kvc.kvc_layout_create_dense(0x100000, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    descs, uniq = kvc.kvc_map_requests_shared(lay_probe, tables)
+    total = sum(d[4] for d in descs)
+    free, _ = torch.cuda.mem_get_info()
+    if free < NB * s.bytes_per_block + total + (4 << 30):
+        pytest.skip("needs %.0f GiB of free device memory" % ((NB * s.bytes_per_block + total) / 2**30))
+    g = orc.Dims(s.L, s.P, NB, s.B, s.H, s.D, s.e)
+    pool = torch.zeros(NB * s.bytes_per_block, dtype=torch.uint8, device=DEV)
+    staging = wl.random_bits_cuda(w.seed + 3, total, DEV)
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    slot, ids, nbs, offs, off = [], [], [], [], 0
+    for (r, c, first, nb, nbytes) in descs:
+        slot.append(staging.data_ptr() + off)
+        ids.append(tables[r].ctypes.data + 4 * first)
+        nbs.append(nb)
+        offs.append(off)
+        off += nbytes
+    kvc.kvc_unpack_batch(lay, kvc.make_chunk_ops(slot, ids, nbs), 0)
+    torch.cuda.synchronize()
+    assert kvc.kvc_layout_launch_count(lay) == 1 and kvc.kvc_poll_device_status(lay) == (0, 0)
+    # sampled elements: op k, block j of it, coordinates (l, p, t, h, d)
+    rng = np.random.default_rng(4)
+    k = rng.integers(0, len(descs), N_SAMPLES)
+    nb_c = np.array(nbs)[k]
+    j = (rng.random(N_SAMPLES) * nb_c).astype(np.int64)
+    l, p = rng.integers(0, g.L, N_SAMPLES), rng.integers(0, g.P, N_SAMPLES)
+    t, h, d = (rng.integers(0, q, N_SAMPLES) for q in (g.B, g.H, g.D))
+    first = np.array([dd[2] for dd in descs])[k]
+    req = np.array([dd[0] for dd in descs])[k]
+    flat_tables = np.concatenate(tables)
+    starts = np.concatenate([[0], np.cumsum([len(t_) for t_ in tables])[:-1]])
+    blk = flat_tables[starts[req] + first + j].astype(np.int64)
+    stage_pos = np.array(offs, dtype=np.int64)[k] // g.e + orc.chunk_elem(g, nb_c, l, p, j, t, h, d)
+    pool_pos = orc.pool_elem(g, l, p, blk, t, h, d)
+    dev_idx = lambda a: torch.from_numpy(a).to(DEV)
+    assert torch.equal(pool.view(torch.int16)[dev_idx(pool_pos)],
+                       staging.view(torch.int16)[dev_idx(stage_pos)])
+    # blocks of no request stay zero; a few hundred written blocks are compared in full
+    named = np.unique(flat_tables)
+    assert len(named) == uniq
+    untouched = np.setdiff1d(np.arange(NB), named)[:128]
+    pool4 = pool.view(s.L * s.P, NB, s.slab_bytes)
+    assert bool((pool4[:, dev_idx(untouched.astype(np.int64))] == 0).all())
+    for kk in rng.integers(0, len(descs), 12):
+        (r, c, f, nb, nbytes) = descs[kk]
+        chunk = staging[offs[kk]:offs[kk] + nbytes].view(s.L * s.P, nb, s.slab_bytes)
+        ids_t = dev_idx(tables[r][f:f + nb].astype(np.int64))
+        assert torch.equal(pool4[:, ids_t], chunk)
+
+
+def test_config5_32k_prefix_streamed_through_8_slot_ring_to_host():
+    """The 32k-token prefix (4 GiB) of the ring config streamed through 8 slots x 256 tokens into
+    pinned host memory: sampled host elements against the oracle's positions in the device pool."""
+    w = wl.WORKLOADS["8b_ring"]
+    s = w.shape
+    NB, n = w.pool_blocks, w.request_blocks
+    g = orc.Dims(s.L, s.P, NB, s.B, s.H, s.D, s.e)
+    from paper_2609_11744_b200 import cuda_rt
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, DEV)
+    src = wl.block_ids(w.seed, NB, n)
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    descs = kvc.kvc_map_request(lay, n)
+    assert len(descs) == 128
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    ring = kvc.kvc_staging_ring_create(cb, int(w.extra["ring_slots"]), kvc.KVC_RING_DEVICE)
+    host = torch.empty(n * s.bytes_per_block, dtype=torch.uint8, pin_memory=True)
+    s_k, s_c = torch.cuda.Stream(), torch.cuda.Stream()
+    off = 0
+    for (_, c, first, nb, nbytes) in descs:
+        slot, dptr, _ = kvc.kvc_staging_ring_acquire(ring, 10_000_000)
+        assert slot == c % 8
+        kvc.kvc_pack(lay, src[first:first + nb], dptr, nbytes, stream=s_k)
+        kvc.kvc_staging_ring_commit(ring, slot, s_k)
+        kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
+        cuda_rt.memcpy_async(host.data_ptr() + off, dptr, nbytes, cuda_rt.D2H, s_c)
+        kvc.kvc_staging_ring_release(ring, slot, s_c)
+        off += nbytes
+    torch.cuda.synchronize()
+    assert kvc.kvc_staging_ring_stats(ring)[1] == 128            # 16 laps of the 8-slot ring
+    blk, stage_pos, src_pos, _ = _sampled_positions(g, src, src, 16, w.seed)
+    want = pool.view(torch.int16)[torch.from_numpy(src_pos).to(DEV)].cpu()
+    got = host.view(torch.int16)[torch.from_numpy(stage_pos)]
+    assert torch.equal(got, want)
+    kvc.kvc_staging_ring_destroy(ring)
