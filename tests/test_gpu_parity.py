@@ -693,3 +693,27 @@ def test_tuning_knobs_do_not_change_results(tuning):
     assert np.array_equal(staging.cpu().numpy(), np.concatenate(want_chunks))
     assert np.array_equal(pool_t.cpu().numpy(), want_pool)
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+# ------------------------------------------------------------------ the C ABI from plain C
+def test_plain_c_program_links_and_runs(tmp_path):
+    """include/kvc.h is a C header: a C99 program built with gcc against libkvc.so packs and
+    unpacks on the GPU and checks the bytes itself."""
+    import os
+    import shutil
+    import subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    if shutil.which("gcc") is None or not os.path.isdir(os.path.join(cuda, "include")):
+        pytest.skip("needs gcc and the CUDA toolkit headers")
+    exe = str(tmp_path / "c_abi_smoke")
+    pkg = os.path.join(root, "paper_2609_11744_b200")
+    build = subprocess.run(
+        ["gcc", "-std=c99", "-O1", "-Wall", os.path.join(root, "tests", "native", "c_abi_smoke.c"),
+         "-I", os.path.join(root, "include"), "-I", os.path.join(cuda, "include"),
+         "-L", pkg, "-lkvc", "-L", os.path.join(cuda, "lib64"), "-lcudart",
+         "-Wl,-rpath," + pkg, "-Wl,-rpath," + os.path.join(cuda, "lib64"), "-o", exe],
+        capture_output=True, text=True)
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+    assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr
