@@ -353,3 +353,13 @@ def test_ring_trace_records_transitions_in_order(fake_events):
     kvc.kvc_staging_ring_acquire(ring)
     assert kvc.kvc_staging_ring_trace_count(ring) == 0
     kvc.kvc_staging_ring_destroy(ring)
+
+
+def test_header_is_plain_c99():
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("needs gcc")
+    r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
+                        "-x", "c", os.path.join(ROOT, "include", "kvc.h")], capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
