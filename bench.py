@@ -618,6 +618,52 @@ def _overlap_case(torch, fn, gemm_loop, s_gemm, s_k, s_c, iters, seconds, one_wa
             "overlap_efficiency": eff}
 
 
+def _grouped_runs(torch, kvc, cuda_rt, pool, s, NB, n, src, dst, hptr, one_way, N, gemm_loop, s_gemm,
+                  s_k, s_c, iters, seconds, GROUP, n_ring, TO):
+    """Several ring slots per launch: one batched pack/unpack serves GROUP slots, so the compute
+    stream is interrupted GROUP times less often."""
+    out = []
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+    descs = kvc.kvc_map_request(lay, n)
+    cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+    ring = kvc.kvc_staging_ring_create(cb, n_ring, kvc.KVC_RING_DEVICE)
+
+    def grouped(direction):
+        off = 0
+        for g0 in range(0, len(descs), GROUP):
+            grp = descs[g0:g0 + GROUP]
+            slots = [kvc.kvc_staging_ring_acquire(ring, TO) for _ in grp]
+            ops = kvc.make_chunk_ops([sl[1] for sl in slots],
+                                     [(src if direction == 0 else dst).ctypes.data + 4 * d[2] for d in grp],
+                                     [d[3] for d in grp])
+            if direction == 0:
+                kvc.kvc_pack_batch(lay, ops, 0, stream=s_k)
+                for (slot, dptr, _), d in zip(slots, grp):
+                    kvc.kvc_staging_ring_commit(ring, slot, s_k)
+                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
+                    cuda_rt.memcpy_async(hptr + off, dptr, d[4], cuda_rt.D2H, s_c)
+                    kvc.kvc_staging_ring_release(ring, slot, s_c)
+                    off += d[4]
+            else:
+                for (slot, dptr, _), d in zip(slots, grp):
+                    cuda_rt.memcpy_async(dptr, hptr + off, d[4], cuda_rt.H2D, s_c)
+                    kvc.kvc_staging_ring_commit(ring, slot, s_c)
+                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_k)
+                    off += d[4]
+                kvc.kvc_unpack_batch(lay, ops, 0, stream=s_k)
+                for (slot, dptr, _) in slots:
+                    kvc.kvc_staging_ring_release(ring, slot, s_k)
+
+    for direction, name in ((0, "offload"), (1, "load")):
+        out.append(_overlap_case(torch, lambda: grouped(direction), gemm_loop, s_gemm, s_k, s_c,
+                                 iters, seconds, one_way, N,
+                                 "device slots + cudaMemcpyAsync, %d slots per launch, %d-slot ring"
+                                 % (GROUP, n_ring), name, 0))
+    kvc.kvc_staging_ring_destroy(ring)
+    kvc.kvc_layout_destroy(lay)
+    return out
+
+
 def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
     """Config 5: a 32k-token prefix (8B shape, 4 GiB) streamed through an 8-slot ring of 256-token
     slots to/from pinned host memory while a bf16 GEMM loop runs on another stream.  Destinations:
@@ -711,47 +757,9 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
                                              one_way, N, kind_name, direction, max_ctas))
             kvc.kvc_staging_ring_destroy(ring)
             kvc.kvc_layout_destroy(lay)
-    # several ring slots per launch: one batched pack/unpack serves GROUP slots, so the compute
-    # stream is interrupted GROUP times less often
-    GROUP = 4
-    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
-    descs = kvc.kvc_map_request(lay, n)
-    cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
-    ring = kvc.kvc_staging_ring_create(cb, int(w.extra["ring_slots"]), kvc.KVC_RING_DEVICE)
-
-    def grouped(direction):
-        off = 0
-        for g0 in range(0, len(descs), GROUP):
-            grp = descs[g0:g0 + GROUP]
-            slots = [kvc.kvc_staging_ring_acquire(ring, TO) for _ in grp]
-            ops = kvc.make_chunk_ops([sl[1] for sl in slots],
-                                     [(src if direction == 0 else dst).ctypes.data + 4 * d[2] for d in grp],
-                                     [d[3] for d in grp])
-            if direction == 0:
-                kvc.kvc_pack_batch(lay, ops, 0, stream=s_k)
-                for (slot, dptr, _), d in zip(slots, grp):
-                    kvc.kvc_staging_ring_commit(ring, slot, s_k)
-                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
-                    cuda_rt.memcpy_async(hptr + off, dptr, d[4], cuda_rt.D2H, s_c)
-                    kvc.kvc_staging_ring_release(ring, slot, s_c)
-                    off += d[4]
-            else:
-                for (slot, dptr, _), d in zip(slots, grp):
-                    cuda_rt.memcpy_async(dptr, hptr + off, d[4], cuda_rt.H2D, s_c)
-                    kvc.kvc_staging_ring_commit(ring, slot, s_c)
-                    kvc.kvc_staging_ring_wait_filled(ring, slot, s_k)
-                    off += d[4]
-                kvc.kvc_unpack_batch(lay, ops, 0, stream=s_k)
-                for (slot, dptr, _) in slots:
-                    kvc.kvc_staging_ring_release(ring, slot, s_k)
-
-    for direction, name in ((0, "offload"), (1, "load")):
-        results.append(_overlap_case(torch, lambda: grouped(direction), gemm_loop, s_gemm, s_k, s_c,
-                                     iters, seconds, one_way, N,
-                                     "device slots + cudaMemcpyAsync, %d slots per launch" % GROUP,
-                                     name, 0))
-    kvc.kvc_staging_ring_destroy(ring)
-    kvc.kvc_layout_destroy(lay)
+    for GROUP, n_ring in ((4, int(w.extra["ring_slots"])), (8, 16)):
+        results.extend(_grouped_runs(torch, kvc, cuda_rt, pool, s, NB, n, src, dst, hptr, one_way, N,
+                                     gemm_loop, s_gemm, s_k, s_c, iters, seconds, GROUP, n_ring, TO))
     # the paper's mechanism for comparison: strided DMA copies straight between the pool and
     # pinned host memory, no kernel, no staging slot
     lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
