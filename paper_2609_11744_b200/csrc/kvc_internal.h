@@ -11,7 +11,8 @@
 
 #define KVC_PARAM_IDS 128u      // block ids that travel inside the kernel parameters
 #define KVC_VEC_THREADS 256u    // threads per block of the vector kernels
-#define KVC_VEC_UNROLL 4u       // 16-byte vectors in flight per thread
+#define KVC_VEC_UNROLL 4u       // vectors in flight per thread
+#define KVC_VEC_WARP_TEAM_MAX_TILE 4096u  // tiles up to this size are copied by one warp each
 #define KVC_HOST_SLOT_DEFAULT_CTAS 16u
 #define KVC_BULK_THREADS 32u    // one warp drives the bulk-copy pipeline
 #define KVC_BULK_MAX_STAGES 16u

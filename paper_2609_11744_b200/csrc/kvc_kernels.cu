@@ -164,39 +164,43 @@ struct Vec<32> {
     }
 };
 
-template <int DIR, bool TABLE, int VB>
+// TEAM threads share one work item: the whole block for ordinary tiles, one warp for tiles of at
+// most 4 KiB (small slabs), so that eight small items are in flight per block instead of one.
+template <int DIR, bool TABLE, int VB, int TEAM>
 __global__ void __launch_bounds__(KVC_VEC_THREADS)
 kvc_vec_kernel(const __grid_constant__ KvcLaunch a)
 {
     constexpr uint32_t SH = VB == 32 ? 5 : 4;
-    const uint32_t tid = threadIdx.x;
+    constexpr uint32_t TEAMS = KVC_VEC_THREADS / TEAM;
+    const uint32_t t = threadIdx.x % TEAM;
     const uint32_t n_items = (uint32_t)a.n_items;
-    uint32_t w = blockIdx.x;
+    const uint64_t stride = (uint64_t)gridDim.x * TEAMS;
+    uint64_t w = (uint64_t)blockIdx.x * TEAMS + threadIdx.x / TEAM;
     grid_dependency_wait();
     if (w >= n_items)
         return;
-    Item cur = decode<TABLE>(a, w, tid == 0);
+    Item cur = decode<TABLE>(a, (uint32_t)w, t == 0);
     while (true) {
         // decode the next item before the copy so its table read overlaps the data loads
-        uint32_t wn = w + gridDim.x;
-        bool more = wn < n_items && wn > w;
+        const uint64_t wn = w + stride;
+        const bool more = wn < n_items;
         Item nxt = cur;
         if (more)
-            nxt = decode<TABLE>(a, wn, tid == 0);
+            nxt = decode<TABLE>(a, (uint32_t)wn, t == 0);
         const uint64_t src = DIR == KVC_DIR_PACK ? cur.pool : cur.slot;
         const uint64_t dst = DIR == KVC_DIR_PACK ? cur.slot : cur.pool;
         const uint32_t nvec = cur.len >> SH;
-        for (uint32_t v0 = 0; v0 < nvec; v0 += KVC_VEC_THREADS * KVC_VEC_UNROLL) {
+        for (uint32_t v0 = 0; v0 < nvec; v0 += TEAM * KVC_VEC_UNROLL) {
             Vec<VB> r[KVC_VEC_UNROLL];
 #pragma unroll
             for (uint32_t u = 0; u < KVC_VEC_UNROLL; ++u) {
-                uint32_t v = v0 + u * KVC_VEC_THREADS + tid;
+                uint32_t v = v0 + u * TEAM + t;
                 if (v < nvec)
                     r[u].load(src + ((uint64_t)v << SH));
             }
 #pragma unroll
             for (uint32_t u = 0; u < KVC_VEC_UNROLL; ++u) {
-                uint32_t v = v0 + u * KVC_VEC_THREADS + tid;
+                uint32_t v = v0 + u * TEAM + t;
                 if (v < nvec)
                     r[u].store(dst + ((uint64_t)v << SH));
             }
@@ -449,9 +453,16 @@ cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t 
         }
         return launch_cfg(kvc_bulk_kernel<DIR, TABLE>, a, grid, KVC_BULK_THREADS, smem, stream);
     }
+    const bool warp_team = a.g.tile_bytes <= KVC_VEC_WARP_TEAM_MAX_TILE;
     if (variant == KVC_VARIANT_VEC32)
-        return launch_cfg(kvc_vec_kernel<DIR, TABLE, 32>, a, grid, KVC_VEC_THREADS, 0, stream);
-    return launch_cfg(kvc_vec_kernel<DIR, TABLE, 16>, a, grid, KVC_VEC_THREADS, 0, stream);
+        return warp_team
+                   ? launch_cfg(kvc_vec_kernel<DIR, TABLE, 32, 32>, a, grid, KVC_VEC_THREADS, 0, stream)
+                   : launch_cfg(kvc_vec_kernel<DIR, TABLE, 32, KVC_VEC_THREADS>, a, grid, KVC_VEC_THREADS,
+                                0, stream);
+    return warp_team
+               ? launch_cfg(kvc_vec_kernel<DIR, TABLE, 16, 32>, a, grid, KVC_VEC_THREADS, 0, stream)
+               : launch_cfg(kvc_vec_kernel<DIR, TABLE, 16, KVC_VEC_THREADS>, a, grid, KVC_VEC_THREADS, 0,
+                            stream);
 }
 
 }  // namespace
@@ -479,5 +490,5 @@ cudaError_t kvc_kernel_limits(int *sm_count, int *vec_blocks_per_sm, int *max_sm
         cudaSuccess)
         return e;
     return cudaOccupancyMaxActiveBlocksPerMultiprocessor(
-        vec_blocks_per_sm, kvc_vec_kernel<KVC_DIR_PACK, true, 32>, KVC_VEC_THREADS, 0);
+        vec_blocks_per_sm, kvc_vec_kernel<KVC_DIR_PACK, true, 32, KVC_VEC_THREADS>, KVC_VEC_THREADS, 0);
 }
