@@ -513,6 +513,53 @@ def suite_chunk_sweep(torch, kvc, dev, reps):
     return out
 
 
+def suite_launch_shapes(torch, kvc, dev, reps):
+    """Same-process comparison of launch shapes and traversal orders on the 80k-token prefix (the
+    boxes of a pool differ by a percent or so, so only numbers from one process compare)."""
+    w = wl.WORKLOADS["8b_80k"]
+    s, NB, n = w.shape, w.pool_blocks, w.request_blocks
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    src, dst = wl.block_ids(w.seed, NB, n), wl.block_ids(w.dst_seed, NB, n)
+    one_way = n * s.bytes_per_block
+    staging = torch.empty(one_way, dtype=torch.uint8, device=dev)
+    other = torch.empty_like(staging)
+    tm, td = _time_ms(torch, lambda: other.copy_(staging), reps)
+    del other
+    out = [{"name": "torch contiguous copy_ of the same bytes (context)", "pack_ms": td,
+            "pack_gbs": 2 * one_way / td / 1e6, "unpack_ms": None, "unpack_gbs": None}]
+    P, B, C = kvc.KVC_ORDER_PLANE_MAJOR, kvc.KVC_ORDER_BLOCK_MAJOR, kvc.KVC_ORDER_CHUNK_MAJOR
+    cands = [
+        ("default: bulk, streaming (2 items/block, 2 stages), chunk-major", dict()),
+        ("bulk streaming, 1 item per block", dict(items_per_cta=1)),
+        ("bulk streaming, 4 items per block", dict(items_per_cta=4)),
+        ("bulk streaming, 8 items per block, 3 stages", dict(items_per_cta=8, stages=3)),
+        ("bulk streaming, plane-major", dict(order=P)),
+        ("bulk streaming, block-major", dict(order=B)),
+        ("bulk persistent 148 blocks, 4 stages, 1 load ahead, chunk-major", dict(max_ctas=148, order=C)),
+        ("bulk persistent 148 blocks, 4 stages, 1 load ahead, plane-major", dict(max_ctas=148, order=P)),
+        ("bulk persistent 148 blocks, 7 stages, 5 loads ahead", dict(max_ctas=148, stages=7, lag=5)),
+        ("bulk persistent 148 blocks, 2 stages (serial)", dict(max_ctas=148, stages=2)),
+        ("bulk persistent 148 blocks, 16 KiB tiles, 8 stages, 1 ahead", dict(max_ctas=148, tile_bytes=16384, stages=8)),
+        ("bulk persistent 148 blocks, L2 evict-first hint", dict(max_ctas=148, l2_hint=2)),
+        ("bulk persistent 96 blocks, 4 stages, 2 loads ahead", dict(max_ctas=96, lag=2)),
+        ("vector streaming (1 item of 32 KiB per block), chunk-major", dict(variant=1)),
+        ("vector persistent 444 blocks, 16 KiB tiles", dict(variant=1, max_ctas=444, tile_bytes=16384)),
+        ("vector persistent 592 blocks, 16 KiB tiles", dict(variant=1, max_ctas=592, tile_bytes=16384)),
+    ]
+    for name, cfg in cands:
+        lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+        kvc.kvc_layout_set_tuning(lay, **cfg)
+        ops_p, k1, _, _ = kvc.request_chunk_ops(lay, src, staging)
+        ops_u, k2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+        pm, pd = _time_ms(torch, lambda: kvc.kvc_pack_batch(lay, ops_p, 0), reps)
+        um, ud = _time_ms(torch, lambda: kvc.kvc_unpack_batch(lay, ops_u, 0), reps)
+        assert kvc.kvc_poll_device_status(lay) == (0, 0)
+        out.append({"name": name, "tuning": cfg, "pack_ms": pd, "pack_gbs": 2 * one_way / pd / 1e6,
+                    "unpack_ms": ud, "unpack_gbs": 2 * one_way / ud / 1e6})
+        kvc.kvc_layout_destroy(lay)
+    return out
+
+
 def suite_8k(torch, kvc, dev, reps):
     """Config 2: 8192-token prefix (1 GiB each way) with L2 flushed between timed launches."""
     w = wl.WORKLOADS["8b_8k"]
@@ -860,6 +907,7 @@ def run_suite(args):
     parts = args.suite.split(",")
     out = {"suite": True, "peak_hbm_gbs": measured_peak()[0], "data": "synthetic"}
     for name, fn in (("host_link", lambda: suite_host_link(torch, cuda_rt, dev)),
+                     ("launch_shapes", lambda: suite_launch_shapes(torch, kvc, dev, args.steps)),
                      ("chunk_sweep", lambda: suite_chunk_sweep(torch, kvc, dev, args.steps)),
                      ("prefix_8k", lambda: suite_8k(torch, kvc, dev, args.steps)),
                      ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
@@ -897,7 +945,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
-                         "host_link,chunk_sweep,prefix_8k,batch_70b,ring_overlap,file_pipeline (1 GPU; prints one JSON line)")
+                         "host_link,launch_shapes,chunk_sweep,prefix_8k,batch_70b,ring_overlap,file_pipeline (1 GPU; prints one JSON line)")
     ap.add_argument("--overlap-seconds", type=float, default=2.0)
     ap.add_argument("--file-roots", default="/tmp,/dev/shm",
                     help="comma list of directories for the file_pipeline suite part")
