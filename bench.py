@@ -497,13 +497,14 @@ def suite_chunk_sweep(torch, kvc, dev, reps):
 
         modes = [("batch", lambda: kvc.kvc_pack_batch(lay, ops_p, 0),
                   lambda: kvc.kvc_unpack_batch(lay, ops_u, 0))]
-        if len(descs) <= 400:   # 5000 single-chunk launches of 2 MiB are launch-bound by design
-            modes.append(("per_chunk", lambda: per_chunk(0, src), lambda: per_chunk(1, dst)))
-            modes.append(("per_chunk_4_streams", lambda: per_chunk_streams(0, src),
-                          lambda: per_chunk_streams(1, dst)))
+        modes.append(("per_chunk", lambda: per_chunk(0, src), lambda: per_chunk(1, dst)))
+        modes.append(("per_chunk_4_streams", lambda: per_chunk_streams(0, src),
+                      lambda: per_chunk_streams(1, dst)))
         for name, fp, fu in modes:
-            pm, pd = _time_ms(torch, fp, reps)
-            um, ud = _time_ms(torch, fu, reps)
+            # 5000 single-chunk launches of 2 MiB are launch-bound by design: fewer repetitions
+            r = reps if len(descs) <= 400 or name == "batch" else max(3, reps // 4)
+            pm, pd = _time_ms(torch, fp, r)
+            um, ud = _time_ms(torch, fu, r)
             out.append({"chunk_tokens": chunk_tokens, "chunks": len(descs), "mode": name,
                         "pack_ms_min": pm, "pack_ms_median": pd, "pack_gbs": 2 * one_way / pd / 1e6,
                         "unpack_ms_min": um, "unpack_ms_median": ud,
