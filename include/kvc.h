@@ -112,10 +112,12 @@ uint32_t kvc_layout_blocks_per_chunk(const kvc_layout *layout);     /* chunk_tok
 uint64_t kvc_layout_chunk_bytes(const kvc_layout *layout, uint32_t n_blocks); /* L*P*n*slab */
 uint32_t kvc_layout_num_chunks(const kvc_layout *layout, uint32_t n_blocks);  /* ceil(n / bpc) */
 
-/* How the copy kernels run.  Zero in every field means "library default". */
+/* How the copy kernels run.  Zero in every field means "library default" (AUTO: the bulk-copy
+ * kernel for slots in device memory, the vector kernel with 16 persistent blocks for slots in
+ * mapped host memory; chunk-major order). */
 typedef enum {
     KVC_VARIANT_AUTO = 0,
-    KVC_VARIANT_VEC = 1,  /* 16-byte vector loads/stores through registers */
+    KVC_VARIANT_VEC = 1,  /* 16- or 32-byte vector loads/stores through registers */
     KVC_VARIANT_BULK = 2  /* bulk async copies global->shared->global, one warp per thread block */
 } kvc_variant;
 typedef enum {
@@ -134,7 +136,8 @@ typedef struct {
                             compute stream */
     uint32_t tile_bytes; /* bytes of one slab moved per work item (0 = default); multiple of 16 */
     uint32_t stages;     /* BULK: shared-memory stages per thread block (0 = default) */
-    uint32_t ctas_per_sm; /* BULK: resident thread blocks per SM, 1..4 (0 = default) */
+    uint32_t ctas_per_sm; /* BULK: thread blocks the shared memory of one SM is divided among,
+                            1..4 (0 = default); bounds stages * tile_bytes per block */
     uint32_t l2_hint;    /* BULK: 0 = default, 1 = no L2 priority hint, 2 = evict-first on loads and stores */
     uint32_t lag;        /* BULK: loads issued ahead of the store they feed, 1..stages-2 (0 = default) */
     uint32_t items_per_cta; /* default launch shape: work items per block (0 = about 64 KiB for
