@@ -363,3 +363,40 @@ def test_header_is_plain_c99():
     r = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only",
                         "-x", "c", os.path.join(ROOT, "include", "kvc.h")], capture_output=True, text=True)
     assert r.returncode == 0, r.stderr
+
+
+def test_descriptor_fuzz_never_crashes_and_derived_sizes_hold():
+    """Random descriptors, valid or not: creation either fails with a status or yields a handle whose
+    derived sizes obey the Sec. 2.1 formula; nothing crashes."""
+    rng = np.random.default_rng(99)
+    made = 0
+    def pick(good, bad):
+        return int(rng.choice(good)) if rng.random() < 0.9 else int(rng.choice(bad))
+
+    for _ in range(400):
+        L, P = pick([1, 2, 4], [0]), pick([1, 2], [0, 3])
+        NB, B = pick([1, 7, 40], [0]), pick([1, 4, 16], [0, 3])
+        H, D = pick([1, 2, 4], [0, 5]), pick([8, 16, 64, 128], [0, 1, 3, 100])
+        e = pick([1, 2, 4], [0, 3, 8])
+        chunk = pick([B, 2 * B, 16 * B], [0, B + 1, 7])
+        base = pick([0x10000, 0x10010], [0, 0x10004])
+        slab = B * H * D * e
+        plane = pick([slab * NB, slab * NB + 16], [0, 8])
+        try:
+            lay = kvc.kvc_layout_create(L, P, NB, B, H, D, e, chunk, base=base,
+                                        layer_stride=plane * max(P, 1), plane_stride=plane,
+                                        block_stride=pick([0, slab], [slab + 16, 7]),
+                                        chunk_order=pick([0, 1], [2]))
+        except kvc.KvcError as err:
+            assert 1 <= err.status <= 13
+            continue
+        made += 1
+        assert kvc.kvc_layout_slab_bytes(lay) == slab and slab % 16 == 0
+        assert kvc.kvc_layout_bytes_per_token(lay) == L * P * H * D * e
+        assert chunk % B == 0 and kvc.kvc_layout_blocks_per_chunk(lay) == chunk // B
+        n = int(rng.integers(0, 200))
+        assert kvc.kvc_layout_chunk_bytes(lay, n) == L * P * n * slab
+        d = kvc.kvc_map_request(lay, n)
+        assert sum(x[3] for x in d) == n and sum(x[4] for x in d) == L * P * n * slab
+        kvc.kvc_layout_destroy(lay)
+    assert made > 3

@@ -350,6 +350,41 @@ def test_batched_unpack_of_many_requests_with_shared_prefix():
 
 
 # ------------------------------------------------------------------ config 5 (reduced): ring streaming
+@pytest.mark.parametrize("variant", VARIANTS)
+def test_small_slabs_through_mapped_host_slots(variant):
+    """Slabs of 512 bytes (the vector kernel gives each to one warp) packed straight into a slot in
+    mapped pinned host memory and unpacked from it."""
+    g = orc.Dims(6, 2, 200, 4, 2, 32, 2)              # S = 512 B
+    pool = wl.random_bits(1500, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 4 * 32)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    src, dst = wl.block_ids(15, g.NB, 70), wl.block_ids(16, g.NB, 70)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 32)
+    ring = kvc.kvc_staging_ring_create((cb + 4095) // 4096 * 4096, 3, kvc.KVC_RING_HOST_MAPPED)
+    want_chunks = orc.pack_request(g, pool, src, 4 * 32)
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, want_chunks, dst, 4 * 32)
+    import ctypes
+    held = []
+    for c, (first, nb) in enumerate(orc.chunk_ranges(70, 32)):     # 3 chunks, 3 slots: pack them all
+        slot, dptr, hptr = kvc.kvc_staging_ring_acquire(ring, 1_000_000)
+        nbytes = kvc.kvc_layout_chunk_bytes(lay, nb)
+        kvc.kvc_pack(lay, src[first:first + nb], dptr, nbytes)
+        kvc.kvc_staging_ring_commit(ring, slot)
+        kvc.kvc_staging_ring_sync_filled(ring, slot)
+        got = np.ctypeslib.as_array((ctypes.c_uint8 * nbytes).from_address(hptr))
+        assert np.array_equal(got, want_chunks[c]), "chunk %d" % c
+        held.append((slot, dptr, first, nb, nbytes))
+    for slot, dptr, first, nb, nbytes in held:                      # then unpack them from the slots
+        kvc.kvc_unpack(lay, dptr, dst[first:first + nb], nbytes)
+        kvc.kvc_staging_ring_release(ring, slot)
+    torch.cuda.synchronize()
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+    kvc.kvc_staging_ring_destroy(ring)
+
+
 @pytest.mark.parametrize("kind", [kvc.KVC_RING_DEVICE, kvc.KVC_RING_HOST_MAPPED])
 def test_prefix_streamed_through_ring_equals_one_shot_pack(kind):
     """A 2048-token prefix (8 chunks of 256 tokens) through a 3-slot ring while the copy stream
