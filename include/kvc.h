@@ -94,6 +94,16 @@ typedef struct {
     uint32_t reserved;     /* must be 0 */
 } kvc_layout_desc;
 
+/* Fills *desc for a pool that is one dense allocation [layer][K|V][block][token][head][dim]
+ * starting at `base` (Sec. 2.1 layout, no padding anywhere): plane_ptrs = NULL, plane stride =
+ * num_blocks * slab bytes, layer stride = kv_planes * plane stride, block stride = slab bytes.
+ * Pure arithmetic, no validation beyond NULL (kvc_layout_create validates).  INVALID_ARG if desc
+ * is NULL or a product overflows 64 bits. */
+kvc_status kvc_layout_desc_init_dense(kvc_layout_desc *desc, const void *base, uint32_t num_layers,
+                                      uint32_t kv_planes, uint32_t num_blocks, uint32_t block_size,
+                                      uint32_t num_kv_heads, uint32_t head_dim, uint32_t elem_bytes,
+                                      uint32_t chunk_tokens, uint32_t chunk_order);
+
 /* Validates and copies the descriptor.  Makes no CUDA call: the small device-side
  * state a launch needs (plane-pointer table, status words, id-table arenas) is
  * allocated by the first pack/unpack call on the handle, which therefore must not
@@ -112,13 +122,15 @@ uint32_t kvc_layout_blocks_per_chunk(const kvc_layout *layout);     /* chunk_tok
 uint64_t kvc_layout_chunk_bytes(const kvc_layout *layout, uint32_t n_blocks); /* L*P*n*slab */
 uint32_t kvc_layout_num_chunks(const kvc_layout *layout, uint32_t n_blocks);  /* ceil(n / bpc) */
 
-/* How the copy kernels run.  Zero in every field means "library default" (AUTO: the bulk-copy
+/* How the copy kernels run (no counterpart in the paper: launch-shape knobs of this
+ * implementation, used by its benchmarks and tests).  Zero in every field means "library default" (AUTO: the bulk-copy
  * kernel for slots in device memory, the vector kernel with 16 persistent blocks for slots in
  * mapped host memory; chunk-major order). */
 typedef enum {
     KVC_VARIANT_AUTO = 0,
     KVC_VARIANT_VEC = 1,  /* 16- or 32-byte vector loads/stores through registers */
-    KVC_VARIANT_BULK = 2  /* bulk async copies global->shared->global, one warp per thread block */
+    KVC_VARIANT_BULK = 2  /* bulk async copies global->shared->global, one warp per thread block;
+                             small slabs are moved several per work item (see kvc_tuning.group) */
 } kvc_variant;
 typedef enum {
     KVC_ORDER_AUTO = 0,
@@ -145,7 +157,15 @@ typedef struct {
     uint32_t pdl;        /* 0 = default (= 2), 1 = plain launches, 2 = programmatic dependent launch:
                             a kernel's blocks may be scheduled while the previous kernel of the
                             stream drains; they wait for its completion before reading memory */
+    uint32_t group;      /* BULK: slabs per work item.  0 = default: when a slab is at most half a
+                            tile, as many whole slabs as fit one tile (a power of two, at most 32)
+                            -- consecutive slabs of a chunk are contiguous in the slot, so one item
+                            is several copies on the pool side and one on the slot side;
+                            1 = one slab (or one tile of a slab) per item; N > 1 = at most N.
+                            Adding KVC_GROUP_FORCE_KERNEL runs the multi-slab kernel even when that
+                            leaves one slab per item (for same-process comparisons) */
 } kvc_tuning;
+#define KVC_GROUP_FORCE_KERNEL 0x100u
 /* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */
 kvc_status kvc_layout_set_tuning(kvc_layout *layout, const kvc_tuning *tuning);
 
@@ -214,7 +234,8 @@ kvc_status kvc_pack_batch(kvc_layout *layout, const kvc_chunk_op *ops, uint32_t 
 kvc_status kvc_unpack_batch(kvc_layout *layout, const kvc_chunk_op *ops, uint32_t n_ops,
                             int ids_on_device, void *stream);
 
-/* Waits for `stream`, then reports and clears the handle's device-side counters:
+/* No counterpart in the paper: the kernels' own health report.
+ * Waits for `stream`, then reports and clears the handle's device-side counters:
  * *n_skipped = blocks skipped because a device-resident id was out of range,
  * *n_wait_expired = bounded waits inside a kernel that gave up (should be 0).
  * Either pointer may be NULL. */
@@ -228,21 +249,31 @@ kvc_status kvc_poll_device_status(kvc_layout *layout, void *stream, uint32_t *n_
  * through this call: it allocates and frees nothing, on the device or on the host, and neither
  * does anything it calls.  Same result as kvc_pack_batch with ids_on_device == 0 (ids must be in
  * HOST memory; they are fully validated before anything is enqueued).
- * The id table, the plane-pointer table and the status words live in a fixed array inside the
+ * The id table, the plane-pointer table and two status counters live in a fixed array inside the
  * library image (about 264 KiB of device memory on every GPU that loads the library, held until
  * the process exits).  Limits: at most KVC_STATIC_MAX_BLOCKS blocks per call, summed over the
  * ops, and at most KVC_STATIC_MAX_PLANES planes for layouts given as plane pointers; beyond
  * either the call returns KVC_ERR_TOO_LARGE and enqueues nothing.
+ * The tables travel to the device inside the parameters of small kernels enqueued on `stream`
+ * ahead of the copy kernel (one per 32 KiB of table: 1 to 9 launches), so the call does not wait
+ * for the stream and the host arrays may be reused as soon as it returns.
  * The first call on a device looks up the array's device address and the device's limits; make
  * that first call outside any stream capture.  Every call shares the one array, which keeps the
- * previous call's contents (the call clears what must start at zero): calls whose GPU work can
- * overlap -- different streams, or several host threads -- race on it, so serialise them on
- * one stream.  The handle's device status counters are not touched by this call.
+ * previous call's contents: calls whose GPU work can overlap -- different streams -- race on it,
+ * so keep them on one stream (back-to-back calls on one stream need no synchronisation between
+ * them).  Host-side the call is serialised by a lock.  The handle's own device status counters are
+ * not touched; this path has its own pair, read with kvc_poll_static_status.
+ * If the handle has launched before, the device it belongs to must be current (INVALID_ARG).
  * Errors: INVALID_ARG, ALIGNMENT, OUT_OF_RANGE, TOO_LARGE, CUDA. */
 #define KVC_STATIC_MAX_BLOCKS 8192u
 #define KVC_STATIC_MAX_PLANES 1024u
 kvc_status kvc_pack_batch_static(kvc_layout *layout, const kvc_chunk_op *ops, uint32_t n_ops,
                                  void *stream);
+/* kvc_poll_device_status for the kvc_pack_batch_static path of the current device (no counterpart
+ * in the paper).  Waits for `stream`, reports and clears the two counters kept in the fixed array:
+ * blocks skipped for a bad id (always 0 here, ids are validated on the host) and bounded in-kernel
+ * waits that gave up (should be 0; non-zero means a pack did not complete).  Allocates nothing. */
+kvc_status kvc_poll_static_status(void *stream, uint32_t *n_skipped, uint32_t *n_wait_expired);
 
 /* Copy-engine variants (the paper's own mechanism, Sec. 6.2 / 6.4: a DMA-based batched block
  * copy between the KV tensors and pinned staging slots; Sec. 5.1 contrasts it with kernel copies).
@@ -258,7 +289,8 @@ kvc_status kvc_pack_copy_engine(kvc_layout *layout, const int32_t *ids, uint32_t
 kvc_status kvc_unpack_copy_engine(kvc_layout *layout, const void *src, uint64_t src_bytes,
                                   const int32_t *ids, uint32_t n_blocks, void *stream);
 
-/* Number of kernel launches issued through this handle so far. */
+/* Number of kernel launches issued through this handle so far (no counterpart in the paper;
+ * the benchmark reports it so that a run that launched nothing cannot pass for a GPU run). */
 uint64_t kvc_layout_launch_count(const kvc_layout *layout);
 
 /* ------------------------------------------------------------------ staging ring (Sec. 6.4) */
@@ -350,6 +382,11 @@ kvc_status kvc_store_publish(kvc_store *store, uint64_t hash, const void *host_b
 /* Reads exactly `bytes`; INVALID_ARG if the entry has another size.  Errors: NOT_FOUND, IO. */
 kvc_status kvc_store_read(kvc_store *store, uint64_t hash, void *host_buf, uint64_t bytes);
 int kvc_store_direct_io_refused(const kvc_store *store);
+/* Test seam (no counterpart in the paper): every file the store opens goes through `fn`
+ * (path, open(2) flags, mode; returns a descriptor or -1 with errno set).  NULL restores open(2).
+ * Process-wide.  Lets a host test play a file system that refuses O_DIRECT. */
+typedef int (*kvc_open_fn)(const char *path, int flags, unsigned mode);
+kvc_status kvc_store_set_open_fn(kvc_open_fn fn);
 
 /* Prefix-hash chaining (Sec. 2.1): the hash of a block covers its tokens and the hash of the
  * block before it, so two requests share an entry only if they agree from the first token on.
@@ -402,7 +439,7 @@ kvc_status kvc_pipeline_load(kvc_layout *layout, kvc_ring *ring, kvc_store *stor
  * `max_speculative` preloads are in flight (0 = no limit); requests for a key (chunk hash) that
  * already holds a slot join it (reference count) instead of reading again, and a demand request
  * joining a preload claims it; with no free slot, foreground work takes over the least recently
- * used retained slot, else a staged preload nobody claimed; an unclaimed preload in flight can be
+ * used retained slot, else a staged preload nobody claimed or still holds; an unclaimed preload in flight can be
  * cancelled; with retain_completed != 0 released staged slots stay as a cache until taken over.
  * Not thread-safe. */
 typedef struct kvc_slot_pool kvc_slot_pool;
@@ -430,12 +467,15 @@ kvc_status kvc_slot_pool_mark_staged(kvc_slot_pool *pool, uint32_t slot);
 /* Drops one reference.  At zero the slot is freed -- or, if staged, kept: as a cache entry when
  * retention is on, or as a finished preload waiting to be claimed. */
 kvc_status kvc_slot_pool_release(kvc_slot_pool *pool, uint32_t slot);
-/* Gives up an unclaimed preload that is still in flight (its read is abandoned and requeued by the
- * caller).  STATE for anything else. */
+/* Gives up an unclaimed preload that is still in flight and has a single holder (its read is
+ * abandoned and requeued by the caller).  STATE for anything else, including a preload that other
+ * preload candidates have joined. */
 kvc_status kvc_slot_pool_cancel(kvc_slot_pool *pool, uint32_t slot);
 kvc_status kvc_slot_pool_get_counters(const kvc_slot_pool *pool, kvc_slot_pool_counters *out);
 
-/* Event provider used by a ring.  The default one wraps CUDA events.  Tests replace it to
+/* Event provider used by a ring (test seam, no counterpart in the paper; the paper's rule it
+ * serves is Sec. 6.4's "a slot is reused only after its CUDA event has completed").
+ * The default one wraps CUDA events.  Tests replace it to
  * drive the slot state machine on a machine without a GPU (events that complete on command);
  * it must be installed before the ring is created and applies to rings created afterwards.
  * Passing NULL restores the CUDA provider. */

@@ -1,8 +1,8 @@
 // Copy-engine variants of pack / unpack: the same byte movement expressed as strided asynchronous
 // memory copies, so that the GPU's DMA engines do the work and no SM is used.  This is how the
 // paper's own system moves blocks (Sec. 6.2, 6.4: a DMA-based batched block copy between the KV
-// tensors and pinned staging slots; Sec. 5.1 contrasts it with kernel copies, which "consume GPU
-// compute resources").  It exists here to put numbers on that trade-off next to the kernels.
+// tensors and pinned staging slots; Sec. 5.1 contrasts it with kernel copies, which take SM time
+// away from the model).  It exists here to put numbers on that trade-off next to the kernels.
 //
 // One 2-D copy moves one block: its L*P slabs are `plane pitch` apart in the pool and
 // nb_c * S apart in the chunk, so pool -> chunk is a copy of L*P rows of S bytes.  When the planes

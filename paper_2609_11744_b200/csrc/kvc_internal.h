@@ -27,6 +27,12 @@
 #define KVC_BULK_STREAMING_BLOCKS_PER_SM 2u
 #define KVC_BULK_STREAMING_STAGES 2u
 #define KVC_BULK_SMEM_HEADER 1024u  // mbarriers + per-stage bookkeeping ahead of the data stages
+// Multi-slab kernel: a work item is a run of up to 32 consecutive slabs (a power of two), at most
+// one tile in total.  Its shared-memory header holds the mbarriers (128 bytes) and, per stage, the
+// address and length of up to 32 stores (384 bytes), rounded up to 128 bytes.
+#define KVC_GROUP_MAX_SLABS 32u
+#define KVC_GROUP_STAGE_INFO_BYTES 384u
+#define KVC_GROUP_SMEM_HEADER(stages) ((128u + (stages) * KVC_GROUP_STAGE_INFO_BYTES + 127u) & ~127u)
 #define KVC_WAIT_LIMIT (1u << 22)   // polls of an mbarrier before a kernel gives up
 
 // Where the planes of the paged pool live (kernel-side copy of the layout).
@@ -71,12 +77,16 @@ struct KvcLaunch {
     uint32_t lag;             // bulk kernels: loads issued ahead of the store they feed
     uint32_t l2_evict_first;  // bulk kernels: attach an evict-first L2 policy to the copies
     uint32_t pdl;             // launch with programmatic stream serialisation
+    uint32_t group_shift;     // multi-slab kernel: log2 of the slabs per work item
+    uint32_t pending;         // bulk kernels: stores that may still read shared memory at a stage reuse
+    uint64_t n_slabs;         // multi-slab kernel: n_ent * LP
     int32_t ids[KVC_PARAM_IDS];
 };
 
 enum { KVC_DIR_PACK = 0, KVC_DIR_UNPACK = 1 };
-// Internal refinement of KVC_VARIANT_VEC: 32-byte vectors when everything is 32-byte aligned.
-enum { KVC_VARIANT_VEC32 = 100 };
+// Internal refinements: 32-byte vectors when everything is 32-byte aligned; the bulk kernel whose
+// work items span several slabs.
+enum { KVC_VARIANT_VEC32 = 100, KVC_VARIANT_BULK_GROUP = 101 };
 
 // Implemented in kvc_kernels.cu.
 cudaError_t kvc_launch_copy(int dir, int variant, const KvcLaunch &a, uint32_t grid,

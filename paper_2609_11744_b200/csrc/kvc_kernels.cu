@@ -20,8 +20,12 @@
 // A block handles items blockIdx.x, blockIdx.x + gridDim.x, ...: with a large grid
 // every block takes a couple of items and retires (the default), with a small one
 // the blocks persist and stride over everything.
-// No cluster, no multicast: every byte is read exactly once by exactly one SM.
+// Every byte is read exactly once by exactly one SM, so blocks never share tiles: no thread-block
+// clusters are launched and every copy is addressed to the issuing block's own shared memory.
 #include <string.h>
+
+#include <atomic>
+#include <mutex>
 
 #include "kvc_internal.h"
 
@@ -122,7 +126,10 @@ __device__ __forceinline__ void grid_dependency_wait()
 
 // A VB-byte vector held in registers.  VB = 32 uses the 256-bit global accesses of sm_100,
 // which also accept an L2 evict-first priority (the data is touched once); VB = 16 is the
-// path for layouts that are only 16-byte aligned.
+// path for layouts that are only 16-byte aligned.  The loads are ordinary coherent loads, not
+// the read-only (.nc) form: with programmatic dependent launch a grid can be resident while an
+// earlier grid of the stream is still writing the same pool blocks, and the read-only path
+// promises nothing about data that changes during the kernel's lifetime.
 template <int VB>
 struct Vec;
 
@@ -131,7 +138,7 @@ struct Vec<16> {
     uint32_t r[4];
     __device__ __forceinline__ void load(uint64_t addr)
     {
-        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+        asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
                      : "l"(addr));
     }
@@ -149,7 +156,7 @@ struct Vec<32> {
     __device__ __forceinline__ void load(uint64_t addr)
     {
         asm volatile(
-            "ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+            "ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
             : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
               "=r"(r[7])
             : "l"(addr));
@@ -252,7 +259,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst_smem, uint64_t src, uint3
                                           uint32_t bar)
 {
     asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
+        "cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::
             "r"(dst_smem),
         "l"(src), "r"(bytes), "r"(bar)
         : "memory");
@@ -276,7 +283,7 @@ __device__ __forceinline__ void bulk_load_hint(uint32_t dst_smem, uint64_t src, 
                                                uint32_t bar, uint64_t pol)
 {
     asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "cp.async.bulk.shared::cta.global.mbarrier::complete_tx::bytes.L2::cache_hint "
         "[%0], [%1], %2, [%3], %4;" ::"r"(dst_smem),
         "l"(src), "r"(bytes), "r"(bar), "l"(pol)
         : "memory");
@@ -301,6 +308,21 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read()
 {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+
+// The instruction takes an immediate; the launch picks how many stores may stay outstanding.
+__device__ __forceinline__ void bulk_wait_read_n(uint32_t n)
+{
+    switch (n) {
+    case 0: bulk_wait_read<0>(); break;
+    case 1: bulk_wait_read<1>(); break;
+    case 2: bulk_wait_read<2>(); break;
+    case 3: bulk_wait_read<3>(); break;
+    case 4: bulk_wait_read<4>(); break;
+    case 5: bulk_wait_read<5>(); break;
+    case 6: bulk_wait_read<6>(); break;
+    default: bulk_wait_read<7>(); break;
+    }
 }
 
 __device__ __forceinline__ void bulk_wait_all()
@@ -414,6 +436,152 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
     }
 }
 
+
+// ------------------------------------------------------------------------------------ BULK, several slabs per item
+//
+// For slabs much smaller than a tile the per-item cost of the kernel above (decode, one mbarrier
+// round trip, one bulk group) is paid per slab and the throughput falls with the slab size.  Here
+// a work item is a run of k = 2^group_shift consecutive slabs in the order the chunk's bytes lie
+// in the slot -- at most one tile.  Consecutive slabs of a chunk are contiguous on the slot side
+// (both chunk byte orders), so an item is k copies on the pool side and ONE copy on the slot side
+// (two where the run crosses into the next chunk; contiguity is detected from the addresses, so
+// any traversal order stays correct).  The k lanes of a segment of the warp each decode one slab
+// and issue their own pool-side copy; all completions of an item count, in bytes, on the stage's
+// one mbarrier.  Every lane commits one bulk group per item, issued or not, so group counts are
+// the same on all lanes and one wait_group.read per lane orders the whole warp's stage reuse.
+struct GroupStageInfo {
+    uint64_t dst[KVC_GROUP_MAX_SLABS];  // where the stage's stores go
+    uint32_t len[KVC_GROUP_MAX_SLABS];  // bytes of each (0 = none)
+};
+static_assert(sizeof(GroupStageInfo) == KVC_GROUP_STAGE_INFO_BYTES, "shared-memory header layout");
+
+template <int DIR, bool TABLE>
+__global__ void __launch_bounds__(KVC_BULK_THREADS, 1)
+kvc_bulk_group_kernel(const __grid_constant__ KvcLaunch a)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem);                       // [stages]
+    GroupStageInfo *info = reinterpret_cast<GroupStageInfo *>(smem + 128);     // [stages]
+    constexpr uint32_t FULL = 0xffffffffu;
+
+    const uint32_t lane = threadIdx.x;
+    const uint32_t stages = a.stages, lag = a.lag, tile = a.g.tile_bytes, S = a.g.slab_bytes;
+    const uint32_t ksh = a.group_shift, k = 1u << ksh;
+    const uint32_t n_items = (uint32_t)a.n_items;
+    const uint64_t n_slabs = a.n_slabs;
+    unsigned char *data = smem + KVC_GROUP_SMEM_HEADER(stages);
+    if (blockIdx.x >= n_items) {
+        grid_dependency_wait();
+        return;
+    }
+    const uint32_t K = (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x;  // my items
+
+    if (lane == 0) {
+        for (uint32_t s = 0; s < stages; ++s)
+            mbar_init(smem_u32(&bars[s]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    grid_dependency_wait();
+    __syncwarp();
+
+    const uint32_t per_round = 32u >> ksh;          // items decoded per round
+    const uint32_t seg = lane >> ksh, sub = lane & (k - 1u);
+    bool ok = true;                                  // no wait has expired (same on all lanes)
+    uint32_t loads_done = 0, stores_done = 0;
+    Item mine;
+    mine.pool = mine.slot = 0;
+    mine.len = 0;
+    for (uint32_t k0 = 0; k0 < K + lag; k0 += per_round) {
+        // lane (seg, sub) decodes slab `sub` of this block's item k0 + seg
+        mine.len = 0;
+        if (k0 + seg < K) {
+            const uint64_t r = (((uint64_t)blockIdx.x + (uint64_t)(k0 + seg) * gridDim.x) << ksh) + sub;
+            if (r < n_slabs)
+                mine = decode<TABLE>(a, (uint32_t)r, true);
+        }
+        for (uint32_t m = 0; m < per_round; ++m) {
+            const uint32_t step = k0 + m;
+            if (step >= K + lag)
+                break;
+            if (ok && step < K) {
+                const uint32_t s = step % stages;
+                if (step >= stages)
+                    bulk_wait_read_n(a.pending);  // the stores that last drained stage s have left it
+                __syncwarp();
+                const bool active = seg == m;
+                const bool valid = active && mine.len != 0;
+                // runs of slabs that are contiguous on the slot side
+                const uint64_t prev_slot = __shfl_up_sync(FULL, mine.slot, 1);
+                const uint32_t prev_len = __shfl_up_sync(FULL, mine.len, 1);
+                const bool head = valid && (sub == 0 || prev_len == 0 || prev_slot + prev_len != mine.slot);
+                const uint32_t vmask = __ballot_sync(FULL, valid);
+                const uint32_t hmask = __ballot_sync(FULL, head);
+                const uint32_t seg_lo = m << ksh;
+                const uint32_t segmask = k == 32u ? FULL : (((1u << k) - 1u) << seg_lo);
+                uint32_t run = 0;  // bytes of the merged copy this lane heads
+                if (head) {
+                    const uint32_t bound = (hmask | ~vmask) & segmask;
+                    const uint32_t above = lane == 31u ? 0u : (bound & (FULL << (lane + 1u)));
+                    const uint32_t next = above ? (uint32_t)__ffs((int)above) - 1u : seg_lo + k;
+                    run = (next - lane) * S;
+                }
+                const uint32_t bar = smem_u32(&bars[s]);
+                if (active && sub == 0)
+                    mbar_expect_tx(bar, (uint32_t)__popc(vmask) * S);
+                __syncwarp();
+                const uint32_t stage_at = smem_u32(data + (size_t)s * tile + (size_t)sub * S);
+                if (DIR == KVC_DIR_PACK) {
+                    if (valid)
+                        bulk_load(stage_at, mine.pool, S, bar);
+                    if (active) {
+                        info[s].dst[sub] = mine.slot;
+                        info[s].len[sub] = run;
+                    }
+                } else {
+                    if (head)
+                        bulk_load(stage_at, mine.slot, run, bar);
+                    if (active) {
+                        info[s].dst[sub] = mine.pool;
+                        info[s].len[sub] = valid ? S : 0u;
+                    }
+                }
+                loads_done = step + 1;
+            }
+            if (ok && step >= lag) {
+                const uint32_t mm = step - lag;
+                const uint32_t s = mm % stages;
+                __syncwarp();
+                const bool done =
+                    __all_sync(FULL, mbar_wait(smem_u32(&bars[s]), (mm / stages) & 1u));
+                if (done) {
+                    if (lane < k) {
+                        const uint32_t len = info[s].len[lane];
+                        if (len) {
+                            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                            bulk_store(info[s].dst[lane],
+                                       smem_u32(data + (size_t)s * tile + (size_t)lane * S), len);
+                        }
+                    }
+                    bulk_commit();
+                    stores_done = mm + 1;
+                } else {
+                    ok = false;
+                    if (lane == 0)
+                        atomicAdd(a.status + 1, 1u);
+                }
+            }
+        }
+    }
+    if (!ok) {
+        // A wait gave up.  Loads that were issued may still land in shared memory: give each one
+        // more bounded wait so the block does not retire under an incoming copy.
+        for (uint32_t m = stores_done; m < loads_done; ++m)
+            (void)mbar_wait(smem_u32(&bars[m % stages]), (m / stages) & 1u);
+    }
+    bulk_wait_all();
+}
+
 template <typename K>
 cudaError_t launch_cfg(K kernel, const KvcLaunch &a, uint32_t grid, uint32_t block, uint32_t smem,
                        cudaStream_t stream)
@@ -431,27 +599,48 @@ cudaError_t launch_cfg(K kernel, const KvcLaunch &a, uint32_t grid, uint32_t blo
     return cudaLaunchKernelEx(&cfg, kernel, a);
 }
 
+// The opt-in dynamic shared-memory size is a per-device attribute of each kernel and is only
+// ever raised.  Handles on different host threads may make their first launches at the same
+// time with different tunings: the raise happens under a lock, the common case is one atomic load.
+template <typename K>
+cudaError_t ensure_smem(K kernel, int which, uint32_t smem)
+{
+    static std::atomic<int> configured[64][8];
+    static std::mutex mu;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess)
+        return e;
+    if (dev < 0 || dev >= 64)
+        return cudaErrorInvalidDevice;
+    std::atomic<int> &have = configured[dev][which];
+    if ((int)smem <= have.load(std::memory_order_acquire))
+        return cudaSuccess;
+    std::lock_guard<std::mutex> lock(mu);
+    if ((int)smem > have.load(std::memory_order_relaxed)) {
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess)
+            return e;
+        have.store((int)smem, std::memory_order_release);
+    }
+    return cudaSuccess;
+}
+
 template <int DIR, bool TABLE>
 cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t smem,
                        cudaStream_t stream)
 {
     if (variant == KVC_VARIANT_BULK) {
-        // the opt-in shared-memory size is a per-device attribute of the kernel
-        static int configured_smem[64][2][2];
-        int dev = 0;
-        cudaError_t e = cudaGetDevice(&dev);
+        cudaError_t e = ensure_smem(kvc_bulk_kernel<DIR, TABLE>, DIR * 2 + (TABLE ? 1 : 0), smem);
         if (e != cudaSuccess)
             return e;
-        if (dev < 0 || dev >= 64)
-            return cudaErrorInvalidDevice;
-        if ((int)smem > configured_smem[dev][DIR][TABLE]) {
-            e = cudaFuncSetAttribute(kvc_bulk_kernel<DIR, TABLE>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-            if (e != cudaSuccess)
-                return e;
-            configured_smem[dev][DIR][TABLE] = (int)smem;
-        }
         return launch_cfg(kvc_bulk_kernel<DIR, TABLE>, a, grid, KVC_BULK_THREADS, smem, stream);
+    }
+    if (variant == KVC_VARIANT_BULK_GROUP) {
+        cudaError_t e = ensure_smem(kvc_bulk_group_kernel<DIR, TABLE>, 4 + DIR * 2 + (TABLE ? 1 : 0), smem);
+        if (e != cudaSuccess)
+            return e;
+        return launch_cfg(kvc_bulk_group_kernel<DIR, TABLE>, a, grid, KVC_BULK_THREADS, smem, stream);
     }
     const bool warp_team = a.g.tile_bytes <= KVC_VEC_WARP_TEAM_MAX_TILE;
     if (variant == KVC_VARIANT_VEC32)

@@ -97,25 +97,48 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     if (tile == 0)
         tile = (variant == KVC_VARIANT_BULK || !persistent) ? 32768u : 16384u;
     tile = (uint32_t)std::min<uint64_t>(tile, lay->slab_bytes);
-    uint32_t stages = 0, lag = 0, smem = 0;
+    uint32_t stages = 0, lag = 0, smem = 0, group_shift = 0;
     if (variant == KVC_VARIANT_BULK) {
         const uint32_t per_sm = t.ctas_per_sm ? t.ctas_per_sm
                                               : (persistent ? 1u : KVC_BULK_STREAMING_BLOCKS_PER_SM);
         // every resident block also costs 1 KiB of system-reserved shared memory
-        const uint32_t room = ((uint32_t)lay->max_smem_optin + 1024u) / per_sm - 1024u - KVC_BULK_SMEM_HEADER;
+        // (the larger header of the multi-slab kernel is assumed for either kernel)
+        const uint32_t room = ((uint32_t)lay->max_smem_optin + 1024u) / per_sm - 1024u -
+                              KVC_GROUP_SMEM_HEADER(KVC_BULK_MAX_STAGES);
         if (tile > room / 2)
             tile = (room / 2) & ~15u;
-        stages = t.stages ? t.stages : (persistent ? KVC_BULK_DEFAULT_STAGES : KVC_BULK_STREAMING_STAGES);
+        // Several slabs per work item: the largest power of two of whole slabs that fits the tile.
+        const uint32_t tile_cap = std::min<uint32_t>(t.tile_bytes ? t.tile_bytes : 32768u, (room / 2) & ~15u);
+        const uint32_t want_group = t.group & ~KVC_GROUP_FORCE_KERNEL;
+        uint32_t group = 1;
+        if (want_group != 1 && lay->slab_bytes <= tile_cap) {
+            const uint32_t cap = std::min<uint32_t>(want_group ? want_group : KVC_GROUP_MAX_SLABS,
+                                                    (uint32_t)(tile_cap / lay->slab_bytes));
+            while (group * 2 <= cap) {
+                group *= 2;
+                ++group_shift;
+            }
+        }
+        const bool grouped = (group > 1 || (t.group & KVC_GROUP_FORCE_KERNEL)) && lay->slab_bytes <= tile_cap;
+        if (grouped) {
+            variant = KVC_VARIANT_BULK_GROUP;
+            tile = group * (uint32_t)lay->slab_bytes;
+        }
+        uint32_t def_stages = persistent ? KVC_BULK_DEFAULT_STAGES : KVC_BULK_STREAMING_STAGES;
+        if (grouped && tile < 32768u)   // smaller items: more of them in flight for the same bytes
+            def_stages = std::max<uint32_t>(def_stages, std::min<uint32_t>(65536u / tile, 8u));
+        stages = t.stages ? t.stages : def_stages;
         stages = std::min<uint32_t>(std::min<uint32_t>(stages, room / tile), KVC_BULK_MAX_STAGES);
         if (stages < 2)
             return KVC_ERR_INVALID_ARG;
-        // a stage is reloaded only when at most one newer store still reads shared memory, so
-        // loads can run at most stages-2 items ahead of the stores
+        // a stage is reloaded only when at most `pending` newer stores still read shared memory,
+        // so loads can run at most stages-2 items ahead of the stores
         lag = stages - 2;
-        const uint32_t want_lag = t.lag ? t.lag : KVC_BULK_DEFAULT_LAG;
+        const uint32_t want_lag = t.lag ? t.lag
+                                        : (grouped ? std::max<uint32_t>(1u, stages / 2 - 1) : KVC_BULK_DEFAULT_LAG);
         if (want_lag < lag)
             lag = want_lag;
-        smem = KVC_BULK_SMEM_HEADER + stages * tile;
+        smem = (grouped ? KVC_GROUP_SMEM_HEADER(stages) : KVC_BULK_SMEM_HEADER) + stages * tile;
     } else {
         // 32-byte vectors need every address the kernel forms to be 32-byte aligned
         bool a32 = (lay->slab_bytes % 32 == 0) && (tile % 32 == 0) && (lay->block_stride % 32 == 0) &&
@@ -130,10 +153,17 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
         variant = a32 ? (int)KVC_VARIANT_VEC32 : (int)KVC_VARIANT_VEC;
     }
     g.tile_bytes = tile;
-    g.parts = (uint32_t)((lay->slab_bytes + tile - 1) / tile);
-    const uint64_t n_items = n_ent * lay->planes_total * g.parts;
-    if (n_items == 0 || n_items > 0xFFFFFFFFull)
+    const bool grouped = variant == KVC_VARIANT_BULK_GROUP;
+    g.parts = grouped ? 1u : (uint32_t)((lay->slab_bytes + tile - 1) / tile);
+    const uint64_t n_slabs = n_ent * lay->planes_total;
+    const uint64_t n_items = grouped ? (n_slabs + (1u << group_shift) - 1) >> group_shift : n_slabs * g.parts;
+    if (n_items == 0 || n_items > 0xFFFFFFFFull || n_slabs > 0xFFFFFFFFull)
         return KVC_ERR_INVALID_ARG;
+    a->n_slabs = n_slabs;
+    a->group_shift = group_shift;
+    // stores that may still be reading shared memory when a stage is reloaded: the stage's last
+    // store is stages-lag groups back, so everything newer than that may stay outstanding
+    a->pending = stages >= 2 + lag ? std::min<uint32_t>(stages - 1 - lag, 7u) : 1u;
     a->n_items = n_items;
     a->n_ent = (uint32_t)n_ent;
     a->order = t.order ? t.order : KVC_ORDER_CHUNK_MAJOR;
@@ -154,8 +184,9 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
         // streaming: about 64 KiB (bulk) or 32 KiB (vector) of items per block
         uint32_t per_block = t.items_per_cta;
         if (per_block == 0) {
-            const uint32_t bytes = variant == KVC_VARIANT_BULK ? 65536u : 32768u;
-            per_block = std::max<uint32_t>(variant == KVC_VARIANT_BULK ? 2u : 1u, bytes / tile);
+            const bool bulk = variant == KVC_VARIANT_BULK || variant == KVC_VARIANT_BULK_GROUP;
+            const uint32_t bytes = bulk ? 65536u : 32768u;
+            per_block = std::max<uint32_t>(bulk ? 2u : 1u, bytes / tile);
         }
         grid = (n_items + per_block - 1) / per_block;
     }
@@ -402,6 +433,38 @@ const char *kvc_status_str(kvc_status s)
     return "unknown status";
 }
 
+kvc_status kvc_layout_desc_init_dense(kvc_layout_desc *d, const void *base, uint32_t num_layers,
+                                      uint32_t kv_planes, uint32_t num_blocks, uint32_t block_size,
+                                      uint32_t num_kv_heads, uint32_t head_dim, uint32_t elem_bytes,
+                                      uint32_t chunk_tokens, uint32_t chunk_order)
+{
+    if (!d)
+        return KVC_ERR_INVALID_ARG;
+    memset(d, 0, sizeof(*d));
+    d->num_layers = num_layers;
+    d->kv_planes = kv_planes;
+    d->num_blocks = num_blocks;
+    d->block_size = block_size;
+    d->num_kv_heads = num_kv_heads;
+    d->head_dim = head_dim;
+    d->elem_bytes = elem_bytes;
+    d->chunk_tokens = chunk_tokens;
+    d->chunk_order = chunk_order;
+    d->base = base;
+    // slab = B*H*D*e, plane = NB*slab, layer = P*plane; every factor is < 2^32
+    unsigned __int128 slab = (unsigned __int128)block_size * num_kv_heads;
+    slab = slab * head_dim * elem_bytes;
+    const unsigned __int128 plane = slab * num_blocks;
+    const unsigned __int128 layer = plane * kv_planes;
+    const unsigned __int128 lim = ~(uint64_t)0;
+    if (slab > lim || plane > lim || layer > lim || layer * num_layers > lim)
+        return KVC_ERR_INVALID_ARG;
+    d->block_stride = (uint64_t)slab;
+    d->plane_stride = (uint64_t)plane;
+    d->layer_stride = (uint64_t)layer;
+    return KVC_OK;
+}
+
 kvc_status kvc_layout_create(const kvc_layout_desc *d, kvc_layout **out)
 {
     if (!d || !out)
@@ -545,6 +608,8 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
     if (t->stages == 1 || t->stages > KVC_BULK_MAX_STAGES)
         return KVC_ERR_INVALID_ARG;
     if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2 || t->items_per_cta > (1u << 20))
+        return KVC_ERR_INVALID_ARG;
+    if ((t->group & ~KVC_GROUP_FORCE_KERNEL) > KVC_GROUP_MAX_SLABS)
         return KVC_ERR_INVALID_ARG;
     lay->tuning = *t;
     return KVC_OK;

@@ -10,10 +10,20 @@
 // nothing is allocated or freed, by it or by anything it calls.
 //
 // The array lives in every device that loads the library until the process exits.  All calls
-// share it and it keeps the previous call's contents: the status words are cleared at the start
-// of every call, the tables are overwritten as far as the call needs them, and two calls whose
-// GPU work overlaps in time (different streams, or different host threads) race on it.
+// share it and it keeps the previous call's contents: the tables are overwritten as far as a
+// call needs them, the two status counters start at zero when the library is loaded and are
+// cleared by kvc_poll_static_status, and two calls whose GPU work overlaps in time (different
+// streams) race on it.
+//
+// The tables reach the device inside kernel parameters: a tiny kernel stores its own parameter
+// block into the array.  A launch copies its parameters before it returns, so the host-side
+// staging buffer can be refilled at once, the call never waits for the stream (an asynchronous
+// copy from pageable memory would: the runtime documents that it first synchronises the stream
+// and returns only when the bytes sit in a driver staging buffer), and no pinned buffer -- which
+// would have to be allocated -- is needed.
 #include <string.h>
+
+#include <mutex>
 
 #include "kvc_internal.h"
 
@@ -30,19 +40,37 @@ static_assert(kTableOffset % 256 == 0, "id table must stay 256-byte aligned");
 // cudaGetSymbolAddress below.
 static __device__ __align__(256) unsigned char kvc_static_scratch[kScratchBytes];
 
+// One parameter block: up to kUploadVecs 16-byte words for scratch[dst_off ...).  Kernel
+// parameters may be up to 32,764 bytes on this architecture.
+constexpr uint32_t kUploadVecs = 2032;
+struct UploadParams {
+    uint32_t dst_off;  // byte offset into the scratch array, multiple of 16
+    uint32_t n_vecs;
+    uint32_t pad[2];
+    uint4 data[kUploadVecs];
+};
+static_assert(sizeof(UploadParams) <= 32764, "parameter block too large");
+
+__global__ void __launch_bounds__(256) kvc_static_upload_kernel(const __grid_constant__ UploadParams p)
+{
+    uint4 *dst = reinterpret_cast<uint4 *>(kvc_static_scratch + p.dst_off);
+    for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < p.n_vecs; i += gridDim.x * blockDim.x)
+        dst[i] = p.data[i];
+}
+
 constexpr int kMaxDevices = 64;
 struct DeviceSetup {
     bool ready;
     unsigned char *scratch;  // device address of kvc_static_scratch on this device
     int sm_count, vec_blocks_per_sm, max_smem_optin;
 };
+// All host-side state of this file is guarded by one mutex; the call is far off any hot path.
+std::mutex g_mu;
 DeviceSetup g_setup[kMaxDevices];
+UploadParams g_params;        // host-side staging of one parameter block
+uint32_t g_host_status[2];    // landing place of kvc_poll_static_status
 
-// Host-side staging of the id table (plain static storage; pageable, so the runtime has copied
-// it out before cudaMemcpyAsync returns and the next call may overwrite it).
-KvcEnt g_host_table[KVC_STATIC_MAX_BLOCKS];
-
-// Once per device, with that device current.
+// Once per device, with that device current.  Caller holds g_mu.
 kvc_status setup_device(DeviceSetup **out)
 {
     int dev = -1;
@@ -69,6 +97,25 @@ kvc_status setup_device(DeviceSetup **out)
         d.ready = true;
     }
     *out = &d;
+    return KVC_OK;
+}
+
+// scratch[dst_off, dst_off + bytes) = src, through kernel parameters.  bytes % 16 == 0.
+kvc_status upload(uint32_t dst_off, const void *src, uint64_t bytes, cudaStream_t st)
+{
+    const unsigned char *p = static_cast<const unsigned char *>(src);
+    while (bytes) {
+        const uint32_t n = (uint32_t)(bytes < kUploadVecs * 16ull ? bytes : kUploadVecs * 16ull);
+        g_params.dst_off = dst_off;
+        g_params.n_vecs = n / 16;
+        memcpy(g_params.data, p, n);
+        kvc_static_upload_kernel<<<(g_params.n_vecs + 255) / 256, 256, 0, st>>>(g_params);
+        if (cudaGetLastError() != cudaSuccess)
+            return KVC_ERR_CUDA;
+        p += n;
+        dst_off += n;
+        bytes -= n;
+    }
     return KVC_OK;
 }
 
@@ -104,11 +151,16 @@ extern "C" kvc_status kvc_pack_batch_static(kvc_layout *lay, const kvc_chunk_op 
             if (ops[i].ids[j] < 0 || (uint32_t)ops[i].ids[j] >= lay->d.num_blocks)
                 return KVC_ERR_OUT_OF_RANGE;
 
+    std::lock_guard<std::mutex> lock(g_mu);
     DeviceSetup *dev = nullptr;
     kvc_status s = setup_device(&dev);
     if (s != KVC_OK)
         return s;
-    if (!lay->dev_ready) {
+    if (lay->dev_ready) {
+        // a handle belongs to the device of its first launch: its pool pointers mean nothing elsewhere
+        if (&g_setup[lay->device] != dev)
+            return KVC_ERR_INVALID_ARG;
+    } else {
         // the planner reads the device limits from the handle; fill them without allocating
         lay->sm_count = dev->sm_count;
         lay->vec_blocks_per_sm = dev->vec_blocks_per_sm;
@@ -121,39 +173,82 @@ extern "C" kvc_status kvc_pack_batch_static(kvc_layout *lay, const kvc_chunk_op 
     if (s != KVC_OK)
         return s;
 
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!lay->plane_ptrs.empty()) {
+        // 8-byte pointers, 16-byte words: an odd count carries one word of padding
+        static uint64_t planes[KVC_STATIC_MAX_PLANES + 1];
+        const size_t n = lay->plane_ptrs.size();
+        for (size_t i = 0; i < n; ++i)
+            planes[i] = (uint64_t)(uintptr_t)lay->plane_ptrs[i];
+        planes[n] = 0;
+        s = upload(kStatusBytes, planes, ((n + 1) / 2) * 16, st);
+        if (s != KVC_OK)
+            return s;
+    }
+    // the id table, one parameter block at a time
+    static KvcEnt ents[kUploadVecs / 2];
+    uint32_t filled = 0, base = 0;
     uint64_t k = 0;
     for (uint32_t i = 0; i < n_ops; ++i) {
         uint64_t ent_step, plane_step;
         kvc_chunk_steps(lay, ops[i].n_blocks, &ent_step, &plane_step);
         const uint32_t first = (uint32_t)k;
         for (uint32_t j = 0; j < ops[i].n_blocks; ++j, ++k) {
-            KvcEnt &e = g_host_table[k];
+            KvcEnt &e = ents[filled++];
             e.slot_addr = (uint64_t)(uintptr_t)ops[i].slot + (uint64_t)j * ent_step;
             e.id_or_ptr = (uint64_t)(uint32_t)ops[i].ids[j];
             e.plane_step = plane_step;
             e.nb_c = ops[i].n_blocks;
             e.first_ent = first;
+            if (filled == kUploadVecs / 2 || k + 1 == n_ent) {
+                s = upload(kTableOffset + base * (uint32_t)sizeof(KvcEnt), ents,
+                           (uint64_t)filled * sizeof(KvcEnt), st);
+                if (s != KVC_OK)
+                    return s;
+                base += filled;
+                filled = 0;
+            }
         }
     }
-    cudaStream_t st = (cudaStream_t)stream;
     unsigned char *scratch = dev->scratch;
-    // status words must start at zero; the tables are rewritten as far as this call reads them
-    if (cudaMemsetAsync(scratch, 0, kStatusBytes, st) != cudaSuccess)
-        return KVC_ERR_CUDA;
-    if (!lay->plane_ptrs.empty() &&
-        cudaMemcpyAsync(scratch + kStatusBytes, lay->plane_ptrs.data(),
-                        lay->plane_ptrs.size() * sizeof(void *), cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return KVC_ERR_CUDA;
-    if (cudaMemcpyAsync(scratch + kTableOffset, g_host_table, n_ent * sizeof(KvcEnt),
-                        cudaMemcpyHostToDevice, st) != cudaSuccess)
-        return KVC_ERR_CUDA;
     a.table = reinterpret_cast<const KvcEnt *>(scratch + kTableOffset);
     a.status = reinterpret_cast<uint32_t *>(scratch);
     a.g.plane_table = lay->plane_ptrs.empty()
                           ? nullptr
                           : reinterpret_cast<const unsigned char *const *>(scratch + kStatusBytes);
+    // The copy kernel reads the tables through the read-only data path, so it must not become
+    // resident while the upload kernels are still writing them: plain stream order, no
+    // programmatic overlap with the preceding kernel.
+    a.pdl = 0;
     if (kvc_launch_copy(KVC_DIR_PACK, plan.variant, a, plan.grid, plan.smem, st) != cudaSuccess)
         return KVC_ERR_CUDA;
     ++lay->launches;
+    return KVC_OK;
+}
+
+extern "C" kvc_status kvc_poll_static_status(void *stream, uint32_t *n_skipped, uint32_t *n_wait_expired)
+{
+    if (n_skipped)
+        *n_skipped = 0;
+    if (n_wait_expired)
+        *n_wait_expired = 0;
+    std::lock_guard<std::mutex> lock(g_mu);
+    DeviceSetup *dev = nullptr;
+    kvc_status s = setup_device(&dev);
+    if (s != KVC_OK)
+        return s;
+    cudaStream_t st = (cudaStream_t)stream;
+    // device -> pageable host: the runtime returns only when the bytes have arrived
+    if (cudaMemcpyAsync(g_host_status, dev->scratch, sizeof(g_host_status), cudaMemcpyDeviceToHost,
+                        st) != cudaSuccess ||
+        cudaMemsetAsync(dev->scratch, 0, sizeof(g_host_status), st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return KVC_ERR_CUDA;
+    }
+    if (n_skipped)
+        *n_skipped = g_host_status[0];
+    if (n_wait_expired)
+        *n_wait_expired = g_host_status[1];
     return KVC_OK;
 }

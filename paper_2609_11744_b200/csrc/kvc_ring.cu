@@ -2,6 +2,7 @@
 // slot returns to the pool only after the event recorded behind its last copy has completed.
 // Host bookkeeping plus two events per slot; no kernel, no device-wide synchronisation.
 #include <chrono>
+#include <mutex>
 #include <new>
 #include <thread>
 #include <vector>
@@ -43,6 +44,8 @@ int cu_sync(void *, void *ev) { return cudaEventSynchronize((cudaEvent_t)ev) == 
 
 const kvc_event_provider kCudaEvents = {nullptr, cu_create, cu_destroy, cu_record,
                                         cu_query, cu_stream_wait, cu_sync};
+// process-wide default for rings created from now on; rings copy it at creation
+std::mutex g_events_mu;
 kvc_event_provider g_events = kCudaEvents;
 bool g_events_custom = false;
 
@@ -114,15 +117,12 @@ extern "C" {
 
 kvc_status kvc_staging_ring_set_event_provider(const kvc_event_provider *p)
 {
-    if (!p) {
-        g_events = kCudaEvents;
-        g_events_custom = false;
-        return KVC_OK;
-    }
-    if (!p->create || !p->destroy || !p->record || !p->query || !p->stream_wait || !p->synchronize)
+    if (p && (!p->create || !p->destroy || !p->record || !p->query || !p->stream_wait ||
+              !p->synchronize))
         return KVC_ERR_INVALID_ARG;
-    g_events = *p;
-    g_events_custom = true;
+    std::lock_guard<std::mutex> lock(g_events_mu);
+    g_events = p ? *p : kCudaEvents;
+    g_events_custom = p != nullptr;
     return KVC_OK;
 }
 
@@ -148,8 +148,11 @@ kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ri
     kvc_ring *r = new (std::nothrow) kvc_ring();
     if (!r)
         return KVC_ERR_NOMEM;
-    r->ev = g_events;
-    r->custom_events = g_events_custom;
+    {
+        std::lock_guard<std::mutex> lock(g_events_mu);
+        r->ev = g_events;
+        r->custom_events = g_events_custom;
+    }
     r->kind = kind;
     r->slot_bytes = slot_bytes;
     r->n_slots = n_slots;
@@ -252,6 +255,10 @@ kvc_status kvc_staging_ring_acquire(kvc_ring *r, int64_t timeout_us, uint32_t *s
     const auto deadline =
         std::chrono::steady_clock::now() + std::chrono::microseconds(timeout_us);
     bool stall_logged = false;
+    // Polling a slot whose "drained" event has not completed yet: a few immediate retries (the
+    // event is often microseconds away), then sleeps that double from 2 to 20 microseconds, so a
+    // waiting thread does not burn a core while the host link drains a 32 MiB slot (~600 us).
+    uint32_t polls = 0, nap_us = 2;
     for (;;) {
         int q = slot_is_free(r, s);
         if (q < 0)
@@ -267,11 +274,15 @@ kvc_status kvc_staging_ring_acquire(kvc_ring *r, int64_t timeout_us, uint32_t *s
             return KVC_ERR_WOULD_BLOCK;
         if (std::chrono::steady_clock::now() >= deadline)
             return KVC_ERR_TIMEOUT;
-        if (s.state != SLOT_DRAINING)
+        if (s.state != SLOT_DRAINING) {
             // held by a producer or consumer of this same thread: only the caller can move it on
             std::this_thread::sleep_for(std::chrono::microseconds(50));
-        else
+        } else if (++polls <= 8) {
             std::this_thread::yield();
+        } else {
+            std::this_thread::sleep_for(std::chrono::microseconds(nap_us));
+            nap_us = nap_us * 2 > 20 ? 20 : nap_us * 2;
+        }
     }
     s.state = SLOT_ACQUIRED;
     *slot = r->head;

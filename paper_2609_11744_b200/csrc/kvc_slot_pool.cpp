@@ -161,7 +161,9 @@ kvc_status kvc_slot_pool_acquire(kvc_slot_pool *p, kvc_slot_class cls, uint64_t 
                 best = ~0ull;
                 for (uint32_t i = 0; i < p->slots.size(); ++i) {
                     const PSlot &s = p->slots[i];
-                    if (s.state == STAGED && s.speculative && s.stamp < best) {
+                    // refs == 0: the preloader has let go of it and nobody joined; a staged preload
+                    // that is still referenced has I/O or a copy in progress on its slot
+                    if (s.state == STAGED && s.speculative && s.refs == 0 && s.stamp < best) {
                         best = s.stamp;
                         take = (int)i;
                     }
@@ -228,8 +230,10 @@ kvc_status kvc_slot_pool_cancel(kvc_slot_pool *p, uint32_t slot)
     if (!p || slot >= p->slots.size())
         return KVC_ERR_INVALID_ARG;
     PSlot &s = p->slots[slot];
-    if (s.state != IN_FLIGHT || !s.speculative)
-        return KVC_ERR_STATE;  // only an unclaimed preload still in flight can be cancelled
+    // only an unclaimed preload still in flight can be cancelled, and only by its sole holder:
+    // other preload candidates that joined it still expect the chunk to arrive in this slot
+    if (s.state != IN_FLIGHT || !s.speculative || s.refs != 1)
+        return KVC_ERR_STATE;
     forget(p, s);
     ++p->c.cancels;
     return KVC_OK;

@@ -65,17 +65,25 @@ bool direct_ok(const void *buf, uint64_t bytes)
     return ((uintptr_t)buf % 4096) == 0 && (bytes % 4096) == 0 && bytes > 0;
 }
 
+int plain_open(const char *path, int flags, unsigned mode) { return open(path, flags, (mode_t)mode); }
+std::atomic<kvc_open_fn> g_open{plain_open};
+
 // Opens with O_DIRECT when asked for and possible; falls back to buffered I/O when the file
-// system refuses the flag (tmpfs, some overlay file systems).
+// system refuses the flag (tmpfs, some overlay file systems).  A refused O_DIRECT open with
+// O_CREAT may already have created the (empty) file before failing: it is removed, or the
+// buffered retry with O_EXCL would find it and fail.
 int open_maybe_direct(kvc_store *st, const char *path, int flags, mode_t mode, bool direct)
 {
+    const kvc_open_fn do_open = g_open.load();
     if (direct) {
-        int fd = open(path, flags | O_DIRECT, mode);
+        int fd = do_open(path, flags | O_DIRECT, (unsigned)mode);
         if (fd >= 0 || errno != EINVAL)
             return fd;
         st->direct_refused.fetch_add(1);
+        if ((flags & (O_CREAT | O_EXCL)) == (O_CREAT | O_EXCL))
+            unlink(path);
     }
-    return open(path, flags, mode);
+    return do_open(path, flags, (unsigned)mode);
 }
 
 kvc_status write_all(int fd, const unsigned char *p, uint64_t n)
@@ -216,8 +224,10 @@ kvc_status kvc_store_publish(kvc_store *st, uint64_t hash, const void *host_buf,
     const std::string tmp = dir + tmp_name;
     const bool direct = st->want_direct && direct_ok(host_buf, bytes);
     int fd = open_maybe_direct(st, tmp.c_str(), O_WRONLY | O_CREAT | O_EXCL, 0666, direct);
-    if (fd < 0)
+    if (fd < 0) {
+        unlink(tmp.c_str());  // a failed create may still have left the name behind
         return KVC_ERR_IO;
+    }
     kvc_status rc = write_all(fd, static_cast<const unsigned char *>(host_buf), bytes);
     if (close(fd) != 0 && rc == KVC_OK)
         rc = KVC_ERR_IO;
@@ -253,5 +263,11 @@ kvc_status kvc_store_read(kvc_store *st, uint64_t hash, void *host_buf, uint64_t
 }
 
 int kvc_store_direct_io_refused(const kvc_store *st) { return st ? st->direct_refused.load() : 0; }
+
+kvc_status kvc_store_set_open_fn(kvc_open_fn fn)
+{
+    g_open.store(fn ? fn : plain_open);
+    return KVC_OK;
+}
 
 }  // extern "C"

@@ -28,6 +28,7 @@ KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR, KVC_ORDER_CHUNK_MA
 KVC_RING_DEVICE, KVC_RING_HOST_MAPPED = 0, 1
 KVC_CHUNK_LAYER_MAJOR, KVC_CHUNK_BLOCK_MAJOR = 0, 1
 KVC_MAP_FULL_CHUNKS_ONLY = 1
+KVC_GROUP_FORCE_KERNEL = 0x100
 
 
 class KvcError(RuntimeError):
@@ -54,7 +55,8 @@ class kvc_tuning(ctypes.Structure):
                 ("max_ctas", ctypes.c_uint32), ("tile_bytes", ctypes.c_uint32),
                 ("stages", ctypes.c_uint32), ("ctas_per_sm", ctypes.c_uint32),
                 ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32),
-                ("items_per_cta", ctypes.c_uint32), ("pdl", ctypes.c_uint32)]
+                ("items_per_cta", ctypes.c_uint32), ("pdl", ctypes.c_uint32),
+                ("group", ctypes.c_uint32)]
 
 
 class kvc_chunk_desc(ctypes.Structure):
@@ -115,6 +117,7 @@ def lib() -> ctypes.CDLL:
     sig = {
         "kvc_status_str": (ctypes.c_char_p, [ci]),
         "kvc_layout_create": (ci, [P(kvc_layout_desc), P(vp)]),
+        "kvc_layout_desc_init_dense": (ci, [P(kvc_layout_desc), vp] + [u32] * 9),
         "kvc_layout_destroy": (ci, [vp]),
         "kvc_layout_slab_bytes": (u64, [vp]),
         "kvc_layout_bytes_per_token": (u64, [vp]),
@@ -130,6 +133,7 @@ def lib() -> ctypes.CDLL:
         "kvc_pack_batch": (ci, [vp, vp, u32, ci, vp]),
         "kvc_unpack_batch": (ci, [vp, vp, u32, ci, vp]),
         "kvc_pack_batch_static": (ci, [vp, vp, u32, vp]),
+        "kvc_poll_static_status": (ci, [vp, P(u32), P(u32)]),
         "kvc_pack_copy_engine": (ci, [vp, vp, u32, vp, u64, vp]),
         "kvc_unpack_copy_engine": (ci, [vp, vp, u64, vp, u32, vp]),
         "kvc_poll_device_status": (ci, [vp, vp, P(u32), P(u32)]),
@@ -278,12 +282,16 @@ def kvc_layout_create(num_layers: int, kv_planes: int, num_blocks: int, block_si
 
 def kvc_layout_create_dense(pool, num_layers, kv_planes, num_blocks, block_size, num_kv_heads,
                             head_dim, elem_bytes, chunk_tokens, chunk_order: int = 0) -> LayoutHandle:
-    """Layout over one dense allocation [L][P][NB][B][H][D] (a tensor or a device address)."""
-    slab = block_size * num_kv_heads * head_dim * elem_bytes
-    plane = slab * num_blocks
-    return kvc_layout_create(num_layers, kv_planes, num_blocks, block_size, num_kv_heads, head_dim,
-                             elem_bytes, chunk_tokens, base=pool, layer_stride=plane * kv_planes,
-                             plane_stride=plane, chunk_order=chunk_order)
+    """Layout over one dense allocation [L][P][NB][B][H][D] (a tensor or a device address):
+    kvc_layout_desc_init_dense followed by kvc_layout_create."""
+    d = kvc_layout_desc()
+    _check(lib().kvc_layout_desc_init_dense(ctypes.byref(d), _ptr(pool), num_layers, kv_planes,
+                                            num_blocks, block_size, num_kv_heads, head_dim,
+                                            elem_bytes, chunk_tokens, chunk_order),
+           "kvc_layout_desc_init_dense")
+    out = ctypes.c_void_p()
+    _check(lib().kvc_layout_create(ctypes.byref(d), ctypes.byref(out)), "kvc_layout_create")
+    return LayoutHandle(out.value, [pool])
 
 
 def kvc_layout_destroy(layout: LayoutHandle) -> None:
@@ -313,9 +321,9 @@ def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
 
 
 def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
-                          ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, pdl=0) -> None:
+                          ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, pdl=0, group=0) -> None:
     t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag,
-                   items_per_cta, pdl)
+                   items_per_cta, pdl, group)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
 
 
@@ -437,6 +445,14 @@ def kvc_pack_batch_static(layout, ops: np.ndarray, stream=None) -> None:
         raise TypeError("ops must be a contiguous array of CHUNK_OP_DTYPE")
     _check(lib().kvc_pack_batch_static(layout.handle, ops.ctypes.data, len(ops), _stream(stream)),
            "kvc_pack_batch_static")
+
+
+def kvc_poll_static_status(stream=None) -> Tuple[int, int]:
+    """kvc_poll_device_status for the kvc_pack_batch_static path of the current device."""
+    a, b = ctypes.c_uint32(), ctypes.c_uint32()
+    _check(lib().kvc_poll_static_status(_stream(stream), ctypes.byref(a), ctypes.byref(b)),
+           "kvc_poll_static_status")
+    return a.value, b.value
 
 
 def kvc_poll_device_status(layout, stream=None) -> Tuple[int, int]:

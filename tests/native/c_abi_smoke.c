@@ -29,10 +29,11 @@ int main(void)
     }
     cudaMemcpy(d_pool, h_pool, pool_bytes, cudaMemcpyHostToDevice);
     kvc_layout_desc desc;
-    memset(&desc, 0, sizeof(desc));
-    desc.num_layers = L, desc.kv_planes = P, desc.num_blocks = NB, desc.block_size = B;
-    desc.num_kv_heads = H, desc.head_dim = D, desc.elem_bytes = e, desc.chunk_tokens = 16 * 16;
-    desc.base = d_pool, desc.layer_stride = plane * P, desc.plane_stride = plane;
+    CK(kvc_layout_desc_init_dense(&desc, d_pool, L, P, NB, B, H, D, e, 16 * 16, KVC_CHUNK_LAYER_MAJOR));
+    if (desc.plane_stride != plane || desc.layer_stride != plane * P || desc.block_stride != slab) {
+        printf("dense strides wrong\n");
+        return 1;
+    }
     kvc_layout *lay = NULL;
     CK(kvc_layout_create(&desc, &lay));
     int32_t ids[9] = {7, 39, 0, 12, 5, 21, 33, 2, 18}, dst[9] = {1, 3, 4, 6, 8, 9, 10, 11, 13};

@@ -1,0 +1,174 @@
+"""Pack / unpack beside other GPU work: the regime of Sec. 2.3 (stores deferred so that they
+overlap the next forward pass) and Sec. 5.1 (a kernel copy shares the GPU with the model).
+Default launches carry the programmatic-dependent-launch attribute and run on high-priority
+streams here while a low-priority stream keeps the tensor cores busy; every byte is then compared
+with the CPU oracle.  Also: kernels of one stream that read what the previous one wrote, and host
+threads whose handles make their first launches at the same moment."""
+import threading
+
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import oracle as orc
+from paper_2609_11744_b200 import cuda_rt, kvc
+import workloads as wl
+from test_gpu_parity import DEV, _pool_8b_384, dense_layout, dims_of, to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+def _gemm_load(stream, seconds=0.7):
+    """Enqueue a bounded bf16 matmul loop (under a second; few enough launches that the host is
+    not held up enqueueing them) on `stream`; returns a 'done' event."""
+    N = 8192
+    with torch.cuda.stream(stream):
+        a = torch.randn(N, N, device=DEV, dtype=torch.bfloat16)
+        b = torch.randn(N, N, device=DEV, dtype=torch.bfloat16)
+        c = torch.empty(N, N, device=DEV, dtype=torch.bfloat16)
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(20):
+            torch.matmul(a, b, out=c)
+        t1.record(stream)
+        t1.synchronize()
+        iters = int(min(900, max(20, seconds * 1e3 / (t0.elapsed_time(t1) / 20))))
+        for _ in range(iters):
+            torch.matmul(a, b, out=c)
+        done = torch.cuda.Event()
+        done.record(stream)
+    return done, (a, b, c)
+
+
+@pytest.mark.parametrize("kind", [kvc.KVC_RING_DEVICE, kvc.KVC_RING_HOST_MAPPED])
+@pytest.mark.parametrize("variant", [kvc.KVC_VARIANT_AUTO, kvc.KVC_VARIANT_VEC])
+def test_ring_streaming_stays_exact_beside_a_compute_stream(kind, variant):
+    """A 2048-token prefix (8 chunks) through a 3-slot ring, offload then load, on high-priority
+    streams with default (programmatic dependent) launches, while a low-priority stream runs a
+    matmul loop for the whole time."""
+    w = wl.WORKLOADS["8b_ring"]
+    g = dims_of(w.shape, 384)
+    pool = _pool_8b_384()
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 256)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    src = wl.block_ids(w.seed, g.NB, 128)
+    dst = wl.block_ids(w.dst_seed, g.NB, 128)
+    descs = kvc.kvc_map_request(lay, len(src))
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    ring = kvc.kvc_staging_ring_create(cb, 3, kind)
+    host_out = torch.empty(len(descs) * cb, dtype=torch.uint8).pin_memory()
+    lo, hi = torch.cuda.Stream.priority_range()
+    s_gemm = torch.cuda.Stream(priority=lo)
+    s_k, s_c = torch.cuda.Stream(priority=hi), torch.cuda.Stream(priority=hi)
+    want_chunks = orc.pack_request(g, pool, src, 256)
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, want_chunks, dst, 256)
+    torch.cuda.synchronize()
+    gemm_done, keep = _gemm_load(s_gemm)
+    overlapped = 0
+    for rep in range(6):            # several passes so that the transfers span the matmul loop
+        for (_, c, first, nb, nbytes) in descs:
+            slot, dptr, hptr = kvc.kvc_staging_ring_acquire(ring, timeout_us=10_000_000)
+            kvc.kvc_pack(lay, src[first:first + nb], dptr, cb, stream=s_k)
+            kvc.kvc_staging_ring_commit(ring, slot, s_k)
+            kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
+            if kind == kvc.KVC_RING_DEVICE:
+                cuda_rt.memcpy_async(host_out.data_ptr() + c * cb, dptr, nbytes, cuda_rt.D2H, s_c)
+            else:
+                cuda_rt.memcpy_async(host_out.data_ptr() + c * cb, hptr, nbytes, cuda_rt.H2H, s_c)
+            kvc.kvc_staging_ring_release(ring, slot, s_c)
+        s_c.synchronize()
+        overlapped += not gemm_done.query()
+        assert np.array_equal(host_out.numpy(), np.concatenate(want_chunks)), "offload pass %d" % rep
+        pool_t.copy_(torch.from_numpy(pool))
+        torch.cuda.current_stream().synchronize()
+        for (_, c, first, nb, nbytes) in descs:
+            slot, dptr, hptr = kvc.kvc_staging_ring_acquire(ring, timeout_us=10_000_000)
+            if kind == kvc.KVC_RING_DEVICE:
+                cuda_rt.memcpy_async(dptr, host_out.data_ptr() + c * cb, nbytes, cuda_rt.H2D, s_c)
+            else:
+                cuda_rt.memcpy_async(hptr, host_out.data_ptr() + c * cb, nbytes, cuda_rt.H2H, s_c)
+            kvc.kvc_staging_ring_commit(ring, slot, s_c)
+            kvc.kvc_staging_ring_wait_filled(ring, slot, s_k)
+            kvc.kvc_unpack(lay, dptr, dst[first:first + nb], cb, stream=s_k)
+            kvc.kvc_staging_ring_release(ring, slot, s_k)
+        s_k.synchronize()
+        overlapped += not gemm_done.query()
+        assert np.array_equal(pool_t.cpu().numpy(), want_pool), "load pass %d" % rep
+    assert overlapped >= 2, "the matmul loop ended before the transfers ran beside it"
+    torch.cuda.synchronize()
+    kvc.kvc_staging_ring_destroy(ring)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+@pytest.mark.parametrize("variant", [kvc.KVC_VARIANT_VEC, kvc.KVC_VARIANT_BULK])
+def test_pack_right_after_unpack_on_one_stream_sees_the_new_data(variant):
+    """unpack(new chunk) -> pack of the same blocks, alternating many times on one stream with
+    programmatic dependent launch: the pack grid may be resident while the unpack grid still
+    writes the pool, and must read the written bytes, never stale ones."""
+    g = orc.Dims(4, 2, 64, 16, 8, 128, 2)
+    pool = wl.random_bits(2024, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 16 * g.B)
+    kvc.kvc_layout_set_tuning(lay, variant=variant, pdl=2)
+    ids = wl.block_ids(5, g.NB, 16)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    reps = 24
+    fresh = [to_dev(wl.random_bits(3000 + i, cb)) for i in range(reps)]
+    outs = [torch.zeros(cb, dtype=torch.uint8, device=DEV) for _ in range(reps)]
+    torch.cuda.synchronize()
+    for i in range(reps):
+        kvc.kvc_unpack(lay, fresh[i], ids)
+        kvc.kvc_pack(lay, ids, outs[i])
+    torch.cuda.synchronize()
+    for i in range(reps):
+        # pack(unpack(chunk)) of the same ids is the chunk itself (round-trip identity of the oracle)
+        assert torch.equal(outs[i], fresh[i]), "round %d read stale pool bytes" % i
+    want_pool = pool.copy()
+    orc.unpack_chunk(g, want_pool, fresh[-1].cpu().numpy(), ids)
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+def test_first_launches_of_two_handles_race_on_two_threads():
+    """Two host threads, each with its own handle and a different shared-memory footprint, make
+    their first bulk launches at the same time (the opt-in shared-memory size of a kernel is
+    process-wide state).  Both must succeed and be exact; repeated with fresh handles."""
+    g = orc.Dims(2, 2, 48, 16, 8, 128, 2)
+    pool = wl.random_bits(77, g.pool_bytes)
+    ids = wl.block_ids(6, g.NB, 20)
+    want = np.concatenate(orc.pack_request(g, pool, ids, 64))
+    pool_t = to_dev(pool)
+    tunings = [dict(max_ctas=8, stages=2), dict(max_ctas=8, stages=6), dict(stages=3, group=kvc.KVC_GROUP_FORCE_KERNEL),
+               dict(max_ctas=4, stages=5, group=kvc.KVC_GROUP_FORCE_KERNEL)]
+    errors = []
+
+    def worker(tuning, barrier, out):
+        try:
+            torch.cuda.set_device(0)
+            st = torch.cuda.Stream()
+            lay = dense_layout(pool_t, g, 64)
+            kvc.kvc_layout_set_tuning(lay, variant=kvc.KVC_VARIANT_BULK, **tuning)
+            ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, ids, out)
+            barrier.wait()
+            for _ in range(5):
+                kvc.kvc_pack_batch(lay, ops, dev, stream=st)
+            st.synchronize()
+            assert kvc.kvc_poll_device_status(lay, stream=st) == (0, 0)
+        except Exception as e:  # reported by the main thread
+            errors.append(repr(e))
+
+    for rnd in range(3):
+        outs = [torch.zeros(want.size, dtype=torch.uint8, device=DEV) for _ in tunings]
+        barrier = threading.Barrier(len(tunings))
+        ts = [threading.Thread(target=worker, args=(t, barrier, o)) for t, o in zip(tunings, outs)]
+        for t in ts:
+            t.start()
+        for t in ts:
+            t.join(timeout=120)
+        assert errors == []
+        torch.cuda.synchronize()
+        for o in outs:
+            assert np.array_equal(o.cpu().numpy(), want)

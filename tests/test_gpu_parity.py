@@ -54,13 +54,13 @@ def _oracle_results(g, pool_np, src_ids, dst_ids, chunk_tokens):
 
 
 def run_pack_unpack(g, pool_np, src_ids, dst_ids, chunk_tokens, variant, order, mode, tile=0,
-                    layout_factory=None, pool_dev=None):
+                    layout_factory=None, pool_dev=None, **tuning):
     """Pack src_ids into a staging area, unpack into dst_ids of the same pool, and compare both
     results with the oracle.  mode: 'chunk' (one call per chunk, host ids), 'chunk_dev'
     (device ids), 'batch' / 'batch_dev' (one launch)."""
     pool_t = to_dev(pool_np) if pool_dev is None else pool_dev
     lay = (layout_factory or dense_layout)(pool_t, g, chunk_tokens)
-    kvc.kvc_layout_set_tuning(lay, variant=variant, order=order, tile_bytes=tile)
+    kvc.kvc_layout_set_tuning(lay, variant=variant, order=order, tile_bytes=tile, **tuning)
     descs = kvc.kvc_map_request(lay, len(src_ids))
     sizes = [d[4] for d in descs]
     total = sum(sizes)

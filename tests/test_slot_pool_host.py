@@ -70,6 +70,34 @@ def test_foreground_takes_over_unclaimed_preloads_and_cancel():
     assert (c["cancels"], c["foreground_refusals"], c["n_free"]) == (1, 1, 0)
 
 
+def test_staged_preload_that_is_still_held_is_not_taken_over():
+    """A preload whose read has finished but whose holder has not let go yet (its copy into the
+    slot may still be running) must not be handed to foreground work; nor may a preload that
+    other candidates joined be cancelled under them."""
+    pool = kvc.kvc_slot_pool_create(2, 1, max_speculative=0)
+    a, _ = kvc.kvc_slot_pool_acquire(pool, P, 1)
+    kvc.kvc_slot_pool_mark_staged(pool, a)                        # staged, the preloader still holds it
+    d, _ = kvc.kvc_slot_pool_acquire(pool, D, 10)                 # the reserved slot
+    assert d != a
+    assert kvc.kvc_slot_pool_acquire(pool, D, 11) is None         # nothing to take: WOULD_BLOCK
+    assert kvc.kvc_slot_pool_get_counters(pool)["reclaims"] == 0
+    kvc.kvc_slot_pool_release(pool, a)                            # now it waits unreferenced
+    got = kvc.kvc_slot_pool_acquire(pool, D, 11)
+    assert got == (a, False)
+    assert kvc.kvc_slot_pool_get_counters(pool)["reclaims"] == 1
+
+    pool = kvc.kvc_slot_pool_create(4, 1, max_speculative=0)
+    b, _ = kvc.kvc_slot_pool_acquire(pool, P, 5)
+    b2, joined = kvc.kvc_slot_pool_acquire(pool, P, 5)            # a second candidate joins the read
+    assert b2 == b and joined
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_slot_pool_cancel(pool, b)
+    assert e.value.status == kvc.KVC_ERR_STATE
+    kvc.kvc_slot_pool_release(pool, b)                            # the joiner leaves
+    kvc.kvc_slot_pool_cancel(pool, b)                             # sole holder: allowed
+    assert kvc.kvc_slot_pool_get_counters(pool)["n_free"] == 4
+
+
 def test_retention_is_an_lru_cache():
     pool = kvc.kvc_slot_pool_create(3, 0, retain_completed=True)
     slots = {}

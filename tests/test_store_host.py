@@ -114,3 +114,50 @@ def test_first_writer_wins_between_processes(tmp_path):
         assert (buf == winners[0]).all()                # complete, and the winner's bytes
     leftovers = [f for _, _, fs in os.walk(str(tmp_path)) for f in fs if f.startswith(".tmp")]
     assert leftovers == []
+
+
+def test_file_system_that_refuses_direct_io_falls_back_and_leaves_no_litter(tmp_path):
+    """Linux creates the file before it refuses O_DIRECT on a file system without it.  The store
+    must remove that empty file, retry with buffered I/O, count the refusal, publish the entry
+    and leave no temporary name behind.  The refusal is played by an open() stand-in."""
+    import ctypes
+    OPEN_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_char_p, ctypes.c_int, ctypes.c_uint, use_errno=True)
+    libc = ctypes.CDLL(None, use_errno=True)
+    libc.open.restype = ctypes.c_int
+    libc.open.argtypes = [ctypes.c_char_p, ctypes.c_int, ctypes.c_uint]
+    refused = []
+
+    def refusing_open(path, flags, mode):
+        if flags & os.O_DIRECT:
+            if flags & os.O_CREAT:                       # what the kernel does: create, then refuse
+                fd = libc.open(path, flags & ~os.O_DIRECT, mode)
+                if fd >= 0:
+                    os.close(fd)
+            refused.append(path)
+            ctypes.set_errno(22)                         # EINVAL
+            return -1
+        fd = libc.open(path, flags, mode)
+        if fd < 0:
+            ctypes.set_errno(ctypes.get_errno())
+        return fd
+
+    hook = OPEN_FN(refusing_open)
+    L = kvc.lib()
+    L.kvc_store_set_open_fn.argtypes = [OPEN_FN]
+    L.kvc_store_set_open_fn.restype = ctypes.c_int
+    st = kvc.kvc_store_open(str(tmp_path), "m", direct_io=True)
+    try:
+        assert L.kvc_store_set_open_fn(hook) == 0
+        data = _aligned(1 << 20, seed=11)
+        assert kvc.kvc_store_publish(st, 0xabcdef, data) is True
+        assert kvc.kvc_store_direct_io_refused(st) == 1 and len(refused) == 1
+        back = _aligned(1 << 20, seed=12)
+        kvc.kvc_store_read(st, 0xabcdef, back)           # the read is refused once too, then buffered
+        assert np.array_equal(back, data)
+        assert kvc.kvc_store_direct_io_refused(st) == 2
+        assert kvc.kvc_store_publish(st, 0xabcdef, data) is False
+    finally:
+        L.kvc_store_set_open_fn(ctypes.cast(None, OPEN_FN))
+        kvc.kvc_store_close(st)
+    leftovers = [f for _, _, fs in os.walk(str(tmp_path)) for f in fs if f.startswith(".tmp")]
+    assert leftovers == []
