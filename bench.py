@@ -531,6 +531,8 @@ def suite_launch_shapes(torch, kvc, dev, reps):
     P, B, C = kvc.KVC_ORDER_PLANE_MAJOR, kvc.KVC_ORDER_BLOCK_MAJOR, kvc.KVC_ORDER_CHUNK_MAJOR
     cands = [
         ("default: bulk, streaming (2 items/block, 2 stages), chunk-major", dict()),
+        ("multi-slab bulk kernel forced, one 32 KiB slab per item (A/B of the two bulk kernels)",
+         dict(group=kvc.KVC_GROUP_FORCE_KERNEL)),
         ("bulk streaming, 1 item per block", dict(items_per_cta=1)),
         ("bulk streaming, 4 items per block", dict(items_per_cta=4)),
         ("bulk streaming, 8 items per block, 3 stages", dict(items_per_cta=8, stages=3)),
@@ -559,6 +561,64 @@ def suite_launch_shapes(torch, kvc, dev, reps):
                     "unpack_ms": ud, "unpack_gbs": 2 * one_way / ud / 1e6})
         kvc.kvc_layout_destroy(lay)
     return out
+
+
+def suite_small_slabs(torch, kvc, dev, reps):
+    """Layouts with small slabs (tensor-parallel shards of the KV heads, 1-byte elements): 2 GiB
+    requests, 32 layers x K,V, 16-token blocks, slab sizes from 32 KiB down to 256 B, 256-token
+    chunks, one batched launch per direction.  Kernels: the default (bulk copies, several slabs
+    per work item), the bulk kernel held to one slab per item, and the vector kernel."""
+    peak = measured_peak()[0]
+    L, P, B = 32, 2, 16
+    out = []
+    for S, H, D, e in ((32768, 8, 128, 2), (8192, 2, 128, 2), (4096, 1, 128, 2), (2048, 1, 128, 1),
+                       (1024, 1, 64, 1), (256, 1, 16, 1)):
+        per_block = L * P * S
+        n = (2 << 30) // per_block
+        NB = 4 * n
+        pool = wl.random_bits_cuda(wl.BASE_SEED + S, NB * per_block, dev)
+        src, dst = wl.block_ids(wl.BASE_SEED + 1, NB, n), wl.block_ids(wl.BASE_SEED + 2, NB, n)
+        staging = torch.empty(n * per_block, dtype=torch.uint8, device=dev)
+        for name, cfg in (("bulk, slabs grouped per item (default)", dict()),
+                          ("bulk, one slab per item", dict(group=1)),
+                          ("vector kernel", dict(variant=1))):
+            lay = kvc.kvc_layout_create_dense(pool, L, P, NB, B, H, D, e, 256)
+            kvc.kvc_layout_set_tuning(lay, **cfg)
+            ops_p, k1, nbytes, _ = kvc.request_chunk_ops(lay, src, staging)
+            ops_u, k2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+            pm, pd = _time_ms(torch, lambda: kvc.kvc_pack_batch(lay, ops_p, 0), reps)
+            um, ud = _time_ms(torch, lambda: kvc.kvc_unpack_batch(lay, ops_u, 0), reps)
+            assert kvc.kvc_poll_device_status(lay) == (0, 0)
+            out.append({"slab_bytes": S, "blocks": n, "bytes_each_way": nbytes, "kernel": name,
+                        "pack_ms": pd, "pack_gbs": 2 * nbytes / pd / 1e6,
+                        "pack_frac_of_measured_peak": 2 * nbytes / pd / 1e6 / peak,
+                        "unpack_ms": ud, "unpack_gbs": 2 * nbytes / ud / 1e6,
+                        "unpack_frac_of_measured_peak": 2 * nbytes / ud / 1e6 / peak})
+            kvc.kvc_layout_destroy(lay)
+        del pool, staging
+        torch.cuda.empty_cache()
+    return out
+
+
+def suite_call_overhead(reps):
+    """Per-call cost of the per-chunk entry points measured from C: builds and runs
+    tests/native/call_overhead.c against the in-tree library (gcc and the CUDA headers needed)."""
+    import subprocess
+    import tempfile
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    pkg = os.path.join(ROOT, "paper_2609_11744_b200")
+    with tempfile.TemporaryDirectory() as d:
+        exe = os.path.join(d, "call_overhead")
+        subprocess.check_call(
+            ["gcc", "-std=c99", "-O2", os.path.join(ROOT, "tests", "native", "call_overhead.c"),
+             "-I", os.path.join(ROOT, "include"), "-I", os.path.join(cuda, "include"),
+             "-L", pkg, "-lkvc", "-L", os.path.join(cuda, "lib64"), "-lcudart",
+             "-Wl,-rpath," + pkg, "-Wl,-rpath," + os.path.join(cuda, "lib64"), "-o", exe])
+        run = subprocess.run([exe, "6000", "5000", str(max(3, min(reps, 15)))], capture_output=True,
+                             text=True, timeout=900)
+    if run.returncode != 0:
+        raise RuntimeError("call_overhead failed (%d): %s" % (run.returncode, run.stderr[-500:]))
+    return [json.loads(l) for l in run.stdout.splitlines() if l.startswith("{")]
 
 
 def suite_8k(torch, kvc, dev, reps):
@@ -910,6 +970,8 @@ def run_suite(args):
     for name, fn in (("host_link", lambda: suite_host_link(torch, cuda_rt, dev)),
                      ("launch_shapes", lambda: suite_launch_shapes(torch, kvc, dev, args.steps)),
                      ("chunk_sweep", lambda: suite_chunk_sweep(torch, kvc, dev, args.steps)),
+                     ("small_slabs", lambda: suite_small_slabs(torch, kvc, dev, args.steps)),
+                     ("call_overhead", lambda: suite_call_overhead(args.steps)),
                      ("prefix_8k", lambda: suite_8k(torch, kvc, dev, args.steps)),
                      ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
                      ("ring_overlap", lambda: suite_ring_overlap(torch, kvc, cuda_rt, dev,
@@ -946,7 +1008,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
-                         "host_link,launch_shapes,chunk_sweep,prefix_8k,batch_70b,ring_overlap,file_pipeline (1 GPU; prints one JSON line)")
+                         "host_link,launch_shapes,chunk_sweep,small_slabs,call_overhead,prefix_8k,batch_70b,"
+                         "ring_overlap,file_pipeline (1 GPU; prints one JSON line)")
     ap.add_argument("--overlap-seconds", type=float, default=2.0)
     ap.add_argument("--file-roots", default="/tmp,/dev/shm",
                     help="comma list of directories for the file_pipeline suite part")
