@@ -445,6 +445,29 @@ def _time_ms(torch, fn, reps, warm=3, flush=None):
     return min(ts), statistics.median(ts)
 
 
+def _kernel_and_call_ms(torch, kvc, lay, fn, reps, warm=9):
+    """(mean kernel ms, shortest kernel ms, ms per call when calls follow one another).  The kernel
+    time comes from the library's own event pair around each launch, so the host work of a call
+    (validating ids, building and uploading the block table) is not in it; the per-call time is
+    reps back-to-back calls on one stream, first event to last, which is what a caller that keeps
+    the stream fed observes (the slower of host work and kernel)."""
+    kvc.kvc_layout_set_kernel_timing(lay, True)
+    for _ in range(warm):   # more calls than the handle has table arenas, so none is allocated later
+        fn()
+    torch.cuda.synchronize()
+    kvc.kvc_layout_kernel_time(lay)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    b.synchronize()
+    n, total, lo, hi = kvc.kvc_layout_kernel_time(lay)
+    kvc.kvc_layout_set_kernel_timing(lay, False)
+    assert n == reps
+    return total / n, lo, a.elapsed_time(b) / reps
+
+
 def suite_chunk_sweep(torch, kvc, dev, reps):
     """8B shape, 80k-token prefix: chunk 16/256/2048 tokens, one batched launch vs one launch per
     chunk, pack and unpack timed separately."""
@@ -563,7 +586,7 @@ def suite_launch_shapes(torch, kvc, dev, reps):
     return out
 
 
-def suite_small_slabs(torch, kvc, dev, reps):
+def suite_small_slabs(torch, kvc, dev, reps, sizes=None, request_mib=2048):
     """Layouts with small slabs (tensor-parallel shards of the KV heads, 1-byte elements): 2 GiB
     requests, 32 layers x K,V, 16-token blocks, slab sizes from 32 KiB down to 256 B, 256-token
     chunks, one batched launch per direction.  Kernels: the default (bulk copies, several slabs
@@ -573,8 +596,10 @@ def suite_small_slabs(torch, kvc, dev, reps):
     out = []
     for S, H, D, e in ((32768, 8, 128, 2), (8192, 2, 128, 2), (4096, 1, 128, 2), (2048, 1, 128, 1),
                        (1024, 1, 64, 1), (256, 1, 16, 1)):
+        if sizes and S not in sizes:
+            continue
         per_block = L * P * S
-        n = (2 << 30) // per_block
+        n = (request_mib << 20) // per_block
         NB = 4 * n
         pool = wl.random_bits_cuda(wl.BASE_SEED + S, NB * per_block, dev)
         src, dst = wl.block_ids(wl.BASE_SEED + 1, NB, n), wl.block_ids(wl.BASE_SEED + 2, NB, n)
@@ -586,14 +611,17 @@ def suite_small_slabs(torch, kvc, dev, reps):
             kvc.kvc_layout_set_tuning(lay, **cfg)
             ops_p, k1, nbytes, _ = kvc.request_chunk_ops(lay, src, staging)
             ops_u, k2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
-            pm, pd = _time_ms(torch, lambda: kvc.kvc_pack_batch(lay, ops_p, 0), reps)
-            um, ud = _time_ms(torch, lambda: kvc.kvc_unpack_batch(lay, ops_u, 0), reps)
+            row = {"slab_bytes": S, "blocks": n, "bytes_each_way": nbytes, "kernel": name}
+            for d, fn in (("pack", lambda: kvc.kvc_pack_batch(lay, ops_p, 0)),
+                          ("unpack", lambda: kvc.kvc_unpack_batch(lay, ops_u, 0))):
+                k_ms, k_min, call_ms = _kernel_and_call_ms(torch, kvc, lay, fn, reps)
+                row.update({d + "_kernel_ms": k_ms, d + "_kernel_ms_min": k_min,
+                            d + "_gbs": 2 * nbytes / k_ms / 1e6,
+                            d + "_frac_of_measured_peak": 2 * nbytes / k_ms / 1e6 / peak,
+                            d + "_call_ms_pipelined": call_ms,
+                            d + "_call_gbs_pipelined": 2 * nbytes / call_ms / 1e6})
             assert kvc.kvc_poll_device_status(lay) == (0, 0)
-            out.append({"slab_bytes": S, "blocks": n, "bytes_each_way": nbytes, "kernel": name,
-                        "pack_ms": pd, "pack_gbs": 2 * nbytes / pd / 1e6,
-                        "pack_frac_of_measured_peak": 2 * nbytes / pd / 1e6 / peak,
-                        "unpack_ms": ud, "unpack_gbs": 2 * nbytes / ud / 1e6,
-                        "unpack_frac_of_measured_peak": 2 * nbytes / ud / 1e6 / peak})
+            out.append(row)
             kvc.kvc_layout_destroy(lay)
         del pool, staging
         torch.cuda.empty_cache()
@@ -970,7 +998,10 @@ def run_suite(args):
     for name, fn in (("host_link", lambda: suite_host_link(torch, cuda_rt, dev)),
                      ("launch_shapes", lambda: suite_launch_shapes(torch, kvc, dev, args.steps)),
                      ("chunk_sweep", lambda: suite_chunk_sweep(torch, kvc, dev, args.steps)),
-                     ("small_slabs", lambda: suite_small_slabs(torch, kvc, dev, args.steps)),
+                     ("small_slabs", lambda: suite_small_slabs(
+                         torch, kvc, dev, args.steps,
+                         [int(x) for x in args.small_slab_sizes.split(",")] if args.small_slab_sizes else None,
+                         args.small_slab_mib)),
                      ("call_overhead", lambda: suite_call_overhead(args.steps)),
                      ("prefix_8k", lambda: suite_8k(torch, kvc, dev, args.steps)),
                      ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
@@ -1010,6 +1041,10 @@ def main():
                     help="run the other configs instead of the bench step: all, or a comma list of "
                          "host_link,launch_shapes,chunk_sweep,small_slabs,call_overhead,prefix_8k,batch_70b,"
                          "ring_overlap,file_pipeline (1 GPU; prints one JSON line)")
+    ap.add_argument("--small-slab-sizes", default="",
+                    help="small_slabs suite part: comma list of slab sizes in bytes (default: all)")
+    ap.add_argument("--small-slab-mib", type=int, default=2048,
+                    help="small_slabs suite part: request size in MiB (small cases for profiler captures)")
     ap.add_argument("--overlap-seconds", type=float, default=2.0)
     ap.add_argument("--file-roots", default="/tmp,/dev/shm",
                     help="comma list of directories for the file_pipeline suite part")

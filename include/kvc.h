@@ -158,12 +158,20 @@ typedef struct {
                             a kernel's blocks may be scheduled while the previous kernel of the
                             stream drains; they wait for its completion before reading memory */
     uint32_t group;      /* BULK: slabs per work item.  0 = default: when a slab is at most half a
-                            tile, as many whole slabs as fit one tile (a power of two, at most 32)
+                            tile, as many whole slabs as fit one tile (a power of two, at most 16;
+                            the default tile is 16 KiB for slabs under 4 KiB)
                             -- consecutive slabs of a chunk are contiguous in the slot, so one item
                             is several copies on the pool side and one on the slot side;
-                            1 = one slab (or one tile of a slab) per item; N > 1 = at most N.
+                            1 = one slab (or one tile of a slab) per item; N > 1 = at most N (<= 32).
+                            VEC: slabs of at most 4 KiB are moved several per warp the same way.
                             Adding KVC_GROUP_FORCE_KERNEL runs the multi-slab kernel even when that
                             leaves one slab per item (for same-process comparisons) */
+    uint32_t slot_memory; /* where the staging slots of this handle's calls live: 0 = ask the CUDA
+                            runtime on every call (one pointer-attribute query, a fraction of a
+                            microsecond), 1 = device memory, 2 = mapped pinned host memory.  A
+                            caller that issues many small per-chunk calls into slots it allocated
+                            itself can save the query; a wrong answer picks a kernel tuned for the
+                            other kind of memory */
 } kvc_tuning;
 #define KVC_GROUP_FORCE_KERNEL 0x100u
 /* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */
@@ -292,6 +300,17 @@ kvc_status kvc_unpack_copy_engine(kvc_layout *layout, const void *src, uint64_t 
 /* Number of kernel launches issued through this handle so far (no counterpart in the paper;
  * the benchmark reports it so that a run that launched nothing cannot pass for a GPU run). */
 uint64_t kvc_layout_launch_count(const kvc_layout *layout);
+
+/* Kernel timing (diagnostic, no counterpart in the paper).  With on != 0 every copy kernel
+ * launched through the handle (not kvc_pack_batch_static) is bracketed by two CUDA events on its
+ * stream, so that the kernel's own duration can be told from the call's host work and table upload.
+ * The events sit between consecutive kernels of a stream and so keep programmatic dependent launch
+ * from overlapping them: leave it off outside measurements.  kvc_layout_kernel_time waits for the
+ * launches timed since its last call and reports their number, summed, shortest and longest
+ * duration in milliseconds (any pointer may be NULL).  Errors: INVALID_ARG, NOMEM, CUDA. */
+kvc_status kvc_layout_set_kernel_timing(kvc_layout *layout, int on);
+kvc_status kvc_layout_kernel_time(kvc_layout *layout, uint32_t *launches, double *total_ms,
+                                  double *min_ms, double *max_ms);
 
 /* ------------------------------------------------------------------ staging ring (Sec. 6.4) */
 

@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <utility>
 #include <vector>
 
 #include "kvc.h"
@@ -13,6 +14,10 @@
 #define KVC_VEC_THREADS 256u    // threads per block of the vector kernels
 #define KVC_VEC_UNROLL 4u       // vectors in flight per thread
 #define KVC_VEC_WARP_TEAM_MAX_TILE 4096u  // tiles up to this size are copied by one warp each
+// Slabs up to this size are moved several per work item by one warp (multi-slab vector kernel);
+// an item is about this many bytes.
+#define KVC_VEC_GROUP_MAX_SLAB 4096u
+#define KVC_VEC_GROUP_ITEM_BYTES 8192u
 #define KVC_HOST_SLOT_DEFAULT_CTAS 16u
 #define KVC_BULK_THREADS 32u    // one warp drives the bulk-copy pipeline
 #define KVC_BULK_MAX_STAGES 16u
@@ -31,6 +36,7 @@
 // one tile in total.  Its shared-memory header holds the mbarriers (128 bytes) and, per stage, the
 // address and length of up to 32 stores (384 bytes), rounded up to 128 bytes.
 #define KVC_GROUP_MAX_SLABS 32u
+#define KVC_GROUP_DEFAULT_SLABS 16u
 #define KVC_GROUP_STAGE_INFO_BYTES 384u
 #define KVC_GROUP_SMEM_HEADER(stages) ((128u + (stages) * KVC_GROUP_STAGE_INFO_BYTES + 127u) & ~127u)
 #define KVC_WAIT_LIMIT (1u << 22)   // polls of an mbarrier before a kernel gives up
@@ -79,14 +85,16 @@ struct KvcLaunch {
     uint32_t pdl;             // launch with programmatic stream serialisation
     uint32_t group_shift;     // multi-slab kernel: log2 of the slabs per work item
     uint32_t pending;         // bulk kernels: stores that may still read shared memory at a stage reuse
-    uint64_t n_slabs;         // multi-slab kernel: n_ent * LP
+    uint64_t n_slabs;         // multi-slab kernels: n_ent * LP
+    uint64_t vec_magic;       // multi-slab vector kernel: 2^32 / (vectors per slab) + 1, for v / vps
     int32_t ids[KVC_PARAM_IDS];
 };
 
 enum { KVC_DIR_PACK = 0, KVC_DIR_UNPACK = 1 };
 // Internal refinements: 32-byte vectors when everything is 32-byte aligned; the bulk kernel whose
 // work items span several slabs.
-enum { KVC_VARIANT_VEC32 = 100, KVC_VARIANT_BULK_GROUP = 101 };
+enum { KVC_VARIANT_VEC32 = 100, KVC_VARIANT_BULK_GROUP = 101, KVC_VARIANT_VEC_GROUP = 102,
+       KVC_VARIANT_VEC32_GROUP = 103 };
 
 // Implemented in kvc_kernels.cu.
 cudaError_t kvc_launch_copy(int dir, int variant, const KvcLaunch &a, uint32_t grid,
@@ -124,7 +132,15 @@ struct kvc_layout {
     uint64_t launches;
     std::vector<uint32_t> seen;  // scratch for duplicate detection: stamp per pool block
     uint32_t seen_stamp;
+    // kernel timing (diagnostic): event pairs around launches not yet collected, and spare events
+    bool time_kernels;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timed;
+    std::vector<cudaEvent_t> spare_events;
 };
+
+// Launches the copy kernel; with kernel timing on, between two events on the same stream.
+kvc_status kvc_launch_timed(kvc_layout *lay, int dir, int variant, const KvcLaunch &a, uint32_t grid,
+                            uint32_t smem, cudaStream_t st);
 
 
 // Where block j, plane lp of a chunk of nb blocks starts, relative to the chunk base:

@@ -219,6 +219,83 @@ kvc_vec_kernel(const __grid_constant__ KvcLaunch a)
     }
 }
 
+
+// ------------------------------------------------------------------------------------ VEC, several slabs per item
+//
+// Small slabs (a tensor-parallel shard of the KV heads, 1-byte elements, small blocks): the cost
+// that matters is per slab -- the table lookups of the decode -- and the remedy is many warps,
+// each with many independent loads in flight.  A work item is a run of R = 2^group_shift
+// consecutive slabs (in slot order) given to ONE warp: lane i decodes slab i, then the warp copies
+// the R*S bytes as one stream of vectors, each lane fetching the addresses of the slab its vector
+// falls in from the decoding lane by shuffle.  The next item is decoded before the current one is
+// copied, so the lookups overlap the copies.
+template <int DIR, bool TABLE, int VB>
+__global__ void __launch_bounds__(KVC_VEC_THREADS)
+kvc_vec_group_kernel(const __grid_constant__ KvcLaunch a)
+{
+    constexpr uint32_t SH = VB == 32 ? 5 : 4;
+    constexpr uint32_t U = VB == 32 ? 4 : 8;     // 128 bytes in flight per lane
+    constexpr uint32_t WARPS = KVC_VEC_THREADS / 32;
+    constexpr uint32_t FULL = 0xffffffffu;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t ksh = a.group_shift, R = 1u << ksh;
+    const uint32_t vps = a.g.slab_bytes >> SH;    // vectors per slab
+    const uint32_t total = R * vps;               // vectors per item
+    const uint64_t magic = a.vec_magic;
+    const uint64_t n_items = a.n_items, n_slabs = a.n_slabs;
+    const uint64_t stride = (uint64_t)gridDim.x * WARPS;
+    uint64_t w = (uint64_t)blockIdx.x * WARPS + (threadIdx.x >> 5);
+    grid_dependency_wait();
+    if (w >= n_items)
+        return;
+    auto decode_mine = [&](uint64_t item) {
+        Item it;
+        it.pool = it.slot = 0;
+        it.len = 0;
+        const uint64_t r = (item << ksh) + lane;
+        if (lane < R && r < n_slabs)
+            it = decode<TABLE>(a, (uint32_t)r, true);
+        return it;
+    };
+    Item cur = decode_mine(w);
+    while (true) {
+        const uint64_t wn = w + stride;
+        const bool more = wn < n_items;
+        Item nxt = cur;
+        if (more)
+            nxt = decode_mine(wn);
+        const uint64_t my_src = DIR == KVC_DIR_PACK ? cur.pool : cur.slot;
+        const uint64_t my_dst = DIR == KVC_DIR_PACK ? cur.slot : cur.pool;
+        for (uint32_t v0 = 0; v0 < total; v0 += 32u * U) {
+            Vec<VB> r[U];
+            uint64_t d[U];
+            bool live[U];
+#pragma unroll
+            for (uint32_t u = 0; u < U; ++u) {
+                const uint32_t v = v0 + u * 32u + lane;
+                uint32_t slab = (uint32_t)(((uint64_t)v * magic) >> 32);  // v / vps
+                slab = min(slab, R - 1u);
+                const uint32_t off = (v - slab * vps) << SH;
+                const uint64_t sa = __shfl_sync(FULL, my_src, slab);
+                const uint64_t da = __shfl_sync(FULL, my_dst, slab);
+                const uint32_t len = __shfl_sync(FULL, cur.len, slab);
+                live[u] = v < total && len != 0;
+                d[u] = da + off;
+                if (live[u])
+                    r[u].load(sa + off);
+            }
+#pragma unroll
+            for (uint32_t u = 0; u < U; ++u)
+                if (live[u])
+                    r[u].store(d[u]);
+        }
+        if (!more)
+            break;
+        cur = nxt;
+        w = wn;
+    }
+}
+
 // ------------------------------------------------------------------------------------ BULK
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
@@ -642,6 +719,10 @@ cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t 
             return e;
         return launch_cfg(kvc_bulk_group_kernel<DIR, TABLE>, a, grid, KVC_BULK_THREADS, smem, stream);
     }
+    if (variant == KVC_VARIANT_VEC32_GROUP)
+        return launch_cfg(kvc_vec_group_kernel<DIR, TABLE, 32>, a, grid, KVC_VEC_THREADS, 0, stream);
+    if (variant == KVC_VARIANT_VEC_GROUP)
+        return launch_cfg(kvc_vec_group_kernel<DIR, TABLE, 16>, a, grid, KVC_VEC_THREADS, 0, stream);
     const bool warp_team = a.g.tile_bytes <= KVC_VEC_WARP_TEAM_MAX_TILE;
     if (variant == KVC_VARIANT_VEC32)
         return warp_team

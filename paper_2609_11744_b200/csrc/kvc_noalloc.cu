@@ -220,6 +220,7 @@ extern "C" kvc_status kvc_pack_batch_static(kvc_layout *lay, const kvc_chunk_op 
     // resident while the upload kernels are still writing them: plain stream order, no
     // programmatic overlap with the preceding kernel.
     a.pdl = 0;
+    // (kvc_launch_copy directly: the timing diagnostic of the handle creates events, this path must not)
     if (kvc_launch_copy(KVC_DIR_PACK, plan.variant, a, plan.grid, plan.smem, st) != cudaSuccess)
         return KVC_ERR_CUDA;
     ++lay->launches;

@@ -56,7 +56,7 @@ class kvc_tuning(ctypes.Structure):
                 ("stages", ctypes.c_uint32), ("ctas_per_sm", ctypes.c_uint32),
                 ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32),
                 ("items_per_cta", ctypes.c_uint32), ("pdl", ctypes.c_uint32),
-                ("group", ctypes.c_uint32)]
+                ("group", ctypes.c_uint32), ("slot_memory", ctypes.c_uint32)]
 
 
 class kvc_chunk_desc(ctypes.Structure):
@@ -138,6 +138,9 @@ def lib() -> ctypes.CDLL:
         "kvc_unpack_copy_engine": (ci, [vp, vp, u64, vp, u32, vp]),
         "kvc_poll_device_status": (ci, [vp, vp, P(u32), P(u32)]),
         "kvc_layout_launch_count": (u64, [vp]),
+        "kvc_layout_set_kernel_timing": (ci, [vp, ci]),
+        "kvc_layout_kernel_time": (ci, [vp, P(u32), P(ctypes.c_double), P(ctypes.c_double),
+                                        P(ctypes.c_double)]),
         "kvc_staging_ring_create": (ci, [u64, u32, ci, vp, u64, P(vp)]),
         "kvc_staging_ring_destroy": (ci, [vp]),
         "kvc_staging_ring_acquire": (ci, [vp, i64, P(u32), P(vp), P(vp)]),
@@ -321,14 +324,28 @@ def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
 
 
 def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
-                          ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, pdl=0, group=0) -> None:
+                          ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, pdl=0, group=0,
+                          slot_memory=0) -> None:
     t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag,
-                   items_per_cta, pdl, group)
+                   items_per_cta, pdl, group, slot_memory)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
 
 
 def kvc_layout_launch_count(layout) -> int:
     return lib().kvc_layout_launch_count(layout.handle)
+
+
+def kvc_layout_set_kernel_timing(layout, on: bool) -> None:
+    _check(lib().kvc_layout_set_kernel_timing(layout.handle, int(on)), "kvc_layout_set_kernel_timing")
+
+
+def kvc_layout_kernel_time(layout) -> Tuple[int, float, float, float]:
+    """(launches, total ms, shortest ms, longest ms) of the kernels timed since the last call."""
+    n = ctypes.c_uint32()
+    t, lo, hi = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    _check(lib().kvc_layout_kernel_time(layout.handle, ctypes.byref(n), ctypes.byref(t),
+                                        ctypes.byref(lo), ctypes.byref(hi)), "kvc_layout_kernel_time")
+    return n.value, t.value, lo.value, hi.value
 
 
 # ------------------------------------------------------------------ mapper

@@ -85,6 +85,31 @@ int main(int argc, char **argv)
     CU(cudaEventCreate(&ev1));
     CU(cudaEventCreateWithFlags(&fork, cudaEventDisableTiming));
 
+    /* the floor: the smallest stream operation the runtime can enqueue (a 16-byte memset), 5000 times */
+    {
+        double host_us[64], dev_ms[64];
+        for (int r = -2; r < reps; ++r) {
+            CU(cudaDeviceSynchronize());
+            CU(cudaEventRecord(ev0, st[0]));
+            const double t0 = now_us();
+            for (int c = 0; c < 5000; ++c)
+                CU(cudaMemsetAsync(staging + 256 * (c % 64), 0, 16, st[0]));
+            const double t1 = now_us();
+            CU(cudaEventRecord(ev1, st[0]));
+            CU(cudaEventSynchronize(ev1));
+            float ms = 0;
+            CU(cudaEventElapsedTime(&ms, ev0, ev1));
+            if (r >= 0) {
+                host_us[r] = (t1 - t0) / 5000;
+                dev_ms[r] = ms;
+            }
+        }
+        const double hm = median(host_us, reps), dm = median(dev_ms, reps);
+        printf("{\"case\": \"floor_16_byte_memset\", \"calls\": 5000, \"streams\": 1, "
+               "\"host_us_per_call\": %.3f, \"device_ms\": %.4f, \"device_us_per_call\": %.3f}\n",
+               hm, dm, dm * 1e3 / 5000);
+    }
+
     const uint32_t chunk_tokens[3] = {16, 256, 2048};
     for (int ci = 0; ci < 3; ++ci) {
         kvc_layout_desc desc;
@@ -93,6 +118,13 @@ int main(int argc, char **argv)
         CK(kvc_layout_create(&desc, &lay));
         const uint32_t bpc = kvc_layout_blocks_per_chunk(lay);
         const uint32_t n_chunks = kvc_layout_num_chunks(lay, n);
+        for (int hint = 0; hint < 2; ++hint) {
+        kvc_tuning tun;
+        memset(&tun, 0, sizeof(tun));
+        tun.slot_memory = (uint32_t)hint; /* 1: the caller vouches that slots are device memory */
+        CK(kvc_layout_set_tuning(lay, &tun));
+        if (hint && ci != 0)
+            continue;
         for (int dir = 0; dir < 2; ++dir) {
             for (int ns = 1; ns <= NSTREAMS; ns += NSTREAMS - 1) {
                 double host_us[64], dev_ms[64];
@@ -129,10 +161,12 @@ int main(int argc, char **argv)
                 }
                 const double hm = median(host_us, reps), dm = median(dev_ms, reps);
                 printf("{\"case\": \"per_chunk\", \"direction\": \"%s\", \"chunk_tokens\": %u, \"calls\": %u, "
-                       "\"streams\": %d, \"host_us_per_call\": %.3f, \"device_ms\": %.4f, \"gbs\": %.1f}\n",
-                       dir ? "unpack" : "pack", chunk_tokens[ci], n_chunks, ns, hm, dm,
-                       2.0 * per_block * n / dm / 1e6);
+                       "\"streams\": %d, \"slot_memory_hint\": %d, \"host_us_per_call\": %.3f, "
+                       "\"device_ms\": %.4f, \"device_us_per_call\": %.3f, \"gbs\": %.1f}\n",
+                       dir ? "unpack" : "pack", chunk_tokens[ci], n_chunks, ns, hint, hm, dm,
+                       dm * 1e3 / n_chunks, 2.0 * per_block * n / dm / 1e6);
             }
+        }
         }
         uint32_t skipped = 0, expired = 0;
         CK(kvc_poll_device_status(lay, st[0], &skipped, &expired));

@@ -16,7 +16,7 @@ import workloads as wl
 from test_gpu_parity import DEV, dense_layout, run_pack_unpack, to_dev
 
 pytestmark = pytest.mark.gpu
-BULK = kvc.KVC_VARIANT_BULK
+BULK, VEC = kvc.KVC_VARIANT_BULK, kvc.KVC_VARIANT_VEC
 
 # (L, P, NB, B, H, D, e): slab bytes = B*H*D*e
 GEOMS = {
@@ -39,22 +39,33 @@ def _case(name, n, chunk_blocks, **kw):
     return g, pool, src, dst, chunk_blocks * g.B
 
 
+@pytest.mark.parametrize("variant", [BULK, VEC])
 @pytest.mark.parametrize("name", sorted(GEOMS))
 @pytest.mark.parametrize("mode", ["chunk", "chunk_dev", "batch", "batch_dev"])
-def test_default_grouping_every_slab_size(name, mode):
+def test_default_grouping_every_slab_size(name, mode, variant):
     # 37 blocks in chunks of 8: four full chunks and a ragged one of 5; planes * blocks per chunk
     # is not a multiple of the slabs per item, so items straddle planes and chunks
     g, pool, src, dst, ct = _case(name, 37, 8)
-    run_pack_unpack(g, pool, src, dst, ct, BULK, 0, mode)
+    run_pack_unpack(g, pool, src, dst, ct, variant, 0, mode)
 
 
+@pytest.mark.parametrize("variant", [BULK, VEC])
 @pytest.mark.parametrize("group", [2, 4, 8, 32, 1, kvc.KVC_GROUP_FORCE_KERNEL | 1])
 @pytest.mark.parametrize("order", [kvc.KVC_ORDER_CHUNK_MAJOR, kvc.KVC_ORDER_PLANE_MAJOR,
                                    kvc.KVC_ORDER_BLOCK_MAJOR])
-def test_slabs_per_item_and_traversal_orders(group, order):
+def test_slabs_per_item_and_traversal_orders(group, order, variant):
     g, pool, src, dst, ct = _case("S1K", 45, 16)
     for mode in ("chunk", "batch_dev"):
-        run_pack_unpack(g, pool, src, dst, ct, BULK, order, mode, group=group)
+        run_pack_unpack(g, pool, src, dst, ct, variant, order, mode, group=group)
+
+
+@pytest.mark.parametrize("tuning", [dict(max_ctas=2), dict(items_per_cta=1), dict(items_per_cta=9),
+                                    dict(pdl=1), dict(group=2, max_ctas=5)],
+                         ids=lambda t: ",".join("%s=%s" % kv for kv in t.items()))
+def test_vector_kernel_launch_shapes_with_grouped_items(tuning):
+    for name, n, cb in (("S64", 71, 16), ("S2K", 61, 16), ("S4K", 35, 4), ("S48", 50, 8)):
+        g, pool, src, dst, ct = _case(name, n, cb)
+        run_pack_unpack(g, pool, src, dst, ct, VEC, 0, "batch", **tuning)
 
 
 @pytest.mark.parametrize("tuning", [
@@ -63,10 +74,12 @@ def test_slabs_per_item_and_traversal_orders(group, order):
     dict(tile_bytes=8192), dict(tile_bytes=4096, stages=5, lag=3), dict(pdl=1), dict(l2_hint=2),
 ], ids=lambda t: ",".join("%s=%s" % kv for kv in t.items()))
 def test_launch_shapes_with_grouped_items(tuning):
+    tuning = dict(tuning)
+    tile = tuning.pop("tile_bytes", 0)
     g, pool, src, dst, ct = _case("S2K", 61, 16)
-    run_pack_unpack(g, pool, src, dst, ct, BULK, 0, "batch", **tuning)
+    run_pack_unpack(g, pool, src, dst, ct, BULK, 0, "batch", tile, **tuning)
     g, pool, src, dst, ct = _case("S256", 33, 4)
-    run_pack_unpack(g, pool, src, dst, ct, BULK, 0, "chunk", **tuning)
+    run_pack_unpack(g, pool, src, dst, ct, BULK, 0, "chunk", tile, **tuning)
 
 
 def test_multi_slab_kernel_with_one_slab_per_item_on_8b_shape():
@@ -79,8 +92,9 @@ def test_multi_slab_kernel_with_one_slab_per_item_on_8b_shape():
         run_pack_unpack(g, pool, src, dst, 256, BULK, 0, mode, group=kvc.KVC_GROUP_FORCE_KERNEL)
 
 
+@pytest.mark.parametrize("variant", [BULK, VEC])
 @pytest.mark.parametrize("name", ["S64", "S1K", "S4K", "S12K"])
-def test_block_major_chunks_with_grouped_items(name):
+def test_block_major_chunks_with_grouped_items(name, variant):
     """Chunk byte order [n][L][P]..: consecutive slabs of the slot are the planes of ONE block."""
     g = orc.Dims(*GEOMS[name])
     pool = wl.random_bits(500 + g.H, g.pool_bytes)
@@ -88,7 +102,7 @@ def test_block_major_chunks_with_grouped_items(name):
     pool_t = to_dev(pool)
     lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 8 * g.B,
                                       chunk_order=kvc.KVC_CHUNK_BLOCK_MAJOR)
-    kvc.kvc_layout_set_tuning(lay, variant=BULK)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
     n = 29
     src, dst = wl.block_ids(15, g.NB, n), wl.block_ids(16, g.NB, n)
     staging = torch.full((n * g.bytes_per_block + 4096,), 0x5A, dtype=torch.uint8, device=DEV)
@@ -114,14 +128,15 @@ def test_block_major_chunks_with_grouped_items(name):
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
 
 
-def test_bad_device_ids_inside_grouped_items():
+@pytest.mark.parametrize("variant", [BULK, VEC])
+def test_bad_device_ids_inside_grouped_items(variant):
     """A bad id in the middle of an item: its slabs are skipped, the slot-side copy is split
     around the hole, and nothing else is disturbed."""
     g = orc.Dims(*GEOMS["S1K"])
     pool = wl.random_bits(77, g.pool_bytes)
     pool_t = to_dev(pool)
     lay = dense_layout(pool_t, g, 16 * g.B)
-    kvc.kvc_layout_set_tuning(lay, variant=BULK)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
     ids = np.array([3, 95, 96, 7, -1, 9, 1 << 30, 0, 31, 2, 5, -7, 11], dtype=np.int32)
     good = (ids >= 0) & (ids < g.NB)
     n_bad = int((~good).sum())
@@ -145,13 +160,15 @@ def test_bad_device_ids_inside_grouped_items():
     assert np.array_equal(pool_t.cpu().numpy(), want_pool)
 
 
-def test_many_requests_in_one_launch_small_slabs():
+@pytest.mark.parametrize("variant", [BULK, VEC])
+def test_many_requests_in_one_launch_small_slabs(variant):
     """Chunks of many requests, of different lengths, in one launch: items cross from one
     request's slot into the next one's, which lies somewhere else."""
     g = orc.Dims(*GEOMS["S2K"])
     pool = wl.random_bits(91, g.pool_bytes)
     pool_t = to_dev(pool)
     lay = dense_layout(pool_t, g, 4 * g.B)
+    kvc.kvc_layout_set_tuning(lay, variant=variant)
     rng = np.random.default_rng(5)
     perm = rng.permutation(g.NB).astype(np.int32)
     lens = [1, 4, 3, 7, 2, 9, 5]
