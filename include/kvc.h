@@ -374,6 +374,7 @@ kvc_status kvc_staging_ring_set_trace(kvc_ring *ring, kvc_ring_trace_entry *buf,
 uint32_t kvc_staging_ring_trace_count(const kvc_ring *ring);
 uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *ring);
 uint32_t kvc_staging_ring_num_slots(const kvc_ring *ring);
+int kvc_staging_ring_pool_mode(const kvc_ring *ring); /* 1 after kvc_staging_ring_set_policy */
 
 /* ------------------------------------------------------------------ chunk files (Sec. 6.3) */
 
@@ -401,6 +402,12 @@ kvc_status kvc_store_publish(kvc_store *store, uint64_t hash, const void *host_b
 /* Reads exactly `bytes`; INVALID_ARG if the entry has another size.  Errors: NOT_FOUND, IO. */
 kvc_status kvc_store_read(kvc_store *store, uint64_t hash, void *host_buf, uint64_t bytes);
 int kvc_store_direct_io_refused(const kvc_store *store);
+/* Entries read and published through this handle so far, and their bytes (completed calls only):
+ * with these a caller can check that a chunk shared by several requests was read once. */
+typedef struct {
+    uint64_t reads, read_bytes, publishes, publish_bytes;
+} kvc_store_counters;
+kvc_status kvc_store_get_counters(const kvc_store *store, kvc_store_counters *out);
 /* Test seam (no counterpart in the paper): every file the store opens goes through `fn`
  * (path, open(2) flags, mode; returns a descriptor or -1 with errno set).  NULL restores open(2).
  * Process-wide.  Lets a host test play a file system that refuses O_DIRECT. */
@@ -448,6 +455,50 @@ kvc_status kvc_pipeline_load(kvc_layout *layout, kvc_ring *ring, kvc_store *stor
                              uint32_t n_blocks, const uint64_t *hashes, uint32_t n_hashes,
                              uint32_t io_threads, int use_copy_engine, void *stream,
                              kvc_pipeline_stats *stats);
+/* Both calls work on a FIFO ring and on a ring in pool mode (below); in pool mode the chunk hash
+ * is the slot key, so a chunk that is already in the staging memory is neither packed nor read
+ * again.  On any error exit every slot the call took is handed back: a slot whose copy was never
+ * enqueued at once, the others after the copy or file operation in progress on them has ended;
+ * queued file operations that had not started are dropped. */
+
+/* Several requests served at once from one staging pool (Sec. 6.4: every mapping that became ready
+ * during one pass of the loop, from whichever request, goes into ONE fused unpack launch; Sec. 6.5:
+ * demand loads before preloads, a chunk already in the pool -- being read, read, or cached -- is
+ * joined, not read again; a finished preload waits in its slot until the demand load for the same
+ * hash claims it).  `ring` must be in pool mode with host-visible slots.
+ * Per request: ids (HOST, n_blocks destination blocks; unused for a preload), one hash per chunk,
+ * and the class, KVC_CLASS_DEMAND_LOAD (chunks are unpacked into ids on `stream`) or
+ * KVC_CLASS_PRELOAD (chunks are only brought into the pool, as far as the policy lets them).
+ * For every request the contiguous prefix of chunks present in the store is processed;
+ * loaded_chunks and ready_seconds (seconds from the start of the call until the request's last
+ * unpack was enqueued, or its last chunk staged) are written back.  Destination blocks of different
+ * requests must be distinct.  Returns when all reads are done and all unpacks ENQUEUED:
+ * synchronise `stream` before using the blocks.  Not re-entrant on the same ring.
+ * Errors: INVALID_ARG, STATE (ring not in pool mode, or a chunk is being filled by another user
+ * of the pool), TIMEOUT, and whatever unpack / the store report. */
+typedef struct {
+    const int32_t *ids;
+    uint32_t n_blocks;
+    const uint64_t *hashes;
+    uint32_t n_hashes;
+    uint32_t cls;           /* kvc_slot_class: KVC_CLASS_DEMAND_LOAD or KVC_CLASS_PRELOAD */
+    uint32_t loaded_chunks; /* out */
+    double ready_seconds;   /* out */
+} kvc_load_request;
+typedef struct {
+    uint64_t bytes_read;       /* bytes read from files by this call */
+    double seconds;            /* wall time of the call */
+    uint32_t chunks;           /* (request, chunk) pairs completed */
+    uint32_t reads;            /* files read */
+    uint32_t joins;            /* chunks served from a slot that already held them */
+    uint32_t claims;           /* preloads claimed by demand loads (pool total so far) */
+    uint32_t unpack_launches;  /* fused unpack launches */
+    uint32_t ring_stalls;      /* acquisition attempts that found nothing available */
+    uint32_t preloads_refused; /* preload chunks given up because the policy left no room */
+} kvc_load_many_stats;
+kvc_status kvc_pipeline_load_many(kvc_layout *layout, kvc_ring *ring, kvc_store *store,
+                                  kvc_load_request *requests, uint32_t n_requests, uint32_t io_threads,
+                                  void *stream, kvc_load_many_stats *stats);
 
 /* ------------------------------------------------------------------ slot policy (Sec. 6.5) */
 
@@ -491,6 +542,49 @@ kvc_status kvc_slot_pool_release(kvc_slot_pool *pool, uint32_t slot);
  * preload candidates have joined. */
 kvc_status kvc_slot_pool_cancel(kvc_slot_pool *pool, uint32_t slot);
 kvc_status kvc_slot_pool_get_counters(const kvc_slot_pool *pool, kvc_slot_pool_counters *out);
+/* One slot's bookkeeping: state (kvc_slot_state), references held, key, and whether it is a
+ * preload no demand request has claimed.  Any pointer may be NULL. */
+typedef enum { KVC_SLOT_FREE = 0, KVC_SLOT_IN_FLIGHT = 1, KVC_SLOT_STAGED = 2, KVC_SLOT_RETAINED = 3 } kvc_slot_state;
+kvc_status kvc_slot_pool_slot_info(const kvc_slot_pool *pool, uint32_t slot, uint32_t *state, uint32_t *refs,
+                                   uint64_t *key, int *speculative);
+
+/* ------------------------------------------------------------------ staging pool mode (Sec. 6.4, 6.5) */
+
+/* The paper's staging memory is ONE pool shared by demand loads, stores and preloads, and any free
+ * slot goes to the most urgent job that is ready (Sec. 6.4, 6.5); a FIFO ring cannot do that: a
+ * slow file read on slot k would hold up every later slot.  kvc_staging_ring_set_policy switches a
+ * ring whose slots are all free to pool mode: slots are then handed out in any order under the
+ * slot-policy rules above (foreground reserve, bound on preloads in flight, one shared
+ * reference-counted slot per key, claims, take-over of retained and of unclaimed staged slots),
+ * and the two events per slot keep their meaning -- a slot returns to the policy only after the
+ * event recorded behind its last GPU consumer has completed.
+ *   acquire_for  class + key (chunk hash).  *joined = 0: a slot for a new operation; fill it, then
+ *                commit / commit_host.  *joined = 1: the key already holds this slot (being filled,
+ *                filled, or cached); the caller holds one more reference and must not fill it --
+ *                kvc_staging_ring_slot_filled tells whether the bytes are there yet.
+ *                timeout_us as for kvc_staging_ring_acquire.  Errors: WOULD_BLOCK, TIMEOUT, STATE
+ *                (ring not in pool mode), NOMEM, CUDA.
+ *   commit, commit_host, wait_filled, sync_filled: as in FIFO mode.
+ *   release      drops ONE reference once the GPU work enqueued so far on consumer_stream has run
+ *                (the slot's "drained" event is re-recorded behind every consumer, chained to the
+ *                previous record); release_host drops one reference at once.  When the last
+ *                reference is gone the slot is free -- or kept as a cached chunk (retention on) or
+ *                as a finished preload waiting to be claimed, until foreground work takes it over.
+ *   cancel       gives up an unclaimed preload that is still being filled (sole holder only).
+ *   abandon      returns a slot that was acquired (not joined by anyone else) and will not be
+ *                filled after all, e.g. because its copy could not be enqueued; also valid in
+ *                FIFO mode.  STATE otherwise.
+ * In pool mode kvc_staging_ring_acquire returns STATE, and the in_flight figure of
+ * kvc_staging_ring_stats counts cached chunks as well. */
+kvc_status kvc_staging_ring_set_policy(kvc_ring *ring, uint32_t foreground_reserve, uint32_t max_speculative,
+                                       int retain_completed);
+kvc_status kvc_staging_ring_acquire_for(kvc_ring *ring, kvc_slot_class cls, uint64_t key, int64_t timeout_us,
+                                        uint32_t *slot, void **dev_ptr, void **host_ptr, int *joined);
+kvc_status kvc_staging_ring_slot_filled(kvc_ring *ring, uint32_t slot, int *filled);
+kvc_status kvc_staging_ring_cancel(kvc_ring *ring, uint32_t slot);
+kvc_status kvc_staging_ring_abandon(kvc_ring *ring, uint32_t slot);
+/* The policy's counters (after handing back references whose GPU work has completed). */
+kvc_status kvc_staging_ring_policy_counters(kvc_ring *ring, kvc_slot_pool_counters *out);
 
 /* Event provider used by a ring (test seam, no counterpart in the paper; the paper's rule it
  * serves is Sec. 6.4's "a slot is reused only after its CUDA event has completed").

@@ -61,6 +61,9 @@ struct Slot {
     void *filled = nullptr;
     void *drained = nullptr;
     bool filled_by_host = false;  // committed by kvc_staging_ring_commit_host: no event to wait for
+    // pool mode: references released by consumers whose GPU work (guarded by `drained`) may still
+    // be reading the slot; they are handed back to the slot policy once the event has completed
+    uint32_t deferred = 0;
 };
 
 }  // namespace
@@ -79,6 +82,7 @@ struct kvc_ring {
     uint64_t acquires, stalls;
     kvc_ring_trace_entry *trace;  // caller's buffer, or nullptr
     uint32_t trace_cap, trace_n;
+    kvc_slot_pool *policy;     // pool mode: who gets which slot (nullptr = FIFO ring)
 };
 
 namespace {
@@ -109,6 +113,36 @@ int slot_is_free(kvc_ring *r, Slot &s)
     if (q == 0)
         s.state = SLOT_FREE;
     return q;
+}
+
+// Pool mode: a slot the policy has freed is free here too (a retained or unclaimed staged slot
+// keeps its bytes and stays FILLED).
+void sync_with_policy(kvc_ring *r, uint32_t slot)
+{
+    uint32_t state = 0;
+    kvc_slot_pool_slot_info(r->policy, slot, &state, nullptr, nullptr, nullptr);
+    if (state == KVC_SLOT_FREE)
+        r->slots[slot].state = SLOT_FREE;
+}
+
+// Pool mode: hands references whose GPU work has completed back to the policy.
+// Returns <0 on an event error.
+int reap_deferred(kvc_ring *r)
+{
+    for (uint32_t i = 0; i < r->n_slots; ++i) {
+        Slot &s = r->slots[i];
+        if (!s.deferred)
+            continue;
+        const int q = r->ev.query(r->ev.ctx, s.drained);
+        if (q < 0)
+            return q;
+        if (q != 0)
+            continue;
+        for (; s.deferred; --s.deferred)
+            kvc_slot_pool_release(r->policy, i);
+        sync_with_policy(r, i);
+    }
+    return 0;
 }
 
 }  // namespace
@@ -162,6 +196,7 @@ kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ri
     r->acquires = r->stalls = 0;
     r->trace = nullptr;
     r->trace_cap = r->trace_n = 0;
+    r->policy = nullptr;
     try {
         r->slots.resize(n_slots);
     } catch (const std::bad_alloc &) {
@@ -229,13 +264,16 @@ kvc_status kvc_staging_ring_destroy(kvc_ring *r)
         // work recorded behind a slot may still touch ring memory: wait for it before freeing
         if (s.state == SLOT_FILLED && s.filled && r->ev.synchronize(r->ev.ctx, s.filled) != 0)
             rc = KVC_ERR_CUDA;
-        if (s.state == SLOT_DRAINING && s.drained && r->ev.synchronize(r->ev.ctx, s.drained) != 0)
+        if ((s.state == SLOT_DRAINING || s.deferred) && s.drained &&
+            r->ev.synchronize(r->ev.ctx, s.drained) != 0)
             rc = KVC_ERR_CUDA;
         if (s.filled)
             r->ev.destroy(r->ev.ctx, s.filled);
         if (s.drained)
             r->ev.destroy(r->ev.ctx, s.drained);
     }
+    if (r->policy)
+        kvc_slot_pool_destroy(r->policy);
     if (r->owns_mem) {
         if (r->kind == KVC_RING_DEVICE)
             cudaFree(r->dev_base);
@@ -251,6 +289,8 @@ kvc_status kvc_staging_ring_acquire(kvc_ring *r, int64_t timeout_us, uint32_t *s
 {
     if (!r || !slot || timeout_us < 0)
         return KVC_ERR_INVALID_ARG;
+    if (r->policy)
+        return KVC_ERR_STATE;  // pool mode: slots are handed out by kvc_staging_ring_acquire_for
     Slot &s = r->slots[r->head];
     const auto deadline =
         std::chrono::steady_clock::now() + std::chrono::microseconds(timeout_us);
@@ -307,6 +347,8 @@ kvc_status kvc_staging_ring_commit(kvc_ring *r, uint32_t slot, void *producer_st
         return KVC_ERR_CUDA;
     s.filled_by_host = false;
     s.state = SLOT_FILLED;
+    if (r->policy)
+        kvc_slot_pool_mark_staged(r->policy, slot);
     trace(r, slot, KVC_TRACE_COMMIT);
     return KVC_OK;
 }
@@ -330,6 +372,22 @@ kvc_status kvc_staging_ring_release(kvc_ring *r, uint32_t slot, void *consumer_s
     Slot &s = r->slots[slot];
     if (s.state != SLOT_FILLED)
         return KVC_ERR_STATE;
+    if (r->policy) {
+        // one consumer lets go; others may still hold the slot.  The event is re-recorded behind
+        // every consumer's stream, each made to wait for the record before it, so its completion
+        // means that all consumers released so far are done.
+        uint32_t refs = 0;
+        kvc_slot_pool_slot_info(r->policy, slot, nullptr, &refs, nullptr, nullptr);
+        if (refs <= s.deferred)
+            return KVC_ERR_STATE;  // more releases than references
+        if (s.deferred && r->ev.stream_wait(r->ev.ctx, consumer_stream, s.drained) != 0)
+            return KVC_ERR_CUDA;
+        if (r->ev.record(r->ev.ctx, s.drained, consumer_stream) != 0)
+            return KVC_ERR_CUDA;
+        ++s.deferred;
+        trace(r, slot, KVC_TRACE_RELEASE);
+        return KVC_OK;
+    }
     if (r->ev.record(r->ev.ctx, s.drained, consumer_stream) != 0)
         return KVC_ERR_CUDA;
     s.state = SLOT_DRAINING;
@@ -346,6 +404,8 @@ kvc_status kvc_staging_ring_commit_host(kvc_ring *r, uint32_t slot)
         return KVC_ERR_STATE;
     s.filled_by_host = true;
     s.state = SLOT_FILLED;
+    if (r->policy)
+        kvc_slot_pool_mark_staged(r->policy, slot);
     trace(r, slot, KVC_TRACE_COMMIT);
     return KVC_OK;
 }
@@ -367,6 +427,18 @@ kvc_status kvc_staging_ring_release_host(kvc_ring *r, uint32_t slot)
     if (!r || slot >= r->n_slots)
         return KVC_ERR_INVALID_ARG;
     Slot &s = r->slots[slot];
+    if (r->policy) {
+        uint32_t refs = 0;
+        kvc_slot_pool_slot_info(r->policy, slot, nullptr, &refs, nullptr, nullptr);
+        // a filled slot: any holder may let go; a slot still being filled: only someone who
+        // joined it (the filler's own reference has to stay until it commits or abandons)
+        if (!(s.state == SLOT_FILLED && refs > s.deferred) && !(s.state == SLOT_ACQUIRED && refs > 1))
+            return KVC_ERR_STATE;
+        kvc_slot_pool_release(r->policy, slot);
+        sync_with_policy(r, slot);
+        trace(r, slot, KVC_TRACE_RELEASE);
+        return KVC_OK;
+    }
     if (s.state != SLOT_FILLED)
         return KVC_ERR_STATE;
     s.state = SLOT_FREE;
@@ -404,6 +476,141 @@ kvc_status kvc_staging_ring_set_trace(kvc_ring *r, kvc_ring_trace_entry *buf, ui
 
 uint32_t kvc_staging_ring_trace_count(const kvc_ring *r) { return r ? r->trace_n : 0; }
 
+kvc_status kvc_staging_ring_set_policy(kvc_ring *r, uint32_t foreground_reserve, uint32_t max_speculative,
+                                       int retain_completed)
+{
+    if (!r)
+        return KVC_ERR_INVALID_ARG;
+    if (r->policy && reap_deferred(r) < 0)
+        return KVC_ERR_CUDA;
+    for (Slot &s : r->slots) {
+        if (s.state == SLOT_DRAINING && slot_is_free(r, s) < 0)
+            return KVC_ERR_CUDA;
+        if (s.state != SLOT_FREE || s.deferred)
+            return KVC_ERR_STATE;  // only while every slot is free (no cached chunk either)
+    }
+    kvc_slot_pool *p = nullptr;
+    kvc_status rc = kvc_slot_pool_create(r->n_slots, foreground_reserve, max_speculative, retain_completed, &p);
+    if (rc != KVC_OK)
+        return rc;
+    if (r->policy)
+        kvc_slot_pool_destroy(r->policy);
+    r->policy = p;
+    for (Slot &s : r->slots) {
+        s.state = SLOT_FREE;
+        s.deferred = 0;
+    }
+    r->head = 0;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_acquire_for(kvc_ring *r, kvc_slot_class cls, uint64_t key, int64_t timeout_us,
+                                        uint32_t *slot, void **dev_ptr, void **host_ptr, int *joined)
+{
+    if (!r || !slot || !joined || timeout_us < 0)
+        return KVC_ERR_INVALID_ARG;
+    if (!r->policy)
+        return KVC_ERR_STATE;
+    const auto deadline = std::chrono::steady_clock::now() + std::chrono::microseconds(timeout_us);
+    bool stall_logged = false;
+    uint32_t polls = 0, nap_us = 2;
+    for (;;) {
+        if (reap_deferred(r) < 0)
+            return KVC_ERR_CUDA;
+        uint32_t got = 0;
+        int j = 0;
+        const kvc_status rc = kvc_slot_pool_acquire(r->policy, cls, key, &got, &j);
+        if (rc == KVC_OK) {
+            Slot &s = r->slots[got];
+            if (!j) {
+                // a fresh slot, or one taken over from a retained / unclaimed staged chunk: its old
+                // references are all back (the policy only gives away unreferenced slots), so no
+                // GPU work can still be touching it
+                s.state = SLOT_ACQUIRED;
+                s.filled_by_host = false;
+                ++r->acquires;
+                trace(r, got, KVC_TRACE_ACQUIRE);
+            }
+            *slot = got;
+            *joined = j;
+            if (dev_ptr)
+                *dev_ptr = r->dev_base + (uint64_t)got * r->slot_bytes;
+            if (host_ptr)
+                *host_ptr = r->host_base ? r->host_base + (uint64_t)got * r->slot_bytes : nullptr;
+            return KVC_OK;
+        }
+        if (rc != KVC_ERR_WOULD_BLOCK)
+            return rc;
+        ++r->stalls;
+        if (!stall_logged) {
+            trace(r, r->n_slots, KVC_TRACE_STALL);
+            stall_logged = true;
+        }
+        if (timeout_us == 0)
+            return KVC_ERR_WOULD_BLOCK;
+        if (std::chrono::steady_clock::now() >= deadline)
+            return KVC_ERR_TIMEOUT;
+        if (++polls <= 8) {
+            std::this_thread::yield();
+        } else {
+            std::this_thread::sleep_for(std::chrono::microseconds(nap_us));
+            nap_us = nap_us * 2 > 20 ? 20 : nap_us * 2;
+        }
+    }
+}
+
+kvc_status kvc_staging_ring_slot_filled(kvc_ring *r, uint32_t slot, int *filled)
+{
+    if (!r || slot >= r->n_slots || !filled)
+        return KVC_ERR_INVALID_ARG;
+    *filled = r->slots[slot].state == SLOT_FILLED;
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_cancel(kvc_ring *r, uint32_t slot)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    if (!r->policy || r->slots[slot].state != SLOT_ACQUIRED)
+        return KVC_ERR_STATE;
+    const kvc_status rc = kvc_slot_pool_cancel(r->policy, slot);
+    if (rc == KVC_OK)
+        r->slots[slot].state = SLOT_FREE;
+    return rc;
+}
+
+kvc_status kvc_staging_ring_abandon(kvc_ring *r, uint32_t slot)
+{
+    if (!r || slot >= r->n_slots)
+        return KVC_ERR_INVALID_ARG;
+    Slot &s = r->slots[slot];
+    if (s.state != SLOT_ACQUIRED)
+        return KVC_ERR_STATE;
+    if (!r->policy) {
+        s.state = SLOT_FREE;
+        return KVC_OK;
+    }
+    uint32_t refs = 0;
+    kvc_slot_pool_slot_info(r->policy, slot, nullptr, &refs, nullptr, nullptr);
+    if (refs != 1)
+        return KVC_ERR_STATE;  // others joined and wait for the bytes
+    kvc_slot_pool_release(r->policy, slot);  // in flight, last reference: the slot is freed
+    sync_with_policy(r, slot);
+    return KVC_OK;
+}
+
+kvc_status kvc_staging_ring_policy_counters(kvc_ring *r, kvc_slot_pool_counters *out)
+{
+    if (!r || !out)
+        return KVC_ERR_INVALID_ARG;
+    if (!r->policy)
+        return KVC_ERR_STATE;
+    if (reap_deferred(r) < 0)
+        return KVC_ERR_CUDA;
+    return kvc_slot_pool_get_counters(r->policy, out);
+}
+
+int kvc_staging_ring_pool_mode(const kvc_ring *r) { return r && r->policy ? 1 : 0; }
 uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *r) { return r ? r->slot_bytes : 0; }
 uint32_t kvc_staging_ring_num_slots(const kvc_ring *r) { return r ? r->n_slots : 0; }
 

@@ -239,6 +239,23 @@ kvc_status kvc_slot_pool_cancel(kvc_slot_pool *p, uint32_t slot)
     return KVC_OK;
 }
 
+kvc_status kvc_slot_pool_slot_info(const kvc_slot_pool *p, uint32_t slot, uint32_t *state, uint32_t *refs,
+                                   uint64_t *key, int *speculative)
+{
+    if (!p || slot >= p->slots.size())
+        return KVC_ERR_INVALID_ARG;
+    const PSlot &s = p->slots[slot];
+    if (state)
+        *state = (uint32_t)s.state;
+    if (refs)
+        *refs = s.refs;
+    if (key)
+        *key = s.key;
+    if (speculative)
+        *speculative = s.speculative ? 1 : 0;
+    return KVC_OK;
+}
+
 kvc_status kvc_slot_pool_get_counters(const kvc_slot_pool *p, kvc_slot_pool_counters *out)
 {
     if (!p || !out)

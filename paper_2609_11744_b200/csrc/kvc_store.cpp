@@ -27,6 +27,7 @@ struct kvc_store {
     bool want_direct;
     std::atomic<int> direct_refused;  // times O_DIRECT was refused and buffered I/O used instead
     std::atomic<uint64_t> seq;        // makes temporary names unique inside the process
+    std::atomic<uint64_t> reads, read_bytes, publishes, publish_bytes;  // completed operations
 };
 
 namespace {
@@ -163,6 +164,7 @@ kvc_status kvc_store_open(const char *root, const char *model_tag, int direct_io
     st->want_direct = direct_io != 0;
     st->direct_refused = 0;
     st->seq = 0;
+    st->reads = st->read_bytes = st->publishes = st->publish_bytes = 0;
     if (!mkdir_p(st->root)) {
         delete st;
         return KVC_ERR_IO;
@@ -237,6 +239,10 @@ kvc_status kvc_store_publish(kvc_store *st, uint64_t hash, const void *host_buf,
             rc = errno == EEXIST ? KVC_ERR_EXISTS : KVC_ERR_IO;
     }
     unlink(tmp.c_str());
+    if (rc == KVC_OK) {
+        st->publishes.fetch_add(1);
+        st->publish_bytes.fetch_add(bytes);
+    }
     return rc;
 }
 
@@ -259,10 +265,25 @@ kvc_status kvc_store_read(kvc_store *st, uint64_t hash, void *host_buf, uint64_t
     else
         rc = read_all(fd, static_cast<unsigned char *>(host_buf), bytes);
     close(fd);
+    if (rc == KVC_OK) {
+        st->reads.fetch_add(1);
+        st->read_bytes.fetch_add(bytes);
+    }
     return rc;
 }
 
 int kvc_store_direct_io_refused(const kvc_store *st) { return st ? st->direct_refused.load() : 0; }
+
+kvc_status kvc_store_get_counters(const kvc_store *st, kvc_store_counters *out)
+{
+    if (!st || !out)
+        return KVC_ERR_INVALID_ARG;
+    out->reads = st->reads.load();
+    out->read_bytes = st->read_bytes.load();
+    out->publishes = st->publishes.load();
+    out->publish_bytes = st->publish_bytes.load();
+    return KVC_OK;
+}
 
 kvc_status kvc_store_set_open_fn(kvc_open_fn fn)
 {

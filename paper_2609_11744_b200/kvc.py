@@ -71,6 +71,22 @@ class kvc_pipeline_stats(ctypes.Structure):
                 ("ring_stalls", ctypes.c_uint32)]
 
 
+class kvc_load_request(ctypes.Structure):
+    _fields_ = [("ids", ctypes.c_void_p), ("n_blocks", ctypes.c_uint32), ("hashes", ctypes.c_void_p),
+                ("n_hashes", ctypes.c_uint32), ("cls", ctypes.c_uint32),
+                ("loaded_chunks", ctypes.c_uint32), ("ready_seconds", ctypes.c_double)]
+
+
+class kvc_load_many_stats(ctypes.Structure):
+    _fields_ = [("bytes_read", ctypes.c_uint64), ("seconds", ctypes.c_double)] + \
+               [(k, ctypes.c_uint32) for k in ("chunks", "reads", "joins", "claims", "unpack_launches",
+                                               "ring_stalls", "preloads_refused")]
+
+
+class kvc_store_counters(ctypes.Structure):
+    _fields_ = [(k, ctypes.c_uint64) for k in ("reads", "read_bytes", "publishes", "publish_bytes")]
+
+
 class kvc_slot_pool_counters(ctypes.Structure):
     _fields_ = [(k, ctypes.c_uint32) for k in ("n_free", "n_in_flight", "n_staged", "n_retained")] + \
                [(k, ctypes.c_uint64) for k in ("acquires", "joins", "claims", "reclaims", "cancels",
@@ -158,6 +174,10 @@ def lib() -> ctypes.CDLL:
         "kvc_staging_ring_release_host": (ci, [vp, u32]),
         "kvc_pipeline_store": (ci, [vp, vp, vp, vp, u32, vp, u32, u32, ci, vp, P(kvc_pipeline_stats)]),
         "kvc_pipeline_load": (ci, [vp, vp, vp, vp, u32, vp, u32, u32, ci, vp, P(kvc_pipeline_stats)]),
+        "kvc_pipeline_load_many": (ci, [vp, vp, vp, P(kvc_load_request), u32, u32, vp,
+                                        P(kvc_load_many_stats)]),
+        "kvc_store_get_counters": (ci, [vp, P(kvc_store_counters)]),
+        "kvc_staging_ring_pool_mode": (ci, [vp]),
         "kvc_slot_pool_create": (ci, [u32, u32, u32, ci, P(vp)]),
         "kvc_slot_pool_destroy": (ci, [vp]),
         "kvc_slot_pool_acquire": (ci, [vp, ci, u64, P(u32), P(ci)]),
@@ -165,6 +185,13 @@ def lib() -> ctypes.CDLL:
         "kvc_slot_pool_release": (ci, [vp, u32]),
         "kvc_slot_pool_cancel": (ci, [vp, u32]),
         "kvc_slot_pool_get_counters": (ci, [vp, P(kvc_slot_pool_counters)]),
+        "kvc_slot_pool_slot_info": (ci, [vp, u32, P(u32), P(u32), P(u64), P(ci)]),
+        "kvc_staging_ring_set_policy": (ci, [vp, u32, u32, ci]),
+        "kvc_staging_ring_acquire_for": (ci, [vp, ci, u64, i64, P(u32), P(vp), P(vp), P(ci)]),
+        "kvc_staging_ring_slot_filled": (ci, [vp, u32, P(ci)]),
+        "kvc_staging_ring_cancel": (ci, [vp, u32]),
+        "kvc_staging_ring_abandon": (ci, [vp, u32]),
+        "kvc_staging_ring_policy_counters": (ci, [vp, P(kvc_slot_pool_counters)]),
         "kvc_store_open": (ci, [ctypes.c_char_p, ctypes.c_char_p, ci, P(vp)]),
         "kvc_store_close": (ci, [vp]),
         "kvc_store_path": (ci, [vp, u64, ctypes.c_char_p, u32]),
@@ -686,6 +713,45 @@ def kvc_pipeline_load(layout, ring, store, ids, hashes, io_threads: int = 0,
                      use_copy_engine, stream)
 
 
+def kvc_pipeline_load_many(layout, ring, store, requests: Sequence[dict], io_threads: int = 0,
+                           stream=None) -> Tuple[dict, List[dict]]:
+    """Serve several requests at once from a ring in pool mode.  Each request is a dict with
+    'hashes', 'cls' (KVC_CLASS_DEMAND_LOAD / KVC_CLASS_PRELOAD) and, for demand loads, 'ids'
+    (a preload gives 'n_blocks' instead).  Returns (stats, [{'loaded_chunks', 'ready_seconds'}])."""
+    n = len(requests)
+    arr = (kvc_load_request * max(1, n))()
+    keep = []
+    for i, q in enumerate(requests):
+        hs = np.ascontiguousarray(np.asarray(q["hashes"], dtype=np.uint64))
+        keep.append(hs)
+        arr[i].hashes, arr[i].n_hashes, arr[i].cls = hs.ctypes.data, hs.size, int(q["cls"])
+        if q.get("ids") is not None:
+            k, p, cnt, dev = _ids(q["ids"])
+            if dev:
+                raise TypeError("the pipelines take host-resident ids")
+            keep.append(k)
+            arr[i].ids, arr[i].n_blocks = p, cnt
+        else:
+            arr[i].ids, arr[i].n_blocks = None, int(q["n_blocks"])
+    stats = kvc_load_many_stats()
+    st = lib().kvc_pipeline_load_many(layout.handle, ring.handle, store.handle, arr, n, io_threads,
+                                      _stream(stream), ctypes.byref(stats))
+    _check(st, "kvc_pipeline_load_many")
+    return ({k: getattr(stats, k) for k, _ in kvc_load_many_stats._fields_},
+            [{"loaded_chunks": arr[i].loaded_chunks, "ready_seconds": arr[i].ready_seconds}
+             for i in range(n)])
+
+
+def kvc_store_get_counters(store) -> dict:
+    c = kvc_store_counters()
+    _check(lib().kvc_store_get_counters(store.handle, ctypes.byref(c)), "kvc_store_get_counters")
+    return {k: getattr(c, k) for k, _ in kvc_store_counters._fields_}
+
+
+def kvc_staging_ring_pool_mode(ring) -> bool:
+    return bool(lib().kvc_staging_ring_pool_mode(ring.handle))
+
+
 # ------------------------------------------------------------------ slot policy
 class SlotPoolHandle:
     """Owns a ``kvc_slot_pool*``."""
@@ -741,6 +807,58 @@ def kvc_slot_pool_cancel(pool, slot: int) -> None:
 def kvc_slot_pool_get_counters(pool) -> dict:
     c = kvc_slot_pool_counters()
     _check(lib().kvc_slot_pool_get_counters(pool.handle, ctypes.byref(c)), "kvc_slot_pool_get_counters")
+    return {k: getattr(c, k) for k, _ in kvc_slot_pool_counters._fields_}
+
+
+KVC_SLOT_FREE, KVC_SLOT_IN_FLIGHT, KVC_SLOT_STAGED, KVC_SLOT_RETAINED = 0, 1, 2, 3
+
+
+def kvc_slot_pool_slot_info(pool, slot: int) -> Tuple[int, int, int, bool]:
+    """(state, references, key, unclaimed preload?) of one slot."""
+    st, refs, key, spec = ctypes.c_uint32(), ctypes.c_uint32(), ctypes.c_uint64(), ctypes.c_int()
+    _check(lib().kvc_slot_pool_slot_info(pool.handle, slot, ctypes.byref(st), ctypes.byref(refs),
+                                         ctypes.byref(key), ctypes.byref(spec)), "kvc_slot_pool_slot_info")
+    return st.value, refs.value, key.value, bool(spec.value)
+
+
+# ------------------------------------------------------------------ staging pool mode
+def kvc_staging_ring_set_policy(ring, foreground_reserve: int, max_speculative: int = 1,
+                                retain_completed: bool = False) -> None:
+    _check(lib().kvc_staging_ring_set_policy(ring.handle, foreground_reserve, max_speculative,
+                                             int(retain_completed)), "kvc_staging_ring_set_policy")
+
+
+def kvc_staging_ring_acquire_for(ring, cls: int, key: int, timeout_us: int = 0):
+    """(slot, device address, host address or 0, joined), or None when nothing is available for
+    this class (timeout_us == 0).  Raises KvcError(TIMEOUT) after a positive timeout."""
+    slot, dp, hp, j = ctypes.c_uint32(), ctypes.c_void_p(), ctypes.c_void_p(), ctypes.c_int()
+    st = lib().kvc_staging_ring_acquire_for(ring.handle, cls, key, timeout_us, ctypes.byref(slot),
+                                            ctypes.byref(dp), ctypes.byref(hp), ctypes.byref(j))
+    if st == KVC_ERR_WOULD_BLOCK:
+        return None
+    _check(st, "kvc_staging_ring_acquire_for")
+    return slot.value, int(dp.value or 0), int(hp.value or 0), bool(j.value)
+
+
+def kvc_staging_ring_slot_filled(ring, slot: int) -> bool:
+    f = ctypes.c_int()
+    _check(lib().kvc_staging_ring_slot_filled(ring.handle, slot, ctypes.byref(f)),
+           "kvc_staging_ring_slot_filled")
+    return bool(f.value)
+
+
+def kvc_staging_ring_cancel(ring, slot: int) -> None:
+    _check(lib().kvc_staging_ring_cancel(ring.handle, slot), "kvc_staging_ring_cancel")
+
+
+def kvc_staging_ring_abandon(ring, slot: int) -> None:
+    _check(lib().kvc_staging_ring_abandon(ring.handle, slot), "kvc_staging_ring_abandon")
+
+
+def kvc_staging_ring_policy_counters(ring) -> dict:
+    c = kvc_slot_pool_counters()
+    _check(lib().kvc_staging_ring_policy_counters(ring.handle, ctypes.byref(c)),
+           "kvc_staging_ring_policy_counters")
     return {k: getattr(c, k) for k, _ in kvc_slot_pool_counters._fields_}
 
 

@@ -290,6 +290,124 @@ def test_ring_streams_a_request_larger_than_itself(fake_events):
     kvc.kvc_staging_ring_destroy(ring)
 
 
+def _pool_ring(n, sb, reserve, max_spec=1, retain=False):
+    mem = np.zeros(n * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    ring = kvc.kvc_staging_ring_create(sb, n, kvc.KVC_RING_DEVICE, base, n * sb)
+    kvc.kvc_staging_ring_set_policy(ring, reserve, max_spec, retain)
+    ring._mem = mem
+    return ring, base
+
+
+def test_pool_mode_any_free_slot_and_events_gate_reuse(fake_events):
+    """Pool mode (Sec. 6.4 / 6.5): slots leave in any order, a slow slot holds up nobody, and a
+    slot goes back to the policy only once the event behind its last consumer has completed."""
+    D, S, P = kvc.KVC_CLASS_DEMAND_LOAD, kvc.KVC_CLASS_STORE, kvc.KVC_CLASS_PRELOAD
+    ring, base = _pool_ring(4, 4096, reserve=1)
+    with pytest.raises(kvc.KvcError) as e:                          # FIFO acquisition is off
+        kvc.kvc_staging_ring_acquire(ring)
+    assert e.value.status == kvc.KVC_ERR_STATE
+    a = kvc.kvc_staging_ring_acquire_for(ring, D, 100)
+    b = kvc.kvc_staging_ring_acquire_for(ring, S, 101)
+    c = kvc.kvc_staging_ring_acquire_for(ring, D, 102)
+    assert [x[0] for x in (a, b, c)] == [0, 1, 2] and not any(x[3] for x in (a, b, c))
+    assert a[1] == base and c[1] == base + 2 * 4096
+    # slot 0 is slow (its read never finishes in this test); slots 1 and 2 complete and are reused
+    for slot in (1, 2):
+        kvc.kvc_staging_ring_commit(ring, slot, 7)
+        kvc.kvc_staging_ring_wait_filled(ring, slot, 8)
+        kvc.kvc_staging_ring_release(ring, slot, 8)
+    d = kvc.kvc_staging_ring_acquire_for(ring, D, 103)
+    assert d[0] == 3                                                 # the last free slot
+    # released slots are not reusable before their events complete: nothing is left
+    assert kvc.kvc_staging_ring_acquire_for(ring, D, 104) is None
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_acquire_for(ring, D, 104, timeout_us=2000)
+    assert e.value.status == kvc.KVC_ERR_TIMEOUT
+    fake_events.complete_all()
+    e1 = kvc.kvc_staging_ring_acquire_for(ring, D, 104)
+    e2 = kvc.kvc_staging_ring_acquire_for(ring, S, 105)
+    assert sorted([e1[0], e2[0]]) == [1, 2]                          # while slot 0 is still held
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["n_free"], c["n_in_flight"], c["acquires"]) == (0, 4, 6)
+    # more releases than references are refused
+    kvc.kvc_staging_ring_commit_host(ring, 0)
+    kvc.kvc_staging_ring_release(ring, 0, 8)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_release(ring, 0, 8)
+    assert e.value.status == kvc.KVC_ERR_STATE
+    kvc.kvc_staging_ring_destroy(ring)
+
+
+def test_pool_mode_reserve_join_claim_and_shared_release(fake_events):
+    D, S, P = kvc.KVC_CLASS_DEMAND_LOAD, kvc.KVC_CLASS_STORE, kvc.KVC_CLASS_PRELOAD
+    ring, base = _pool_ring(4, 4096, reserve=2, max_spec=2)
+    p1 = kvc.kvc_staging_ring_acquire_for(ring, P, 1)
+    p2 = kvc.kvc_staging_ring_acquire_for(ring, P, 2)
+    assert p1[0] == 0 and p2[0] == 1
+    assert kvc.kvc_staging_ring_acquire_for(ring, P, 3) is None      # the reserve is for foreground work
+    # a demand load for key 1 joins the preload that is still being read, and claims it
+    j = kvc.kvc_staging_ring_acquire_for(ring, D, 1)
+    assert j[0] == 0 and j[3] is True
+    assert kvc.kvc_staging_ring_slot_filled(ring, 0) is False
+    with pytest.raises(kvc.KvcError) as e:                           # claimed: no longer cancellable
+        kvc.kvc_staging_ring_cancel(ring, 0)
+    assert e.value.status == kvc.KVC_ERR_STATE
+    kvc.kvc_staging_ring_cancel(ring, 1)                             # the unclaimed one is
+    assert kvc.kvc_staging_ring_policy_counters(ring)["cancels"] == 1
+    kvc.kvc_staging_ring_commit_host(ring, 0)                        # the read finished
+    assert kvc.kvc_staging_ring_slot_filled(ring, 0) is True
+    kvc.kvc_staging_ring_release_host(ring, 0)                       # the preloader's reference
+    kvc.kvc_staging_ring_wait_filled(ring, 0, 5)
+    kvc.kvc_staging_ring_release(ring, 0, 5)                         # the demand load's, after its unpack
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["joins"], c["claims"], c["n_staged"], c["n_free"]) == (1, 1, 1, 3)   # event not complete yet
+    fake_events.complete_all()
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["n_staged"], c["n_free"]) == (0, 4)
+    # two consumers on different streams share a slot: the event is re-recorded behind each
+    a = kvc.kvc_staging_ring_acquire_for(ring, D, 9)
+    b = kvc.kvc_staging_ring_acquire_for(ring, D, 9)
+    assert b[0] == a[0] and b[3]
+    kvc.kvc_staging_ring_commit(ring, a[0], 3)
+    n0 = len(fake_events.recorded)
+    kvc.kvc_staging_ring_release(ring, a[0], 5)
+    kvc.kvc_staging_ring_release(ring, a[0], 6)
+    assert [s for _, s in fake_events.recorded[n0:]] == [5, 6]
+    assert kvc.kvc_staging_ring_policy_counters(ring)["n_free"] == 3
+    fake_events.complete_all()
+    assert kvc.kvc_staging_ring_policy_counters(ring)["n_free"] == 4
+    # abandon: an acquired slot that will not be filled goes back at once
+    x = kvc.kvc_staging_ring_acquire_for(ring, S, 77)
+    kvc.kvc_staging_ring_abandon(ring, x[0])
+    assert kvc.kvc_staging_ring_policy_counters(ring)["n_free"] == 4
+    kvc.kvc_staging_ring_destroy(ring)
+
+
+def test_pool_mode_finished_preload_is_kept_then_claimed_or_taken_over(fake_events):
+    D, S, P = kvc.KVC_CLASS_DEMAND_LOAD, kvc.KVC_CLASS_STORE, kvc.KVC_CLASS_PRELOAD
+    ring, base = _pool_ring(3, 4096, reserve=1, max_spec=2)
+    for key in (1, 2):
+        s, dp, hp, j = kvc.kvc_staging_ring_acquire_for(ring, P, key)
+        kvc.kvc_staging_ring_commit_host(ring, s)
+        kvc.kvc_staging_ring_release_host(ring, s)                   # finished preloads wait unclaimed
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["n_staged"], c["n_free"]) == (2, 1)
+    s, dp, hp, j = kvc.kvc_staging_ring_acquire_for(ring, D, 2)      # the request arrives: no read
+    assert j and kvc.kvc_staging_ring_slot_filled(ring, s)
+    d1 = kvc.kvc_staging_ring_acquire_for(ring, D, 50)               # last free slot
+    d2 = kvc.kvc_staging_ring_acquire_for(ring, D, 51)               # takes over the unclaimed preload (key 1)
+    assert d1[0] == 2 and d2[0] == 0 and not d2[3]
+    assert kvc.kvc_staging_ring_slot_filled(ring, 0) is False        # to be filled anew
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["claims"], c["reclaims"]) == (1, 1)
+    # policy can only be replaced while everything is free
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_staging_ring_set_policy(ring, 0)
+    assert e.value.status == kvc.KVC_ERR_STATE
+    kvc.kvc_staging_ring_destroy(ring)
+
+
 def test_ring_create_validation(fake_events):
     for args, want in [((4096, 0, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
                        ((0, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),

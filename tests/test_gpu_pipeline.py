@@ -66,3 +66,143 @@ def test_store_then_load_through_files(tmp_path, use_copy_engine):
         kvc.kvc_pipeline_store(lay, dring, store, src, hashes)
     assert e.value.status == kvc.KVC_ERR_INVALID_ARG
     assert kvc.kvc_staging_ring_stats(dring)[0] == 0
+
+
+def _hashes(seed, n_chunks, shared=0, shared_seed=999):
+    """Chain hashes (Sec. 2.1) of a request whose first `shared` chunks hold a common prefix."""
+    out, h = [], 0
+    for c in range(n_chunks):
+        rng = np.random.default_rng((shared_seed if c < shared else seed) * 1000 + c)
+        h = kvc.kvc_chain_hash(h, rng.integers(0, 50000, 256).astype(np.int32))
+        out.append(h)
+    return out
+
+
+@pytest.mark.parametrize("pool_mode", [False, True])
+def test_failing_pack_inside_the_store_pipeline_returns_every_slot(tmp_path, pool_mode):
+    """An out-of-range block id in the third chunk: the call reports OUT_OF_RANGE, no slot stays
+    taken, and the next store on the same ring runs normally."""
+    g = orc.Dims(4, 2, 96, 16, 8, 128, 2)
+    pool = wl.random_bits(701, g.pool_bytes)
+    pool_t = torch.from_numpy(pool).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    ring = kvc.kvc_staging_ring_create(cb, 3, kvc.KVC_RING_HOST_MAPPED)
+    if pool_mode:
+        kvc.kvc_staging_ring_set_policy(ring, 1)
+    store = kvc.kvc_store_open(str(tmp_path), "m", direct_io=True)
+    src = wl.block_ids(73, g.NB, 80)                       # 5 chunks
+    bad = src.copy()
+    bad[37] = g.NB                                         # inside chunk 2
+    hashes = _hashes(1, 5)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_pipeline_store(lay, ring, store, bad, hashes, io_threads=2)
+    assert e.value.status == kvc.KVC_ERR_OUT_OF_RANGE
+    torch.cuda.synchronize()
+    if pool_mode:
+        c = kvc.kvc_staging_ring_policy_counters(ring)
+        assert (c["n_free"], c["n_in_flight"], c["n_staged"]) == (3, 0, 0)
+    else:
+        assert kvc.kvc_staging_ring_stats(ring)[0] == 0
+    # chunks before the failure may have been published; none after it
+    assert kvc.kvc_store_lookup(store, hashes[3]) is None and kvc.kvc_store_lookup(store, hashes[4]) is None
+    st = kvc.kvc_pipeline_store(lay, ring, store, src, hashes, io_threads=2)
+    assert st["chunks"] == 5 and st["published"] + st["already_present"] == 5
+    want = orc.pack_request(g, pool, src, 256)
+    for c, hh in enumerate(hashes):
+        assert np.array_equal(np.fromfile(kvc.kvc_store_path(store, hh), dtype=np.uint8), want[c])
+    # the same for loads: a bad destination id in the second chunk
+    dst = wl.block_ids(74, g.NB, 80)
+    bad = dst.copy()
+    bad[20] = -5
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_pipeline_load(lay, ring, store, bad, hashes, io_threads=2)
+    assert e.value.status == kvc.KVC_ERR_OUT_OF_RANGE
+    torch.cuda.synchronize()
+    if pool_mode:
+        c = kvc.kvc_staging_ring_policy_counters(ring)
+        assert (c["n_free"], c["n_in_flight"], c["n_staged"]) == (3, 0, 0)
+    else:
+        assert kvc.kvc_staging_ring_stats(ring)[0] == 0
+    pool_t.copy_(torch.from_numpy(pool))
+    ld = kvc.kvc_pipeline_load(lay, ring, store, dst, hashes, io_threads=2)
+    torch.cuda.synchronize()
+    assert ld["chunks"] == 5
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, want, dst, 256)
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+def test_four_requests_sharing_a_prefix_are_served_from_one_pool(tmp_path):
+    """Four requests whose first 1024 tokens (4 chunks) are the same prefix, loaded at once through
+    files and one staging pool (Sec. 6.5): every shared chunk is read once and joined by the other
+    three requests, every request's blocks equal the oracle's, and chunks preloaded by an earlier
+    call are claimed by the demand loads instead of being read again."""
+    g = orc.Dims(4, 2, 400, 16, 8, 128, 2)                 # 8B shape cut to 4 layers; chunk = 4 MiB
+    pool = wl.random_bits(702, g.pool_bytes)
+    pool_t = torch.from_numpy(pool).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    store = kvc.kvc_store_open(str(tmp_path), "m", direct_io=True)
+    # what is in the store: a "source" request per stored request, all with the same first 64 blocks
+    perm = np.random.default_rng(8).permutation(g.NB).astype(np.int32)
+    shared_src = perm[:64]
+    lens = [64 + 40, 64 + 16, 64 + 75, 64]                 # blocks; two ragged tails, one prefix-only
+    srcs, cur = [], 64
+    for n in lens:
+        srcs.append(np.ascontiguousarray(np.concatenate([shared_src, perm[cur:cur + n - 64]])))
+        cur += n - 64
+    hashes = [_hashes(10 + r, kvc.kvc_layout_num_chunks(lay, n), shared=4) for r, n in enumerate(lens)]
+    fifo = kvc.kvc_staging_ring_create(cb, 4, kvc.KVC_RING_HOST_MAPPED)
+    for r in range(4):
+        kvc.kvc_pipeline_store(lay, fifo, store, srcs[r], hashes[r], io_threads=3)
+    kvc.kvc_staging_ring_destroy(fifo)
+    want_chunks = [orc.pack_request(g, pool, s, 256) for s in srcs]
+    n_files = len({h for hs in hashes for h in hs})
+    assert kvc.kvc_store_get_counters(store)["publishes"] == n_files == 4 + 3 + 1 + 5
+    # destination blocks: distinct for every request
+    dsts = []
+    for n in lens:
+        dsts.append(np.ascontiguousarray(perm[cur:cur + n]))
+        cur += n
+    assert cur <= g.NB
+    want_pool = pool.copy()
+    for r in range(4):
+        orc.unpack_request(g, want_pool, want_chunks[r], dsts[r], 256)
+
+    ring = kvc.kvc_staging_ring_create(cb, 6, kvc.KVC_RING_HOST_MAPPED)
+    kvc.kvc_staging_ring_set_policy(ring, foreground_reserve=2, max_speculative=4)
+    reads0 = kvc.kvc_store_get_counters(store)["reads"]
+    # 1. a preload of request 2's prefix, issued before anything is scheduled
+    stats, res = kvc.kvc_pipeline_load_many(lay, ring, store, [
+        dict(hashes=hashes[2], n_blocks=lens[2], cls=kvc.KVC_CLASS_PRELOAD)], io_threads=3)
+    staged = res[0]["loaded_chunks"]
+    assert 1 <= staged <= 4                                  # bounded by the reserve: 6 slots - 2
+    assert stats["reads"] == staged and stats["unpack_launches"] == 0
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert c["n_staged"] == staged and c["n_in_flight"] == 0
+    # 2. all four requests as demand loads in one call
+    reqs = [dict(ids=dsts[r], hashes=hashes[r], cls=kvc.KVC_CLASS_DEMAND_LOAD) for r in range(4)]
+    stats, res = kvc.kvc_pipeline_load_many(lay, ring, store, reqs, io_threads=3)
+    torch.cuda.synchronize()
+    assert [x["loaded_chunks"] for x in res] == [kvc.kvc_layout_num_chunks(lay, n) for n in lens]
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    total_pairs = sum(kvc.kvc_layout_num_chunks(lay, n) for n in lens)
+    assert stats["chunks"] == total_pairs
+    # every file is read at most once over both calls; the shared chunks exactly once
+    reads = kvc.kvc_store_get_counters(store)["reads"] - reads0
+    assert reads == n_files
+    assert stats["reads"] == n_files - staged
+    assert stats["joins"] == total_pairs - stats["reads"]
+    assert stats["claims"] >= 1                              # the preload was claimed, not re-read
+    assert stats["unpack_launches"] <= stats["reads"] + 2   # fused: never one launch per (request, chunk)
+    assert all(x["ready_seconds"] > 0 for x in res)
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["n_free"], c["n_in_flight"], c["n_staged"]) == (6, 0, 0)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+    # a FIFO ring is refused by the many-request call
+    fifo = kvc.kvc_staging_ring_create(cb, 2, kvc.KVC_RING_HOST_MAPPED)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_pipeline_load_many(lay, fifo, store, reqs)
+    assert e.value.status == kvc.KVC_ERR_STATE
