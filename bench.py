@@ -921,6 +921,92 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
             "ring_slots": int(w.extra["ring_slots"]), "slot_bytes": cb, "runs": results}
 
 
+def suite_duplex(torch, kvc, cuda_rt, dev, reps):
+    """Sec. 6.4: loads, stores and preloads share one staging pool.  Request A (32k tokens, 8B shape,
+    4 GiB) is offloaded to pinned host memory while request B (same size) is loaded from pinned host
+    memory, through ONE 8-slot pool, chunk by chunk in alternation, each direction on its own kernel
+    and copy stream.  Reported against the duplex ceiling of the host link measured in the same
+    process (two 1 GiB cudaMemcpyAsync, one per direction, running at once)."""
+    w = wl.WORKLOADS["8b_ring"]
+    s, NB, n = w.shape, w.pool_blocks, w.request_blocks // 2
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    perm = wl.block_ids(w.seed, NB, NB)
+    ids_a, ids_b = perm[:n], np.ascontiguousarray(perm[n:2 * n])
+    one_way = n * s.bytes_per_block
+    host_a = torch.empty(one_way, dtype=torch.uint8, pin_memory=True)
+    host_b = torch.empty(one_way, dtype=torch.uint8, pin_memory=True)
+    s_pack, s_d2h, s_h2d, s_unpack = (torch.cuda.Stream() for _ in range(4))
+    # duplex ceiling
+    nb1 = 1 << 30
+    dbuf = torch.empty(2 * nb1, dtype=torch.uint8, device=dev)
+    best = None
+    for _ in range(6):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        torch.cuda.synchronize()
+        e[0].record(s_d2h)
+        e[2].record(s_h2d)
+        cuda_rt.memcpy_async(host_a.data_ptr(), dbuf.data_ptr(), nb1, cuda_rt.D2H, s_d2h)
+        cuda_rt.memcpy_async(dbuf.data_ptr() + nb1, host_b.data_ptr(), nb1, cuda_rt.H2D, s_h2d)
+        e[1].record(s_d2h)
+        e[3].record(s_h2d)
+        torch.cuda.synchronize()
+        t = max(e[0].elapsed_time(e[1]), e[2].elapsed_time(e[3]))
+        cand = {"d2h_gbs": nb1 / e[0].elapsed_time(e[1]) / 1e6, "h2d_gbs": nb1 / e[2].elapsed_time(e[3]) / 1e6,
+                "aggregate_gbs": 2 * nb1 / t / 1e6}
+        if best is None or cand["aggregate_gbs"] > best["aggregate_gbs"]:
+            best = cand
+    del dbuf
+    out = {"prefix_bytes_each_direction": one_way, "duplex_ceiling": best, "runs": []}
+    TO = 20_000_000
+    for kind, kind_name in ((kvc.KVC_RING_DEVICE, "device slots + cudaMemcpyAsync"),
+                            (kvc.KVC_RING_HOST_MAPPED, "mapped pinned host slots (kernels cross the link)")):
+        lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+        descs = kvc.kvc_map_request(lay, n)
+        cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+        ring = kvc.kvc_staging_ring_create(cb, int(w.extra["ring_slots"]), kind)
+        kvc.kvc_staging_ring_set_policy(ring, 0)
+
+        def both():
+            off = 0
+            for (_, c, first, nb, nbytes) in descs:
+                slot, dptr, hp, _ = kvc.kvc_staging_ring_acquire_for(ring, kvc.KVC_CLASS_STORE, 2 * c, TO)
+                kvc.kvc_pack(lay, ids_a[first:first + nb], dptr, nbytes, stream=s_pack)
+                kvc.kvc_staging_ring_commit(ring, slot, s_pack)
+                kvc.kvc_staging_ring_wait_filled(ring, slot, s_d2h)
+                if kind == kvc.KVC_RING_DEVICE:
+                    cuda_rt.memcpy_async(host_a.data_ptr() + off, dptr, nbytes, cuda_rt.D2H, s_d2h)
+                kvc.kvc_staging_ring_release(ring, slot, s_d2h)
+                slot, dptr, hp, _ = kvc.kvc_staging_ring_acquire_for(ring, kvc.KVC_CLASS_DEMAND_LOAD,
+                                                                     2 * c + 1, TO)
+                if kind == kvc.KVC_RING_DEVICE:
+                    cuda_rt.memcpy_async(dptr, host_b.data_ptr() + off, nbytes, cuda_rt.H2D, s_h2d)
+                kvc.kvc_staging_ring_commit(ring, slot, s_h2d)
+                kvc.kvc_staging_ring_wait_filled(ring, slot, s_unpack)
+                kvc.kvc_unpack(lay, dptr, ids_b[first:first + nb], nbytes, stream=s_unpack)
+                kvc.kvc_staging_ring_release(ring, slot, s_unpack)
+                off += nbytes
+
+        both()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(max(3, reps // 4)):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            both()
+            torch.cuda.synchronize()
+            ts.append(time.perf_counter() - t0)
+        t = statistics.median(ts)
+        c = kvc.kvc_staging_ring_policy_counters(ring)
+        out["runs"].append({"slots": kind_name, "seconds": t, "per_direction_gbs": one_way / t / 1e9,
+                            "aggregate_gbs": 2 * one_way / t / 1e9,
+                            "frac_of_duplex_ceiling": 2 * one_way / t / 1e9 / best["aggregate_gbs"],
+                            "acquires": c["acquires"]})
+        assert kvc.kvc_poll_device_status(lay) == (0, 0)
+        kvc.kvc_staging_ring_destroy(ring)
+        kvc.kvc_layout_destroy(lay)
+    return out
+
+
 def suite_host_link(torch, cuda_rt, dev):
     """Host-link ceiling of this machine: cudaMemcpyAsync of 1 GiB of pinned memory, each direction,
     best of 10."""
@@ -988,6 +1074,103 @@ def suite_file_pipeline(torch, kvc, dev, root):
     return out
 
 
+def suite_preload_trace(torch, kvc, dev, roots):
+    """Sec. 6.5 in miniature: a queue of requests, each needing its 2048-token prefix (8 chunks of
+    32 MiB, 8B shape; the first 1024 tokens are common to all) loaded from chunk files before a
+    forward pass of ~40 ms (a matmul burst) can run.  Without preloading every request pays the file
+    reads on its critical path.  With preloading the NEXT request's chunks are read into the staging
+    pool while the current forward pass runs on the GPU, so its demand load finds them staged, claims
+    them and only the unpack remains.  One staging pool of 12 slots, 4 reserved for demand work."""
+    import shutil
+    import tempfile
+    w = wl.WORKLOADS["8b_ring"]
+    s, NB = w.shape, w.pool_blocks
+    n_req, n_blocks, shared_blocks = 10, 128, 64
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    perm = wl.block_ids(w.seed, NB, NB)
+    shared = perm[:shared_blocks]
+    srcs, dsts, cur = [], [], shared_blocks
+    for r in range(n_req):
+        srcs.append(np.ascontiguousarray(np.concatenate([shared, perm[cur:cur + n_blocks - shared_blocks]])))
+        cur += n_blocks - shared_blocks
+    for r in range(n_req):
+        dsts.append(np.ascontiguousarray(perm[cur:cur + n_blocks]))
+        cur += n_blocks
+    N = 8192
+    A = torch.randn(N, N, device=dev, dtype=torch.bfloat16)
+    B = torch.randn(N, N, device=dev, dtype=torch.bfloat16)
+    C = torch.empty(N, N, device=dev, dtype=torch.bfloat16)
+    s_fwd = torch.cuda.Stream()
+
+    def forward_pass():
+        with torch.cuda.stream(s_fwd):
+            for _ in range(50):
+                torch.matmul(A, B, out=C)
+
+    out = []
+    for base in roots.split(","):
+        if not os.path.isdir(base):
+            continue
+        d = tempfile.mkdtemp(prefix="kvc_trace_", dir=base)
+        try:
+            lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+            kvc.kvc_layout_set_tuning(lay, max_ctas=16)
+            cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+            store = kvc.kvc_store_open(d, "8b", direct_io=True)
+            hashes = []
+            for r in range(n_req):
+                hs, h = [], 0
+                for c in range(n_blocks // 16):
+                    tag = b"shared" if c < shared_blocks // 16 else b"req%d" % r
+                    h = kvc.kvc_fnv1a64(tag + b".%d.%d" % (c, h))
+                    hs.append(h)
+                hashes.append(hs)
+            fifo = kvc.kvc_staging_ring_create(cb, 8, kvc.KVC_RING_HOST_MAPPED)
+            for r in range(n_req):
+                kvc.kvc_pipeline_store(lay, fifo, store, srcs[r], hashes[r], io_threads=4)
+            kvc.kvc_staging_ring_destroy(fifo)
+            forward_pass()
+            torch.cuda.synchronize()
+            for preload in (False, True):
+                ring = kvc.kvc_staging_ring_create(cb, 12, kvc.KVC_RING_HOST_MAPPED)
+                kvc.kvc_staging_ring_set_policy(ring, foreground_reserve=4, max_speculative=8)
+                reads0 = kvc.kvc_store_get_counters(store)["reads"]
+                lat, joins, claims = [], 0, 0
+                t_start = time.perf_counter()
+                for r in range(n_req):
+                    t0 = time.perf_counter()
+                    st, res = kvc.kvc_pipeline_load_many(
+                        lay, ring, store, [dict(ids=dsts[r], hashes=hashes[r], cls=kvc.KVC_CLASS_DEMAND_LOAD)],
+                        io_threads=4)
+                    torch.cuda.current_stream().synchronize()
+                    lat.append(time.perf_counter() - t0)
+                    joins += st["joins"]
+                    claims = st["claims"]
+                    forward_pass()                      # asynchronous: the GPU is busy, the host is not
+                    if preload and r + 1 < n_req:
+                        kvc.kvc_pipeline_load_many(
+                            lay, ring, store,
+                            [dict(hashes=hashes[r + 1], n_blocks=n_blocks, cls=kvc.KVC_CLASS_PRELOAD)],
+                            io_threads=4)
+                    s_fwd.synchronize()
+                total = time.perf_counter() - t_start
+                out.append({"root": base, "preloading": preload, "requests": n_req,
+                            "prefix_bytes": n_blocks * s.bytes_per_block,
+                            "demand_load_ms_mean": statistics.mean(lat) * 1e3,
+                            "demand_load_ms_median": statistics.median(lat) * 1e3,
+                            "demand_load_ms_first": lat[0] * 1e3, "total_s": total,
+                            "file_reads": kvc.kvc_store_get_counters(store)["reads"] - reads0,
+                            "joins": joins, "claims": claims})
+                torch.cuda.synchronize()
+                kvc.kvc_staging_ring_destroy(ring)
+            assert kvc.kvc_poll_device_status(lay) == (0, 0)
+            kvc.kvc_store_close(store)
+            kvc.kvc_layout_destroy(lay)
+        finally:
+            shutil.rmtree(d, ignore_errors=True)
+    return out
+
+
 def run_suite(args):
     import torch
     from paper_2609_11744_b200 import cuda_rt, kvc
@@ -1007,7 +1190,9 @@ def run_suite(args):
                      ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
                      ("ring_overlap", lambda: suite_ring_overlap(torch, kvc, cuda_rt, dev,
                                                                  args.overlap_seconds)),
-                     ("file_pipeline", lambda: suite_file_pipeline(torch, kvc, dev, args.file_roots))):
+                     ("duplex", lambda: suite_duplex(torch, kvc, cuda_rt, dev, args.steps)),
+                     ("file_pipeline", lambda: suite_file_pipeline(torch, kvc, dev, args.file_roots)),
+                     ("preload_trace", lambda: suite_preload_trace(torch, kvc, dev, args.file_roots))):
         if "all" in parts or name in parts:
             out[name] = fn()
             torch.cuda.synchronize()
@@ -1040,7 +1225,7 @@ def main():
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
                          "host_link,launch_shapes,chunk_sweep,small_slabs,call_overhead,prefix_8k,batch_70b,"
-                         "ring_overlap,file_pipeline (1 GPU; prints one JSON line)")
+                         "ring_overlap,duplex,file_pipeline,preload_trace (1 GPU; prints one JSON line)")
     ap.add_argument("--small-slab-sizes", default="",
                     help="small_slabs suite part: comma list of slab sizes in bytes (default: all)")
     ap.add_argument("--small-slab-mib", type=int, default=2048,

@@ -356,8 +356,8 @@ kvc_status kvc_staging_ring_release(kvc_ring *ring, uint32_t slot, void *consume
 kvc_status kvc_staging_ring_commit_host(kvc_ring *ring, uint32_t slot);
 kvc_status kvc_staging_ring_sync_filled(kvc_ring *ring, uint32_t slot);
 kvc_status kvc_staging_ring_release_host(kvc_ring *ring, uint32_t slot);
-/* in_flight = slots acquired and not yet observed free; stalls = acquire polls that found the
- * next slot still busy.  Any pointer may be NULL. */
+/* in_flight = slots that are not free right now (the events of released slots are queried);
+ * stalls = acquire polls that found the next slot still busy.  Any pointer may be NULL. */
 kvc_status kvc_staging_ring_stats(const kvc_ring *ring, uint32_t *in_flight, uint64_t *acquires,
                                   uint64_t *stalls);
 /* Slot transitions with host timestamps, for timelines of a transfer (the paper traces its

@@ -452,9 +452,16 @@ kvc_status kvc_staging_ring_stats(const kvc_ring *r, uint32_t *in_flight, uint64
     if (!r)
         return KVC_ERR_INVALID_ARG;
     if (in_flight) {
+        // released slots whose event has completed meanwhile count as free: ask the events
+        kvc_ring *rw = const_cast<kvc_ring *>(r);
+        if (rw->policy)
+            (void)reap_deferred(rw);
         uint32_t n = 0;
-        for (const Slot &s : r->slots)
+        for (Slot &s : rw->slots) {
+            if (s.state == SLOT_DRAINING)
+                (void)slot_is_free(rw, s);
             n += s.state != SLOT_FREE;
+        }
         *in_flight = n;
     }
     if (acquires)

@@ -184,3 +184,69 @@ def test_first_launches_of_two_handles_race_on_two_threads():
         torch.cuda.synchronize()
         for o in outs:
             assert np.array_equal(o.cpu().numpy(), want)
+
+
+@pytest.mark.parametrize("kind", [kvc.KVC_RING_DEVICE, kvc.KVC_RING_HOST_MAPPED])
+def test_offload_and_load_share_one_staging_pool_at_the_same_time(kind):
+    """Sec. 6.4: loads and stores draw from the same pool.  Request A is offloaded (pack -> slot ->
+    host) while request B is loaded (host -> slot -> unpack) through ONE 4-slot pool, chunk by
+    chunk in alternation, each direction on its own pair of streams.  Host bytes of A and the
+    blocks of B must equal the oracle's."""
+    w = wl.WORKLOADS["8b_ring"]
+    g = dims_of(w.shape, 384)
+    pool = _pool_8b_384()
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 256)
+    ids_a = wl.block_ids(31, g.NB, 150)                     # offloaded: 9 full chunks + 6 blocks
+    perm = wl.block_ids(32, g.NB, g.NB)
+    rest = np.array([b for b in perm if b not in set(ids_a.tolist())], dtype=np.int32)
+    ids_b = np.ascontiguousarray(rest[:120])                # loaded into blocks A does not read
+    src_b = wl.block_ids(33, g.NB, 120)                     # what B's chunks hold (packed by the oracle)
+    chunks_b = orc.pack_request(g, pool, src_b, 256)
+    host_b = torch.from_numpy(np.concatenate(chunks_b)).pin_memory()
+    want_a = np.concatenate(orc.pack_request(g, pool, ids_a, 256))
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, chunks_b, ids_b, 256)
+    host_a = torch.zeros(want_a.size, dtype=torch.uint8).pin_memory()
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    ring = kvc.kvc_staging_ring_create(cb, 4, kind)
+    kvc.kvc_staging_ring_set_policy(ring, foreground_reserve=0)
+    s_pack, s_d2h, s_h2d, s_unpack = (torch.cuda.Stream() for _ in range(4))
+    da, db = kvc.kvc_map_request(lay, len(ids_a)), kvc.kvc_map_request(lay, len(ids_b))
+    TO = 10_000_000
+    off_a = off_b = 0
+    for i in range(max(len(da), len(db))):
+        if i < len(da):
+            _, c, first, nb, nbytes = da[i]
+            slot, dptr, hptr, joined = kvc.kvc_staging_ring_acquire_for(ring, kvc.KVC_CLASS_STORE, 1000 + c, TO)
+            assert not joined
+            kvc.kvc_pack(lay, ids_a[first:first + nb], dptr, nbytes, stream=s_pack)
+            kvc.kvc_staging_ring_commit(ring, slot, s_pack)
+            kvc.kvc_staging_ring_wait_filled(ring, slot, s_d2h)
+            if kind == kvc.KVC_RING_DEVICE:
+                cuda_rt.memcpy_async(host_a.data_ptr() + off_a, dptr, nbytes, cuda_rt.D2H, s_d2h)
+            else:
+                cuda_rt.memcpy_async(host_a.data_ptr() + off_a, hptr, nbytes, cuda_rt.H2H, s_d2h)
+            kvc.kvc_staging_ring_release(ring, slot, s_d2h)
+            off_a += nbytes
+        if i < len(db):
+            _, c, first, nb, nbytes = db[i]
+            slot, dptr, hptr, joined = kvc.kvc_staging_ring_acquire_for(ring, kvc.KVC_CLASS_DEMAND_LOAD,
+                                                                        2000 + c, TO)
+            assert not joined
+            if kind == kvc.KVC_RING_DEVICE:
+                cuda_rt.memcpy_async(dptr, host_b.data_ptr() + off_b, nbytes, cuda_rt.H2D, s_h2d)
+            else:
+                cuda_rt.memcpy_async(hptr, host_b.data_ptr() + off_b, nbytes, cuda_rt.H2H, s_h2d)
+            kvc.kvc_staging_ring_commit(ring, slot, s_h2d)
+            kvc.kvc_staging_ring_wait_filled(ring, slot, s_unpack)
+            kvc.kvc_unpack(lay, dptr, ids_b[first:first + nb], nbytes, stream=s_unpack)
+            kvc.kvc_staging_ring_release(ring, slot, s_unpack)
+            off_b += nbytes
+    torch.cuda.synchronize()
+    assert np.array_equal(host_a.numpy(), want_a)
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["n_free"], c["acquires"]) == (4, len(da) + len(db))
+    kvc.kvc_staging_ring_destroy(ring)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)

@@ -139,7 +139,7 @@ def test_four_requests_sharing_a_prefix_are_served_from_one_pool(tmp_path):
     files and one staging pool (Sec. 6.5): every shared chunk is read once and joined by the other
     three requests, every request's blocks equal the oracle's, and chunks preloaded by an earlier
     call are claimed by the demand loads instead of being read again."""
-    g = orc.Dims(4, 2, 400, 16, 8, 128, 2)                 # 8B shape cut to 4 layers; chunk = 4 MiB
+    g = orc.Dims(4, 2, 640, 16, 8, 128, 2)                 # 8B shape cut to 4 layers; chunk = 4 MiB
     pool = wl.random_bits(702, g.pool_bytes)
     pool_t = torch.from_numpy(pool).to(DEV)
     lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256)
