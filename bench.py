@@ -40,6 +40,29 @@ import workloads as wl  # noqa: E402
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 METRIC = "pack+unpack GB/s (bytes read+written), 80k-token prefix, 8B KV shape"
+# DRAM bytes of one launch of the default workload, and where the figure comes from.  The capture
+# predates later edits of the kernel file; `kernel_file_sha256_at_capture` is compared with the file
+# as it is now and the line says whether they still match (a mismatch means: capture again).
+TRAFFIC_8B_80K = {
+    "bytes": 20_920_170_000.0,
+    "source": "profiles/kvc_bulk_kernel_8b_80k_dram_traffic.md",
+    "kernel_file": "paper_2609_11744_b200/csrc/kvc_kernels.cu",
+    "kernel_file_sha256_at_last_check": "b528a8cad9dd4a79956e3dfa7ad5a988ff000f81ad03ee6eac235525eea9939a",
+}
+
+
+def traffic_source_note():
+    """Where roofline.traffic comes from, and whether the kernel source still is the file the
+    figure was last checked against."""
+    import hashlib
+    try:
+        with open(os.path.join(ROOT, TRAFFIC_8B_80K["kernel_file"]), "rb") as f:
+            now = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        now = None
+    same = now == TRAFFIC_8B_80K["kernel_file_sha256_at_last_check"]
+    return "%s (kernel source %s since the last check of this figure)" % (
+        TRAFFIC_8B_80K["source"], "unchanged" if same else "CHANGED")
 
 
 def measured_peak():
@@ -301,28 +324,32 @@ def run_ours(args, rank, world, local_rank):
     if not args.no_e2e:
         e2e = run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, dist)
     peak, peak_kind = measured_peak()
-    traffic = args.traffic_bytes
+    traffic, traffic_source = args.traffic_bytes, "--traffic-bytes" if args.traffic_bytes else None
     if traffic is None and (args.workload, NB, n, args.chunk_tokens, args.variant) == \
             ("8b_80k", 20000, 5000, 256, 0):
         # dram__bytes_read.sum + dram__bytes_write.sum of one launch of this exact workload, from a
         # one-pass ncu capture (its summary is kept under profiles/): mean of the
         # pack launch (20,919,990,000) and the unpack launch (20,920,350,000)
-        traffic = 20_920_170_000.0
+        traffic = TRAFFIC_8B_80K["bytes"]
+        traffic_source = traffic_source_note()
     launch_ms = statistics.mean(pack_ms + unpack_ms)
     achieved = 2 * one_way / (launch_ms * 1e-3) / 1e9
     roof = {
         "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-        "traffic": traffic, "peak_kind": peak_kind,
+        "traffic": traffic, "traffic_source": traffic_source, "peak_kind": peak_kind,
         "kernel": "kvc_bulk_kernel (pack and unpack instantiations)" if args.variant != 1
                   else "kvc_vec_kernel (pack and unpack instantiations)",
         "algorithmic_bytes_per_launch": 2 * one_way,
         "avg_launch_ms": launch_ms,
         "pack": {"ms": statistics.mean(pack_ms), "min_ms": min(pack_ms),
+                 "median_ms": statistics.median(pack_ms), "max_ms": max(pack_ms),
                  "gbs": 2 * one_way / statistics.mean(pack_ms) / 1e6,
                  "frac": 2 * one_way / statistics.mean(pack_ms) / 1e6 / peak},
         "unpack": {"ms": statistics.mean(unpack_ms), "min_ms": min(unpack_ms),
+                   "median_ms": statistics.median(unpack_ms), "max_ms": max(unpack_ms),
                    "gbs": 2 * one_way / statistics.mean(unpack_ms) / 1e6,
                    "frac": 2 * one_way / statistics.mean(unpack_ms) / 1e6 / peak},
+        "per_step_ms": {"pack": [round(x, 4) for x in pack_ms], "unpack": [round(x, 4) for x in unpack_ms]},
         "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
     }
     if rank != 0:
@@ -594,8 +621,8 @@ def suite_small_slabs(torch, kvc, dev, reps, sizes=None, request_mib=2048):
     peak = measured_peak()[0]
     L, P, B = 32, 2, 16
     out = []
-    for S, H, D, e in ((32768, 8, 128, 2), (8192, 2, 128, 2), (4096, 1, 128, 2), (2048, 1, 128, 1),
-                       (1024, 1, 64, 1), (256, 1, 16, 1)):
+    for S, H, D, e in ((32768, 8, 128, 2), (16384, 4, 128, 2), (8192, 2, 128, 2), (4096, 1, 128, 2),
+                       (2048, 1, 128, 1), (1024, 1, 64, 1), (512, 1, 32, 1), (256, 1, 16, 1)):
         if sizes and S not in sizes:
             continue
         per_block = L * P * S

@@ -14,9 +14,9 @@
 #define KVC_VEC_THREADS 256u    // threads per block of the vector kernels
 #define KVC_VEC_UNROLL 4u       // vectors in flight per thread
 #define KVC_VEC_WARP_TEAM_MAX_TILE 4096u  // tiles up to this size are copied by one warp each
-// Slabs up to this size are moved several per work item by one warp (multi-slab vector kernel);
-// an item is about this many bytes.
-#define KVC_VEC_GROUP_MAX_SLAB 4096u
+// Slabs up to this size go through the multi-slab vector kernel, one warp per work item; an item
+// is about KVC_VEC_GROUP_ITEM_BYTES (several small slabs, or one slab of 8-16 KiB).
+#define KVC_VEC_GROUP_MAX_SLAB 16384u
 #define KVC_VEC_GROUP_ITEM_BYTES 8192u
 #define KVC_HOST_SLOT_DEFAULT_CTAS 16u
 #define KVC_BULK_THREADS 32u    // one warp drives the bulk-copy pipeline
