@@ -985,9 +985,13 @@ def suite_duplex(torch, kvc, cuda_rt, dev, reps):
     del dbuf
     out = {"prefix_bytes_each_direction": one_way, "duplex_ceiling": best, "runs": []}
     TO = 20_000_000
-    for kind, kind_name in ((kvc.KVC_RING_DEVICE, "device slots + cudaMemcpyAsync"),
-                            (kvc.KVC_RING_HOST_MAPPED, "mapped pinned host slots (kernels cross the link)")):
+    mapped = "mapped pinned host slots (kernels cross the link), %s blocks per kernel"
+    for kind, kind_name, ctas in ((kvc.KVC_RING_DEVICE, "device slots + cudaMemcpyAsync", 0),
+                                  (kvc.KVC_RING_HOST_MAPPED, mapped % "16 (default)", 0),
+                                  (kvc.KVC_RING_HOST_MAPPED, mapped % "32", 32),
+                                  (kvc.KVC_RING_HOST_MAPPED, mapped % "64", 64)):
         lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+        kvc.kvc_layout_set_tuning(lay, max_ctas=ctas)
         descs = kvc.kvc_map_request(lay, n)
         cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
         ring = kvc.kvc_staging_ring_create(cb, int(w.extra["ring_slots"]), kind)

@@ -665,6 +665,22 @@ def kvc_store_direct_io_refused(store) -> int:
     return lib().kvc_store_direct_io_refused(store.handle)
 
 
+_OPEN_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_char_p, ctypes.c_int, ctypes.c_uint, use_errno=True)
+_open_keep = None
+
+
+def kvc_store_set_open_fn(fn) -> None:
+    """Test seam: route every open() of the store through fn(path: bytes, flags, mode) -> fd or -1
+    (set errno with ctypes.set_errno before returning -1); None restores open(2)."""
+    global _open_keep
+    L = lib()
+    L.kvc_store_set_open_fn.argtypes = [_OPEN_FN]
+    L.kvc_store_set_open_fn.restype = ctypes.c_int
+    cb = ctypes.cast(None, _OPEN_FN) if fn is None else _OPEN_FN(fn)
+    _check(L.kvc_store_set_open_fn(cb), "kvc_store_set_open_fn")
+    _open_keep = None if fn is None else cb
+
+
 def kvc_chain_hash(prev: int, tokens) -> int:
     t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
     return lib().kvc_chain_hash(prev, t.ctypes.data, t.size)

@@ -408,6 +408,47 @@ def test_pool_mode_finished_preload_is_kept_then_claimed_or_taken_over(fake_even
     kvc.kvc_staging_ring_destroy(ring)
 
 
+def test_rings_created_on_several_threads_while_the_provider_is_replaced(fake_events):
+    """The event provider is process-wide state copied into a ring at creation.  Threads create,
+    use and destroy rings while another thread keeps re-installing the provider: every ring must
+    see one complete provider (never a half-written one) and work."""
+    import threading
+    errors = []
+    stop = threading.Event()
+
+    def churn():
+        p = fake_events.provider()
+        while not stop.is_set():
+            kvc.kvc_staging_ring_set_event_provider(p)
+
+    def worker(seed):
+        try:
+            for it in range(40):
+                mem = np.zeros(3 * 4096 + 64, dtype=np.uint8)
+                base = (mem.ctypes.data + 15) // 16 * 16
+                ring = kvc.kvc_staging_ring_create(4096, 3, kvc.KVC_RING_DEVICE, base, 3 * 4096)
+                for _ in range(3):
+                    slot, dp, _h = kvc.kvc_staging_ring_acquire(ring)
+                    kvc.kvc_staging_ring_commit(ring, slot, seed)
+                    kvc.kvc_staging_ring_wait_filled(ring, slot, seed + 1)
+                    kvc.kvc_staging_ring_release(ring, slot, seed + 1)
+                assert kvc.kvc_staging_ring_stats(ring)[1] == 3
+                kvc.kvc_staging_ring_destroy(ring)
+        except Exception as e:
+            errors.append(repr(e))
+
+    c = threading.Thread(target=churn)
+    ws = [threading.Thread(target=worker, args=(10 * i,)) for i in range(4)]
+    c.start()
+    for t in ws:
+        t.start()
+    for t in ws:
+        t.join(timeout=120)
+    stop.set()
+    c.join(timeout=30)
+    assert errors == []
+
+
 def test_ring_create_validation(fake_events):
     for args, want in [((4096, 0, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
                        ((0, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),

@@ -264,6 +264,22 @@ def test_lp_range_partition_is_the_whole():
     for lo, hi in [(0, 3), (3, 4), (4, 8)]:
         orc.pack_chunk_into(g, pool, ids, parts, (lo, hi))
     assert np.array_equal(whole, parts)
+    # unpack side: scattering the chunk plane range by plane range equals scattering it whole,
+    # and a single range touches only its own planes
+    before = rng.integers(0, 256, g.pool_bytes, dtype=np.uint8)
+    dst = rng.permutation(g.NB)[:5].astype(np.int32)
+    want = before.copy()
+    orc.unpack_chunk(g, want, whole, dst)
+    only = before.copy()
+    orc.unpack_chunk(g, only, whole, dst, (3, 4))
+    pb = g.NB * g.slab_bytes
+    assert np.array_equal(only[:3 * pb], before[:3 * pb]) and np.array_equal(only[4 * pb:], before[4 * pb:])
+    assert np.array_equal(only[3 * pb:4 * pb], want[3 * pb:4 * pb])
+    assert not np.array_equal(only[3 * pb:4 * pb], before[3 * pb:4 * pb])
+    pieces = before.copy()
+    for lo, hi in [(0, 3), (3, 4), (4, 8)]:
+        orc.unpack_chunk(g, pieces, whole, dst, (lo, hi))
+    assert np.array_equal(pieces, want)
 
 
 def test_out_of_range_ids_rejected():

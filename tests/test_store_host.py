@@ -121,7 +121,6 @@ def test_file_system_that_refuses_direct_io_falls_back_and_leaves_no_litter(tmp_
     must remove that empty file, retry with buffered I/O, count the refusal, publish the entry
     and leave no temporary name behind.  The refusal is played by an open() stand-in."""
     import ctypes
-    OPEN_FN = ctypes.CFUNCTYPE(ctypes.c_int, ctypes.c_char_p, ctypes.c_int, ctypes.c_uint, use_errno=True)
     libc = ctypes.CDLL(None, use_errno=True)
     libc.open.restype = ctypes.c_int
     libc.open.argtypes = [ctypes.c_char_p, ctypes.c_int, ctypes.c_uint]
@@ -141,13 +140,9 @@ def test_file_system_that_refuses_direct_io_falls_back_and_leaves_no_litter(tmp_
             ctypes.set_errno(ctypes.get_errno())
         return fd
 
-    hook = OPEN_FN(refusing_open)
-    L = kvc.lib()
-    L.kvc_store_set_open_fn.argtypes = [OPEN_FN]
-    L.kvc_store_set_open_fn.restype = ctypes.c_int
     st = kvc.kvc_store_open(str(tmp_path), "m", direct_io=True)
     try:
-        assert L.kvc_store_set_open_fn(hook) == 0
+        kvc.kvc_store_set_open_fn(refusing_open)
         data = _aligned(1 << 20, seed=11)
         assert kvc.kvc_store_publish(st, 0xabcdef, data) is True
         assert kvc.kvc_store_direct_io_refused(st) == 1 and len(refused) == 1
@@ -157,7 +152,7 @@ def test_file_system_that_refuses_direct_io_falls_back_and_leaves_no_litter(tmp_
         assert kvc.kvc_store_direct_io_refused(st) == 2
         assert kvc.kvc_store_publish(st, 0xabcdef, data) is False
     finally:
-        L.kvc_store_set_open_fn(ctypes.cast(None, OPEN_FN))
+        kvc.kvc_store_set_open_fn(None)
         kvc.kvc_store_close(st)
     leftovers = [f for _, _, fs in os.walk(str(tmp_path)) for f in fs if f.startswith(".tmp")]
     assert leftovers == []
