@@ -752,3 +752,45 @@ def test_plain_c_program_links_and_runs(tmp_path):
     assert build.returncode == 0, build.stderr
     run = subprocess.run([exe], capture_output=True, text=True, timeout=120)
     assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr
+
+
+def test_kernel_timing_and_slot_memory_hint():
+    """Diagnostics and hints do not change a byte: with kernel timing on, every launch is reported
+    with a positive duration; with the slot_memory hint the pointer query is skipped and the right
+    kernel family still runs for device slots (hint 1) and mapped host slots (hint 2)."""
+    g = dims_of(wl.LLAMA_8B, 384)
+    pool = _pool_8b_384()
+    pool_t = to_dev(pool)
+    ids = wl.block_ids(88, g.NB, 37)
+    want = np.concatenate(orc.pack_request(g, pool, ids, 256))
+    lay = dense_layout(pool_t, g, 256)
+    kvc.kvc_layout_set_tuning(lay, slot_memory=1)
+    kvc.kvc_layout_set_kernel_timing(lay, True)
+    out = torch.zeros(want.size, dtype=torch.uint8, device=DEV)
+    ops, keep, nbytes, dev = kvc.request_chunk_ops(lay, ids, out)
+    kvc.kvc_pack_batch(lay, ops, dev)
+    kvc.kvc_pack(lay, ids[:16], out[:kvc.kvc_layout_chunk_bytes(lay, 16)])
+    n, total, lo, hi = kvc.kvc_layout_kernel_time(lay)
+    assert n == 2 and 0 < lo <= hi and abs(total - (lo + hi)) < 1e-6
+    assert kvc.kvc_layout_kernel_time(lay)[0] == 0               # collected once
+    kvc.kvc_layout_set_kernel_timing(lay, False)
+    kvc.kvc_pack_batch(lay, ops, dev)
+    assert kvc.kvc_layout_kernel_time(lay)[0] == 0
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy(), want)
+    # mapped host slots with the hint
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    ring = kvc.kvc_staging_ring_create(cb, 1, kvc.KVC_RING_HOST_MAPPED)
+    kvc.kvc_layout_set_tuning(lay, slot_memory=2)
+    slot, dptr, hptr = kvc.kvc_staging_ring_acquire(ring, 1_000_000)
+    kvc.kvc_pack(lay, ids[:16], dptr, cb)
+    kvc.kvc_staging_ring_commit(ring, slot)
+    kvc.kvc_staging_ring_sync_filled(ring, slot)
+    import ctypes
+    got = np.ctypeslib.as_array((ctypes.c_uint8 * cb).from_address(hptr))
+    assert np.array_equal(got, want[:cb])
+    kvc.kvc_staging_ring_release(ring, slot)
+    with pytest.raises(kvc.KvcError):
+        kvc.kvc_layout_set_tuning(lay, slot_memory=3)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+    kvc.kvc_staging_ring_destroy(ring)

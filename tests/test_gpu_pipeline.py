@@ -206,3 +206,49 @@ def test_four_requests_sharing_a_prefix_are_served_from_one_pool(tmp_path):
     with pytest.raises(kvc.KvcError) as e:
         kvc.kvc_pipeline_load_many(lay, fifo, store, reqs)
     assert e.value.status == kvc.KVC_ERR_STATE
+
+
+def test_retained_chunks_serve_a_later_call_without_a_read(tmp_path):
+    """Retention (the paper's optional DRAM cache inside the pool, Sec. 6.4): chunks of a finished
+    load stay in their slots, so a second request with the same hashes is served without touching
+    the files, until foreground work needs the slots."""
+    g = orc.Dims(4, 2, 256, 16, 8, 128, 2)
+    pool = wl.random_bits(703, g.pool_bytes)
+    pool_t = torch.from_numpy(pool).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    store = kvc.kvc_store_open(str(tmp_path), "m", direct_io=True)
+    perm = wl.block_ids(75, g.NB, g.NB)
+    src, dst1, dst2, dst3 = (np.ascontiguousarray(perm[i * 48:(i + 1) * 48]) for i in range(4))
+    hashes = _hashes(3, 3)
+    fifo = kvc.kvc_staging_ring_create(cb, 2, kvc.KVC_RING_HOST_MAPPED)
+    kvc.kvc_pipeline_store(lay, fifo, store, src, hashes)
+    kvc.kvc_staging_ring_destroy(fifo)
+    chunks = orc.pack_request(g, pool, src, 256)
+    ring = kvc.kvc_staging_ring_create(cb, 4, kvc.KVC_RING_HOST_MAPPED)
+    kvc.kvc_staging_ring_set_policy(ring, foreground_reserve=1, max_speculative=1, retain_completed=True)
+    want_pool = pool.copy()
+    s1, _ = kvc.kvc_pipeline_load_many(lay, ring, store, [dict(ids=dst1, hashes=hashes, cls=kvc.KVC_CLASS_DEMAND_LOAD)])
+    torch.cuda.synchronize()
+    orc.unpack_request(g, want_pool, chunks, dst1, 256)
+    assert s1["reads"] == 3 and s1["joins"] == 0
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert (c["n_retained"], c["n_free"]) == (3, 1)
+    reads0 = kvc.kvc_store_get_counters(store)["reads"]
+    s2, _ = kvc.kvc_pipeline_load_many(lay, ring, store, [dict(ids=dst2, hashes=hashes, cls=kvc.KVC_CLASS_DEMAND_LOAD)])
+    torch.cuda.synchronize()
+    orc.unpack_request(g, want_pool, chunks, dst2, 256)
+    assert s2["reads"] == 0 and s2["joins"] == 3 and s2["unpack_launches"] == 1
+    assert kvc.kvc_store_get_counters(store)["reads"] == reads0
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    # other work needs the slots: cached chunks give way, least recently used first
+    other = _hashes(4, 3)
+    kvc.kvc_pipeline_store(lay, ring, store, dst1, other)            # three stores through the same pool
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert c["reclaims"] >= 2
+    s3, _ = kvc.kvc_pipeline_load_many(lay, ring, store, [dict(ids=dst3, hashes=hashes, cls=kvc.KVC_CLASS_DEMAND_LOAD)])
+    torch.cuda.synchronize()
+    orc.unpack_request(g, want_pool, chunks, dst3, 256)
+    assert s3["reads"] >= 2                                          # evicted chunks are read again
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
