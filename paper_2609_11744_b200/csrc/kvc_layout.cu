@@ -720,8 +720,36 @@ kvc_status kvc_map_requests_shared(const kvc_layout *lay, const int32_t *const *
         // same staged block exactly when they reach the same node.  Longer requests go first, so
         // a chunk that is a truncation of another request's chunk arrives after it and finds its
         // last node already covered.
-        std::map<std::pair<uint32_t, int32_t>, uint32_t> child;
+        // child(parent node, block id) -> node, in an open-addressing table (total table length is
+        // known up front, so it never grows)
+        uint64_t total_len = 0;
+        for (uint32_t r = 0; r < n_requests; ++r)
+            total_len += lens[r];
+        uint64_t tcap = 16;
+        while (tcap < 2 * total_len + 2)
+            tcap *= 2;
+        const uint64_t kEmpty = ~0ull;
+        std::vector<uint64_t> keys(tcap, kEmpty);
+        std::vector<uint32_t> vals(tcap, 0);
+        auto child_of = [&](uint32_t node, int32_t id, uint32_t next_id, bool *created) {
+            const uint64_t key = ((uint64_t)node << 32) | (uint32_t)id;
+            uint64_t h = key * 0x9E3779B97F4A7C15ull;
+            h ^= h >> 29;
+            for (uint64_t i = h & (tcap - 1);; i = (i + 1) & (tcap - 1)) {
+                if (keys[i] == key) {
+                    *created = false;
+                    return vals[i];
+                }
+                if (keys[i] == kEmpty) {
+                    keys[i] = key;
+                    vals[i] = next_id;
+                    *created = true;
+                    return next_id;
+                }
+            }
+        };
         std::vector<char> covered(1, 0);  // node 0 = root
+        covered.reserve(total_len + 1);
         std::vector<uint32_t> order(n_requests);
         for (uint32_t r = 0; r < n_requests; ++r)
             order[r] = r;
@@ -729,7 +757,8 @@ kvc_status kvc_map_requests_shared(const kvc_layout *lay, const int32_t *const *
                          [&](uint32_t x, uint32_t y) { return lens[x] > lens[y]; });
         std::vector<kvc_chunk_desc> kept;
         std::vector<uint32_t> kept_end;            // trie node where each kept chunk ends
-        std::map<uint32_t, uint32_t> owner;        // chunk end node -> lowest request ending a chunk there
+        const uint32_t kNobody = ~0u;
+        std::vector<uint32_t> owner(total_len + 1, kNobody);  // chunk end node -> lowest request ending a chunk there
         std::vector<uint32_t> path;
         uint64_t uniq = 0;
         for (uint32_t r : order) {
@@ -737,14 +766,10 @@ kvc_status kvc_map_requests_shared(const kvc_layout *lay, const int32_t *const *
             path.resize(n);
             uint32_t node = 0;
             for (uint32_t i = 0; i < n; ++i) {
-                auto key = std::make_pair(node, tables[r][i]);
-                auto it = child.find(key);
-                if (it == child.end()) {
-                    uint32_t id = (uint32_t)covered.size();
+                bool created = false;
+                node = child_of(node, tables[r][i], (uint32_t)covered.size(), &created);
+                if (created)
                     covered.push_back(0);
-                    it = child.emplace(key, id).first;
-                }
-                node = it->second;
                 path[i] = node;
             }
             uint32_t c = 0;
@@ -753,11 +778,8 @@ kvc_status kvc_map_requests_shared(const kvc_layout *lay, const int32_t *const *
                 if (nb < lay->bpc && (flags & KVC_MAP_FULL_CHUNKS_ONLY))
                     break;
                 const uint32_t end = path[first + nb - 1];
-                auto ow = owner.find(end);
-                if (ow == owner.end())
+                if (owner[end] == kNobody || r < owner[end])
                     owner[end] = r;
-                else if (r < ow->second)
-                    ow->second = r;
                 if (covered[end])
                     continue;
                 for (uint32_t i = 0; i < nb; ++i) {

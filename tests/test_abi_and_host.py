@@ -449,6 +449,87 @@ def test_rings_created_on_several_threads_while_the_provider_is_replaced(fake_ev
     assert errors == []
 
 
+@pytest.mark.parametrize("seed", [1, 2, 3, 4])
+def test_pool_mode_random_walk_keeps_its_invariants(fake_events, seed):
+    """Random acquire / commit / release / cancel / abandon / event-completion sequences against a
+    small model of who holds what.  Whatever the policy decides, these must hold: a slot handed
+    out for a new operation has no holder left and no unfinished release event; a join lands on
+    the slot that holds the key; counters add up; releases beyond the references are refused."""
+    D, S, P = kvc.KVC_CLASS_DEMAND_LOAD, kvc.KVC_CLASS_STORE, kvc.KVC_CLASS_PRELOAD
+    rng = np.random.default_rng(seed)
+    n = 5
+    ring, base = _pool_ring(n, 4096, reserve=int(rng.integers(0, 3)), max_spec=int(rng.integers(0, 3)),
+                            retain=bool(rng.integers(0, 2)))
+    drained_ev = {i: 2 * i + 2 for i in range(n)}     # events are created slot by slot: filled, drained
+    held = {i: 0 for i in range(n)}                   # references this test holds per slot
+    key_of, filled, filler = {}, {}, {}
+    for step in range(600):
+        op = rng.integers(0, 7)
+        if op <= 1:
+            cls, key = [D, S, P][rng.integers(0, 3)], int(rng.integers(0, 7))
+            got = kvc.kvc_staging_ring_acquire_for(ring, cls, key)
+            if got is None:
+                continue
+            slot, dp, hp, joined = got
+            assert dp == base + slot * 4096
+            if joined:
+                assert key_of.get(slot) == key
+            else:
+                assert held[slot] == 0, "slot %d handed out while references remain" % slot
+                assert fake_events.done[drained_ev[slot]], "slot %d reused before its event" % slot
+                key_of[slot], filled[slot], filler[slot] = key, False, True
+            held[slot] += 1
+        elif op == 2:
+            cands = [i for i in range(n) if held[i] and not filled.get(i, True) and filler.get(i)]
+            if cands:
+                i = int(rng.choice(cands))
+                (kvc.kvc_staging_ring_commit_host(ring, i) if rng.integers(0, 2)
+                 else kvc.kvc_staging_ring_commit(ring, i, 3))
+                filled[i] = True
+        elif op == 3:
+            cands = [i for i in range(n) if held[i] and filled.get(i)]
+            if cands:
+                i = int(rng.choice(cands))
+                (kvc.kvc_staging_ring_release(ring, i, int(rng.integers(4, 9))) if rng.integers(0, 2)
+                 else kvc.kvc_staging_ring_release_host(ring, i))
+                held[i] -= 1
+        elif op == 4:
+            for ev in list(fake_events.done):
+                if rng.integers(0, 2):
+                    fake_events.done[ev] = True
+        elif op == 5:
+            cands = [i for i in range(n) if held[i] == 1 and not filled.get(i, True) and filler.get(i)]
+            if cands:
+                i = int(rng.choice(cands))
+                try:
+                    kvc.kvc_staging_ring_abandon(ring, i)
+                    held[i] -= 1
+                    filler[i] = False
+                except kvc.KvcError as e:
+                    assert e.status == kvc.KVC_ERR_STATE
+        else:
+            i = int(rng.integers(0, n))
+            if held[i] == 0 and filled.get(i):
+                with pytest.raises(kvc.KvcError) as e:      # nothing left to release
+                    kvc.kvc_staging_ring_release_host(ring, i)
+                assert e.value.status == kvc.KVC_ERR_STATE
+        c = kvc.kvc_staging_ring_policy_counters(ring)
+        assert c["n_free"] + c["n_in_flight"] + c["n_staged"] + c["n_retained"] == n
+    # wind down: fill what is being filled, let go of everything, finish every event
+    for i in range(n):
+        if held[i] and not filled.get(i, True):
+            kvc.kvc_staging_ring_commit_host(ring, i)
+            filled[i] = True
+        while held[i]:
+            kvc.kvc_staging_ring_release(ring, i, 9)
+            held[i] -= 1
+    fake_events.complete_all()
+    c = kvc.kvc_staging_ring_policy_counters(ring)
+    assert c["n_in_flight"] == 0
+    assert c["n_free"] + c["n_staged"] + c["n_retained"] == n
+    kvc.kvc_staging_ring_destroy(ring)
+
+
 def test_ring_create_validation(fake_events):
     for args, want in [((4096, 0, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
                        ((0, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
