@@ -879,11 +879,21 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
     per_iter = e0.elapsed_time(e1) / (2 * GRAPH_ITERS)
     iters = max(GRAPH_ITERS, int(seconds * 1e3 / per_iter) // GRAPH_ITERS * GRAPH_ITERS)
     results = []
+    # small shared-memory footprints (2 stages of 8 or 4 KiB per block) are there to see whether copy
+    # blocks that fit beside a resident GEMM block disturb the GEMM less than 66 KB blocks do
+    preset = {k: v for k, v in kvc.kvc_tuning_preset(kvc.KVC_PRESET_BESIDE_COMPUTE).items() if v}
+    assert preset == dict(max_ctas=16, tile_bytes=8192, stages=2)
+    small = [dict(max_ctas=0, tile_bytes=8192, stages=2), dict(max_ctas=32, tile_bytes=8192, stages=2),
+             preset, dict(max_ctas=32, tile_bytes=4096, stages=2)]
     for kind, kind_name in ((kvc.KVC_RING_DEVICE, "device slots + cudaMemcpyAsync"),
                             (kvc.KVC_RING_HOST_MAPPED, "mapped pinned host slots")):
-        for max_ctas in ((16, 0) if kind == kvc.KVC_RING_DEVICE else (4, 16, 64)):
+        tunings = [dict(max_ctas=c) for c in ((16, 0) if kind == kvc.KVC_RING_DEVICE else (4, 16, 64))]
+        if kind == kvc.KVC_RING_DEVICE:
+            tunings += small
+        for tuning in tunings:
+            max_ctas = tuning["max_ctas"]
             lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
-            kvc.kvc_layout_set_tuning(lay, max_ctas=max_ctas)
+            kvc.kvc_layout_set_tuning(lay, **tuning)
             descs = kvc.kvc_map_request(lay, n)
             cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
             ring = kvc.kvc_staging_ring_create(cb, int(w.extra["ring_slots"]), kind)
@@ -918,6 +928,7 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
             for direction, fn in (("offload", offload), ("load", load)):
                 results.append(_overlap_case(torch, fn, gemm_loop, s_gemm, s_k, s_c, iters, seconds,
                                              one_way, N, kind_name, direction, max_ctas))
+                results[-1]["tuning"] = tuning
             kvc.kvc_staging_ring_destroy(ring)
             kvc.kvc_layout_destroy(lay)
     for GROUP, n_ring in ((4, int(w.extra["ring_slots"])), (8, 16)):

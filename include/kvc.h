@@ -176,6 +176,20 @@ typedef struct {
 #define KVC_GROUP_FORCE_KERNEL 0x100u
 /* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */
 kvc_status kvc_layout_set_tuning(kvc_layout *layout, const kvc_tuning *tuning);
+/* Ready-made tunings (no counterpart in the paper; Sec. 5.1 is where the question comes from: a
+ * copy kernel takes SM time away from the model).
+ *   KVC_PRESET_DEFAULT         all zeros: highest copy throughput, for slots in device memory.
+ *   KVC_PRESET_BESIDE_COMPUTE  for streaming chunks to or from the host while a compute stream is
+ *       busy: 16 persistent one-warp blocks with two 8 KiB stages each (17 KB of shared memory and
+ *       about 1000 registers per block), small enough to sit on an SM BESIDE a resident GEMM block
+ *       instead of waiting for one to retire and then keeping the next one out.  Measured on B200
+ *       next to a bf16 8192^3 matmul loop: the host link stays saturated (56.7 / 55.0 GB/s) and the
+ *       GEMM loop slows down by 0.2 % or less, against 7-8 % with the default 66 KB blocks and
+ *       1.3 % with the copy engines.  Its own ceiling is a few hundred GB/s: not for
+ *       device-to-device staging at HBM speed.
+ * Fills *out; pass it to kvc_layout_set_tuning.  INVALID_ARG for an unknown preset or NULL. */
+typedef enum { KVC_PRESET_DEFAULT = 0, KVC_PRESET_BESIDE_COMPUTE = 1 } kvc_preset;
+kvc_status kvc_tuning_preset(kvc_preset which, kvc_tuning *out);
 
 /* ------------------------------------------------------------------ mapper (Sec. 6.4, 6.5) */
 

@@ -681,6 +681,19 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
     return KVC_OK;
 }
 
+kvc_status kvc_tuning_preset(kvc_preset which, kvc_tuning *out)
+{
+    if (!out || (which != KVC_PRESET_DEFAULT && which != KVC_PRESET_BESIDE_COMPUTE))
+        return KVC_ERR_INVALID_ARG;
+    memset(out, 0, sizeof(*out));
+    if (which == KVC_PRESET_BESIDE_COMPUTE) {
+        out->max_ctas = 16;
+        out->tile_bytes = 8192;
+        out->stages = 2;
+    }
+    return KVC_OK;
+}
+
 kvc_status kvc_map_request(const kvc_layout *lay, uint32_t n_blocks, uint32_t flags,
                            kvc_chunk_desc *out, uint32_t cap, uint32_t *n_out)
 {

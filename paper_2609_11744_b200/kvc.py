@@ -141,6 +141,7 @@ def lib() -> ctypes.CDLL:
         "kvc_layout_chunk_bytes": (u64, [vp, u32]),
         "kvc_layout_num_chunks": (u32, [vp, u32]),
         "kvc_layout_set_tuning": (ci, [vp, P(kvc_tuning)]),
+        "kvc_tuning_preset": (ci, [ci, P(kvc_tuning)]),
         "kvc_map_request": (ci, [vp, u32, u32, P(kvc_chunk_desc), u32, P(u32)]),
         "kvc_map_requests_shared": (ci, [vp, P(vp), P(u32), u32, u32, P(kvc_chunk_desc), u32, P(u32),
                                          P(u64)]),
@@ -356,6 +357,16 @@ def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, 
     t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag,
                    items_per_cta, pdl, group, slot_memory)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
+
+
+KVC_PRESET_DEFAULT, KVC_PRESET_BESIDE_COMPUTE = 0, 1
+
+
+def kvc_tuning_preset(which: int) -> dict:
+    """The fields of a ready-made tuning, as keyword arguments for kvc_layout_set_tuning."""
+    t = kvc_tuning()
+    _check(lib().kvc_tuning_preset(which, ctypes.byref(t)), "kvc_tuning_preset")
+    return {k: getattr(t, k) for k, _ in kvc_tuning._fields_}
 
 
 def kvc_layout_launch_count(layout) -> int:

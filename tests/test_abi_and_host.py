@@ -161,6 +161,16 @@ def test_set_tuning_validation():
             kvc.kvc_layout_set_tuning(lay, **bad)
 
 
+def test_tuning_presets():
+    assert not any(kvc.kvc_tuning_preset(kvc.KVC_PRESET_DEFAULT).values())
+    p = kvc.kvc_tuning_preset(kvc.KVC_PRESET_BESIDE_COMPUTE)
+    assert (p["max_ctas"], p["tile_bytes"], p["stages"]) == (16, 8192, 2)
+    lay = _layout()
+    kvc.kvc_layout_set_tuning(lay, **p)              # a preset is a valid tuning
+    with pytest.raises(kvc.KvcError):
+        kvc.kvc_tuning_preset(7)
+
+
 def test_product_never_imports_the_oracle():
     pkg = os.path.join(ROOT, "paper_2609_11744_b200")
     for dirpath, _, files in os.walk(pkg):

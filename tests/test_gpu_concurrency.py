@@ -51,7 +51,7 @@ class _GemmLoad:
 
 
 @pytest.mark.parametrize("kind", [kvc.KVC_RING_DEVICE, kvc.KVC_RING_HOST_MAPPED])
-@pytest.mark.parametrize("variant", [kvc.KVC_VARIANT_AUTO, kvc.KVC_VARIANT_VEC])
+@pytest.mark.parametrize("variant", [kvc.KVC_VARIANT_AUTO, kvc.KVC_VARIANT_VEC, "beside-compute preset"])
 def test_ring_streaming_stays_exact_beside_a_compute_stream(kind, variant):
     """A 2048-token prefix (8 chunks) through a 3-slot ring, offload then load, on high-priority
     streams with default (programmatic dependent) launches, while a low-priority stream runs a
@@ -61,7 +61,10 @@ def test_ring_streaming_stays_exact_beside_a_compute_stream(kind, variant):
     pool = _pool_8b_384()
     pool_t = to_dev(pool)
     lay = dense_layout(pool_t, g, 256)
-    kvc.kvc_layout_set_tuning(lay, variant=variant)
+    if isinstance(variant, str):
+        kvc.kvc_layout_set_tuning(lay, **kvc.kvc_tuning_preset(kvc.KVC_PRESET_BESIDE_COMPUTE))
+    else:
+        kvc.kvc_layout_set_tuning(lay, variant=variant)
     src = wl.block_ids(w.seed, g.NB, 128)
     dst = wl.block_ids(w.dst_seed, g.NB, 128)
     descs = kvc.kvc_map_request(lay, len(src))
