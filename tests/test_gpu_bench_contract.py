@@ -30,6 +30,11 @@ def test_bench_line_has_the_contract_keys():
     assert roof["bound"] == "hbm" and roof["unit"] == "GB/s" and roof["peak"] > 1000
     assert abs(roof["frac"] - roof["achieved"] / roof["peak"]) < 1e-9
     assert roof["algorithmic_bytes_per_launch"] == 2 * d["config"]["bytes_each_way"]
+    for side in ("pack", "unpack"):                     # jitter is visible in the record itself
+        t = roof[side]
+        assert t["min_ms"] <= t["median_ms"] <= t["max_ms"] and t["min_ms"] <= t["ms"] <= t["max_ms"]
+        assert len(roof["per_step_ms"][side]) == 3
+    assert "traffic_source" in roof and roof["traffic"] is None   # not the workload the capture was of
     e2e = d["e2e"]
     assert e2e["h2d_bytes_per_step"] == e2e["d2h_bytes_per_step"] == d["config"]["bytes_each_way"]
     assert 0 < e2e["value"] < d["value"]                # the host link is slower than HBM
