@@ -172,6 +172,11 @@ typedef struct {
                             caller that issues many small per-chunk calls into slots it allocated
                             itself can save the query; a wrong answer picks a kernel tuned for the
                             other kind of memory */
+    uint32_t vec_threads; /* VEC: threads per block, a multiple of 32 up to 256 (0 = 256).  Fewer than
+                            256 makes every warp copy its own tile of at most 4 KiB; one-warp blocks
+                            (32) hold about 2000 registers and can share an SM with a resident
+                            compute block.  With fewer threads per block, max_ctas still counts
+                            blocks: give 8 times as many one-warp blocks for the same bytes in flight */
 } kvc_tuning;
 #define KVC_GROUP_FORCE_KERNEL 0x100u
 /* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */

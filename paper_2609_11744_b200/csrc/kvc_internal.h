@@ -86,6 +86,7 @@ struct KvcLaunch {
     uint32_t group_shift;     // multi-slab kernel: log2 of the slabs per work item
     uint32_t pending;         // bulk kernels: stores that may still read shared memory at a stage reuse
     uint64_t n_slabs;         // multi-slab kernels: n_ent * LP
+    uint32_t vec_threads;     // vector kernels with one warp per item: threads per block (0 = 256)
     uint64_t vec_magic;       // multi-slab vector kernel: 2^32 / (vectors per slab) + 1, for v / vps
     int32_t ids[KVC_PARAM_IDS];
 };

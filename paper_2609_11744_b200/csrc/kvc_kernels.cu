@@ -178,7 +178,7 @@ __global__ void __launch_bounds__(KVC_VEC_THREADS)
 kvc_vec_kernel(const __grid_constant__ KvcLaunch a)
 {
     constexpr uint32_t SH = VB == 32 ? 5 : 4;
-    constexpr uint32_t TEAMS = KVC_VEC_THREADS / TEAM;
+    const uint32_t TEAMS = blockDim.x / TEAM;  // blocks of fewer than 256 threads: warp teams only
     const uint32_t t = threadIdx.x % TEAM;
     const uint32_t n_items = (uint32_t)a.n_items;
     const uint64_t stride = (uint64_t)gridDim.x * TEAMS;
@@ -235,7 +235,7 @@ kvc_vec_group_kernel(const __grid_constant__ KvcLaunch a)
 {
     constexpr uint32_t SH = VB == 32 ? 5 : 4;
     constexpr uint32_t U = VB == 32 ? 4 : 8;     // 128 bytes in flight per lane
-    constexpr uint32_t WARPS = KVC_VEC_THREADS / 32;
+    const uint32_t WARPS = blockDim.x / 32u;
     constexpr uint32_t FULL = 0xffffffffu;
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t ksh = a.group_shift, R = 1u << ksh;
@@ -719,18 +719,20 @@ cudaError_t launch_one(int variant, const KvcLaunch &a, uint32_t grid, uint32_t 
             return e;
         return launch_cfg(kvc_bulk_group_kernel<DIR, TABLE>, a, grid, KVC_BULK_THREADS, smem, stream);
     }
+    // kernels that give every warp its own work item run with any whole number of warps per block
+    const uint32_t wt = a.vec_threads ? a.vec_threads : KVC_VEC_THREADS;
     if (variant == KVC_VARIANT_VEC32_GROUP)
-        return launch_cfg(kvc_vec_group_kernel<DIR, TABLE, 32>, a, grid, KVC_VEC_THREADS, 0, stream);
+        return launch_cfg(kvc_vec_group_kernel<DIR, TABLE, 32>, a, grid, wt, 0, stream);
     if (variant == KVC_VARIANT_VEC_GROUP)
-        return launch_cfg(kvc_vec_group_kernel<DIR, TABLE, 16>, a, grid, KVC_VEC_THREADS, 0, stream);
+        return launch_cfg(kvc_vec_group_kernel<DIR, TABLE, 16>, a, grid, wt, 0, stream);
     const bool warp_team = a.g.tile_bytes <= KVC_VEC_WARP_TEAM_MAX_TILE;
     if (variant == KVC_VARIANT_VEC32)
         return warp_team
-                   ? launch_cfg(kvc_vec_kernel<DIR, TABLE, 32, 32>, a, grid, KVC_VEC_THREADS, 0, stream)
+                   ? launch_cfg(kvc_vec_kernel<DIR, TABLE, 32, 32>, a, grid, wt, 0, stream)
                    : launch_cfg(kvc_vec_kernel<DIR, TABLE, 32, KVC_VEC_THREADS>, a, grid, KVC_VEC_THREADS,
                                 0, stream);
     return warp_team
-               ? launch_cfg(kvc_vec_kernel<DIR, TABLE, 16, 32>, a, grid, KVC_VEC_THREADS, 0, stream)
+               ? launch_cfg(kvc_vec_kernel<DIR, TABLE, 16, 32>, a, grid, wt, 0, stream)
                : launch_cfg(kvc_vec_kernel<DIR, TABLE, 16, KVC_VEC_THREADS>, a, grid, KVC_VEC_THREADS, 0,
                             stream);
 }

@@ -100,6 +100,9 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     uint32_t tile = t.tile_bytes;
     if (tile == 0)
         tile = (variant == KVC_VARIANT_BULK || !persistent) ? 32768u : 16384u;
+    const bool small_vec_blocks = variant != KVC_VARIANT_BULK && t.vec_threads && t.vec_threads < KVC_VEC_THREADS;
+    if (small_vec_blocks)  // blocks of fewer than 256 threads exist for the one-warp-per-tile kernels only
+        tile = std::min<uint32_t>(tile, KVC_VEC_WARP_TEAM_MAX_TILE);
     tile = (uint32_t)std::min<uint64_t>(tile, lay->slab_bytes);
     uint32_t stages = 0, lag = 0, smem = 0, group_shift = 0;
     if (variant == KVC_VARIANT_BULK) {
@@ -183,6 +186,7 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     if (n_items == 0 || n_items > 0xFFFFFFFFull || n_slabs > 0xFFFFFFFFull)
         return KVC_ERR_INVALID_ARG;
     a->n_slabs = n_slabs;
+    a->vec_threads = small_vec_blocks ? t.vec_threads : 0;
     a->group_shift = group_shift;
     // stores that may still be reading shared memory when a stage is reloaded: the stage's last
     // store is stages-lag groups back, so everything newer than that may stay outstanding
@@ -209,7 +213,8 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
         if (vec_grouped) {
             // one item per warp at a time: a block of 8 warps takes 8 * items_per_cta items
             // (default 16 per warp, about 1 MiB per block: measured 3-5 % faster than 4)
-            per_block = 8u * (per_block ? per_block : 16u);
+            const uint32_t warps = (a->vec_threads ? a->vec_threads : KVC_VEC_THREADS) / 32u;
+            per_block = warps * (per_block ? per_block : 16u);
         } else if (per_block == 0) {
             const bool bulk = variant == KVC_VARIANT_BULK || variant == KVC_VARIANT_BULK_GROUP;
             const uint32_t bytes = bulk ? 65536u : 32768u;
@@ -676,6 +681,8 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
     if (t->ctas_per_sm > 4 || t->l2_hint > 2 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2 || t->items_per_cta > (1u << 20))
         return KVC_ERR_INVALID_ARG;
     if ((t->group & ~KVC_GROUP_FORCE_KERNEL) > KVC_GROUP_MAX_SLABS || t->slot_memory > 2)
+        return KVC_ERR_INVALID_ARG;
+    if (t->vec_threads % 32 || t->vec_threads > KVC_VEC_THREADS)
         return KVC_ERR_INVALID_ARG;
     lay->tuning = *t;
     return KVC_OK;

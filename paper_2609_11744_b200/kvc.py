@@ -56,7 +56,8 @@ class kvc_tuning(ctypes.Structure):
                 ("stages", ctypes.c_uint32), ("ctas_per_sm", ctypes.c_uint32),
                 ("l2_hint", ctypes.c_uint32), ("lag", ctypes.c_uint32),
                 ("items_per_cta", ctypes.c_uint32), ("pdl", ctypes.c_uint32),
-                ("group", ctypes.c_uint32), ("slot_memory", ctypes.c_uint32)]
+                ("group", ctypes.c_uint32), ("slot_memory", ctypes.c_uint32),
+                ("vec_threads", ctypes.c_uint32)]
 
 
 class kvc_chunk_desc(ctypes.Structure):
@@ -353,9 +354,9 @@ def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
 
 def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
                           ctas_per_sm=0, l2_hint=0, lag=0, items_per_cta=0, pdl=0, group=0,
-                          slot_memory=0) -> None:
+                          slot_memory=0, vec_threads=0) -> None:
     t = kvc_tuning(variant, order, max_ctas, tile_bytes, stages, ctas_per_sm, l2_hint, lag,
-                   items_per_cta, pdl, group, slot_memory)
+                   items_per_cta, pdl, group, slot_memory, vec_threads)
     _check(lib().kvc_layout_set_tuning(layout.handle, ctypes.byref(t)), "kvc_layout_set_tuning")
 
 
@@ -590,7 +591,7 @@ def kvc_staging_ring_num_slots(ring) -> int:
     return lib().kvc_staging_ring_num_slots(ring.handle)
 
 
-_provider_keep = None
+_provider_keep = []   # rings copy the provider when they are created: its callbacks must outlive them
 
 
 def kvc_staging_ring_set_event_provider(provider: Optional[dict]) -> None:
@@ -600,7 +601,7 @@ def kvc_staging_ring_set_event_provider(provider: Optional[dict]) -> None:
     global _provider_keep
     if provider is None:
         _check(lib().kvc_staging_ring_set_event_provider(None), "kvc_staging_ring_set_event_provider")
-        _provider_keep = None
+        _provider_keep = []   # rings copy the provider when they are created: its callbacks must outlive them
         return
     p = kvc_event_provider()
     fns = {}
@@ -609,7 +610,7 @@ def kvc_staging_ring_set_event_provider(provider: Optional[dict]) -> None:
         setattr(p, name, fns[name])
     _check(lib().kvc_staging_ring_set_event_provider(ctypes.byref(p)),
            "kvc_staging_ring_set_event_provider")
-    _provider_keep = (p, fns)
+    _provider_keep.append((p, fns))
 
 
 # ------------------------------------------------------------------ chunk files

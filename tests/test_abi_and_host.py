@@ -427,9 +427,13 @@ def test_rings_created_on_several_threads_while_the_provider_is_replaced(fake_ev
     stop = threading.Event()
 
     def churn():
+        import time
         p = fake_events.provider()
-        while not stop.is_set():
+        for _ in range(400):                      # (every installation keeps its callbacks alive)
+            if stop.is_set():
+                break
             kvc.kvc_staging_ring_set_event_provider(p)
+            time.sleep(0.0005)
 
     def worker(seed):
         try:

@@ -754,6 +754,17 @@ def test_plain_c_program_links_and_runs(tmp_path):
     assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr
 
 
+@pytest.mark.parametrize("vec_threads", [32, 64, 224])
+def test_vector_kernel_with_small_blocks_on_8b_shape(vec_threads):
+    """Blocks of fewer than 256 threads: every warp copies its own 4 KiB tile of the 32 KiB slabs."""
+    g = dims_of(wl.LLAMA_8B, 384)
+    pool = _pool_8b_384()
+    src, dst = wl.block_ids(8, g.NB, 40), wl.block_ids(9, g.NB, 40)
+    for mode, tuning in (("batch", dict()), ("chunk", dict(max_ctas=24))):
+        run_pack_unpack(g, pool, src, dst, 256, kvc.KVC_VARIANT_VEC, 0, mode, vec_threads=vec_threads,
+                        **tuning)
+
+
 def test_kernel_timing_and_slot_memory_hint():
     """Diagnostics and hints do not change a byte: with kernel timing on, every launch is reported
     with a positive duration; with the slot_memory hint the pointer query is skipped and the right

@@ -60,7 +60,8 @@ def test_slabs_per_item_and_traversal_orders(group, order, variant):
 
 
 @pytest.mark.parametrize("tuning", [dict(max_ctas=2), dict(items_per_cta=1), dict(items_per_cta=9),
-                                    dict(pdl=1), dict(group=2, max_ctas=5)],
+                                    dict(pdl=1), dict(group=2, max_ctas=5), dict(vec_threads=32),
+                                    dict(vec_threads=96, max_ctas=7), dict(vec_threads=32, max_ctas=40)],
                          ids=lambda t: ",".join("%s=%s" % kv for kv in t.items()))
 def test_vector_kernel_launch_shapes_with_grouped_items(tuning):
     for name, n, cb in (("S64", 71, 16), ("S2K", 61, 16), ("S4K", 35, 4), ("S48", 50, 8)):
