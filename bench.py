@@ -890,9 +890,8 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
         tunings = [dict(max_ctas=c) for c in ((16, 0) if kind == kvc.KVC_RING_DEVICE else (4, 16, 64))]
         if kind == kvc.KVC_RING_DEVICE:
             tunings += small
-        else:   # one-warp vector blocks: about 2000 registers each, may fit beside a GEMM block
-            tunings += [dict(max_ctas=128, vec_threads=32), dict(max_ctas=256, vec_threads=32),
-                        dict(max_ctas=64, vec_threads=64)]
+        else:   # one-warp vector blocks (about 2000 registers each): measured WORSE for the GEMM
+            tunings += [dict(max_ctas=128, vec_threads=32)]
         for tuning in tunings:
             max_ctas = tuning["max_ctas"]
             lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
