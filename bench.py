@@ -583,6 +583,9 @@ def suite_launch_shapes(torch, kvc, dev, reps):
         ("default: bulk, streaming (2 items/block, 2 stages), chunk-major", dict()),
         ("multi-slab bulk kernel forced, one 32 KiB slab per item (A/B of the two bulk kernels)",
          dict(group=kvc.KVC_GROUP_FORCE_KERNEL)),
+        ("bulk streaming, L2 evict-first hint on loads and stores", dict(l2_hint=2)),
+        ("bulk streaming, L2 evict-first hint on loads only", dict(l2_hint=3)),
+        ("bulk streaming, L2 evict-first hint on stores only", dict(l2_hint=4)),
         ("bulk streaming, 1 item per block", dict(items_per_cta=1)),
         ("bulk streaming, 4 items per block", dict(items_per_cta=4)),
         ("bulk streaming, 8 items per block, 3 stages", dict(items_per_cta=8, stages=3)),
@@ -652,6 +655,47 @@ def suite_small_slabs(torch, kvc, dev, reps, sizes=None, request_mib=2048):
             kvc.kvc_layout_destroy(lay)
         del pool, staging
         torch.cuda.empty_cache()
+    return out
+
+
+def suite_row_gather(torch, dev, reps):
+    """Ceiling probe, independent of the library: random gather / scatter of S-byte rows by a plain
+    kernel (tests/native/row_gather_probe.cu, built here with nvcc).  2 GiB of rows out of an 8 GiB
+    array, best of a few launch shapes.  Context for the small_slabs part."""
+    import ctypes
+    import subprocess
+    import tempfile
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    out = []
+    with tempfile.TemporaryDirectory() as d:
+        so = os.path.join(d, "librow_gather_probe.so")
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-shared",
+                               "-Xcompiler", "-fPIC", "-cudart", "static", "-o", so,
+                               os.path.join(ROOT, "tests", "native", "row_gather_probe.cu")])
+        L = ctypes.CDLL(so)
+        L.probe_rows.argtypes = [ctypes.c_void_p] * 3 + [ctypes.c_int] * 5 + [ctypes.c_void_p]
+        L.probe_rows.restype = ctypes.c_int
+        st = torch.cuda.current_stream().cuda_stream
+        for S in (32768, 8192, 4096, 2048, 1024, 512, 256):
+            total = 8 << 30
+            N = total // S
+            n = N // 4
+            src = wl.random_bits_cuda(wl.BASE_SEED + S, total, dev)
+            dst = torch.empty(n * S, dtype=torch.uint8, device=dev)
+            idx = torch.from_numpy(wl.block_ids(wl.BASE_SEED + 3, N, n)).to(dev)
+            best = {"gather_gbs": 0.0, "scatter_gbs": 0.0}
+            for R in sorted({1, max(1, 4096 // S), max(1, 16384 // S)}):
+                for grid in (148 * 8, 148 * 16):
+                    def run(scatter, a, b):
+                        rc = L.probe_rows(a.data_ptr(), b.data_ptr(), idx.data_ptr(), n, S, R, scatter, grid, st)
+                        assert rc == 0
+                    _, g = _time_ms(torch, lambda: run(0, src, dst), max(5, reps // 2))
+                    _, sc = _time_ms(torch, lambda: run(1, dst, src), max(5, reps // 2))
+                    best["gather_gbs"] = max(best["gather_gbs"], 2 * n * S / g / 1e6)
+                    best["scatter_gbs"] = max(best["scatter_gbs"], 2 * n * S / sc / 1e6)
+            out.append(dict(row_bytes=S, rows=n, **best))
+            del src, dst, idx
+            torch.cuda.empty_cache()
     return out
 
 
@@ -1229,6 +1273,7 @@ def run_suite(args):
                          torch, kvc, dev, args.steps,
                          [int(x) for x in args.small_slab_sizes.split(",")] if args.small_slab_sizes else None,
                          args.small_slab_mib)),
+                     ("row_gather", lambda: suite_row_gather(torch, dev, args.steps)),
                      ("call_overhead", lambda: suite_call_overhead(args.steps)),
                      ("prefix_8k", lambda: suite_8k(torch, kvc, dev, args.steps)),
                      ("batch_70b", lambda: suite_batch(torch, kvc, dev, args.steps)),
@@ -1268,7 +1313,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
-                         "host_link,launch_shapes,chunk_sweep,small_slabs,call_overhead,prefix_8k,batch_70b,"
+                         "host_link,launch_shapes,chunk_sweep,small_slabs,row_gather,call_overhead,prefix_8k,batch_70b,"
                          "ring_overlap,duplex,file_pipeline,preload_trace (1 GPU; prints one JSON line)")
     ap.add_argument("--small-slab-sizes", default="",
                     help="small_slabs suite part: comma list of slab sizes in bytes (default: all)")

@@ -150,7 +150,8 @@ typedef struct {
     uint32_t stages;     /* BULK: shared-memory stages per thread block (0 = default) */
     uint32_t ctas_per_sm; /* BULK: thread blocks the shared memory of one SM is divided among,
                             1..4 (0 = default); bounds stages * tile_bytes per block */
-    uint32_t l2_hint;    /* BULK: 0 = default, 1 = no L2 priority hint, 2 = evict-first on loads and stores */
+    uint32_t l2_hint;    /* BULK (single-slab kernel): 0 = default (= 1), 1 = no L2 priority hint,
+                            2 = evict-first on loads and stores, 3 = on loads only, 4 = on stores only */
     uint32_t lag;        /* BULK: loads issued ahead of the store they feed, 1..stages-2 (0 = default) */
     uint32_t items_per_cta; /* default launch shape: work items per block (0 = about 64 KiB for
                             BULK, 32 KiB for VEC) */

@@ -81,7 +81,7 @@ struct KvcLaunch {
     uint32_t block_major_chunks;  // chunk layout is [n][L][P].. (else [L][P][n]..)
     uint32_t stages;          // bulk kernels
     uint32_t lag;             // bulk kernels: loads issued ahead of the store they feed
-    uint32_t l2_evict_first;  // bulk kernels: attach an evict-first L2 policy to the copies
+    uint32_t l2_evict_first;  // single-slab bulk kernel: evict-first L2 policy on loads (bit 0), stores (bit 1)
     uint32_t pdl;             // launch with programmatic stream serialisation
     uint32_t group_shift;     // multi-slab kernel: log2 of the slabs per work item
     uint32_t pending;         // bulk kernels: stores that may still read shared memory at a stage reuse

@@ -439,7 +439,7 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
     grid_dependency_wait();
     __syncwarp();
 
-    const bool hint = a.l2_evict_first != 0;
+    const bool hint_ld = (a.l2_evict_first & 1u) != 0, hint_st = (a.l2_evict_first & 2u) != 0;
     const uint64_t pol = policy_evict_first();
     bool ok = true;          // lane 0: no wait has expired
     uint32_t loads_done = 0; // lane 0: items whose load was issued (for the drain on failure)
@@ -473,7 +473,7 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
                     mbar_expect_tx(bar, len);
                     if (len) {
                         const uint64_t from = DIR == KVC_DIR_PACK ? pool : slot;
-                        if (hint)
+                        if (hint_ld)
                             bulk_load_hint(smem_u32(data + (size_t)s * tile), from, len, bar, pol);
                         else
                             bulk_load(smem_u32(data + (size_t)s * tile), from, len, bar);
@@ -487,7 +487,7 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
                         const uint32_t l2 = st_len[s];
                         if (l2) {
                             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                            if (hint)
+                            if (hint_st)
                                 bulk_store_hint(st_dst[s], smem_u32(data + (size_t)s * tile), l2, pol);
                             else
                                 bulk_store(st_dst[s], smem_u32(data + (size_t)s * tile), l2);
