@@ -52,8 +52,14 @@ def _full_size_case(w, chunk_tokens, n_free_check=64):
     staging = torch.full((one_way + 4096,), 0x77, dtype=torch.uint8, device=DEV)
     lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, chunk_tokens)
     assert kvc.kvc_layout_num_chunks(lay, n) == len(orc.chunk_ranges(n, bpc))
-    pool16, stage16 = pool.view(torch.int16), staging[:one_way].view(torch.int16)
+    # element-typed views: the oracle's positions are in elements of s.e bytes
+    elem_t = {1: torch.uint8, 2: torch.int16, 4: torch.int32}[s.e]
+    pool16, stage16 = pool.view(elem_t), staging[:one_way].view(elem_t)
+    assert pool16.numel() == g.pool_bytes // g.e
     blk, stage_pos, src_pos, dst_pos = _sampled_positions(g, src, dst, bpc, w.seed)
+    # positions are checked here, on the host, before any of them indexes a device tensor
+    assert 0 <= stage_pos.min() and stage_pos.max() < stage16.numel()
+    assert 0 <= min(src_pos.min(), dst_pos.min()) and max(src_pos.max(), dst_pos.max()) < pool16.numel()
     dev_idx = lambda a: torch.from_numpy(a).to(DEV)
 
     # ---- pack: one launch
@@ -184,3 +190,58 @@ def test_config5_32k_prefix_streamed_through_8_slot_ring_to_host():
     got = host.view(torch.int16)[torch.from_numpy(stage_pos)]
     assert torch.equal(got, want)
     kvc.kvc_staging_ring_destroy(ring)
+
+
+@pytest.mark.parametrize("elem_bytes", [2, 1])
+def test_tensor_parallel_shard_of_the_80k_prefix(elem_bytes):
+    """The 80k-token prefix as ONE GPU of an 8-way tensor-parallel 8B model sees it: one KV head per
+    GPU, so 4 KiB slabs (2 KiB with 1-byte elements) -- the shapes the multi-slab kernels exist for.
+    Sampled elements at the oracle's positions over the 20,000-block pool, whole chunks, untouched
+    blocks; launch configuration as in the benchmark (one batched call per direction)."""
+    shape = wl.KVShape(L=32, P=2, B=16, H=1, D=128, e=elem_bytes)
+    w = wl.Workload("8b_80k_tp8", 5 + elem_bytes, shape, 20000, 80000, (256,))
+    _full_size_case(w, 256)
+
+
+def test_tensor_parallel_shard_whole_prefix_against_the_oracle_loops():
+    """The same shard shape with every byte compared: 5000 blocks (1.22 GiB) out of a 6000-block
+    pool, the oracle's plain loops run over (layer, K|V) ranges on the host cores."""
+    from concurrent.futures import ThreadPoolExecutor
+    shape = wl.KVShape(L=32, P=2, B=16, H=1, D=128, e=2)
+    NB, n, bpc = 6000, 5000, 16
+    g = orc.Dims(shape.L, shape.P, NB, shape.B, shape.H, shape.D, shape.e)
+    pool = wl.random_bits(wl.BASE_SEED + 77, g.pool_bytes)
+    src, dst = wl.block_ids(wl.BASE_SEED + 78, NB, n), wl.block_ids(wl.BASE_SEED + 79, NB, n)
+    pool_t = torch.from_numpy(pool).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, NB, g.B, g.H, g.D, g.e, 256)
+    one_way = n * g.bytes_per_block
+    staging = torch.full((one_way + 4096,), 0x77, dtype=torch.uint8, device=DEV)
+    ops, keep, nbytes, on_dev = kvc.request_chunk_ops(lay, src, staging)
+    kvc.kvc_pack_batch(lay, ops, on_dev)
+    ops2, keep2, _, _ = kvc.request_chunk_ops(lay, dst, staging)
+    kvc.kvc_unpack_batch(lay, ops2, on_dev)
+    torch.cuda.synchronize()
+    ranges = orc.chunk_ranges(n, bpc)
+    want = np.zeros(one_way, dtype=np.uint8)
+    want_pool = pool.copy()
+    lp = g.L * g.P
+    cuts = [(a, min(lp, a + 8)) for a in range(0, lp, 8)]
+
+    def pack_part(r):
+        for first, nb in ranges:
+            lo = first * g.bytes_per_block
+            orc.pack_chunk_into(g, pool, src[first:first + nb], want[lo:lo + nb * g.bytes_per_block], r)
+
+    def unpack_part(r):
+        for first, nb in ranges:
+            lo = first * g.bytes_per_block
+            orc.unpack_chunk(g, want_pool, want[lo:lo + nb * g.bytes_per_block], dst[first:first + nb], r)
+
+    with ThreadPoolExecutor(len(cuts)) as ex:
+        list(ex.map(pack_part, cuts))
+        list(ex.map(unpack_part, cuts))
+    host = staging.cpu().numpy()
+    assert np.array_equal(host[:one_way], want), "pack"
+    assert (host[one_way:] == 0x77).all()
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool), "unpack"
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)

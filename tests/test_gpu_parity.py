@@ -530,6 +530,54 @@ def test_random_tiny_layouts():
         done += 1
 
 
+@pytest.mark.parametrize("seed", [7, 8, 9])
+def test_random_layouts_with_random_launch_shapes(seed):
+    """As above, and the launch shape is drawn at random too: slabs per work item, stages, loads
+    ahead, blocks (persistent or streaming), items per block, threads per vector block, L2 hints,
+    dependent launch on or off.  No knob may change a byte."""
+    rng = np.random.default_rng(seed)
+    done = 0
+    while done < 30:
+        e = int(rng.choice([1, 2, 4]))
+        L, P = int(rng.integers(1, 6)), int(rng.integers(1, 3))
+        B, H = int(rng.integers(1, 17)), int(rng.integers(1, 9))
+        D = int(rng.choice([8, 16, 32, 64, 128]))
+        S = B * H * D * e
+        if S % 16 or S > 65536:
+            continue
+        NB = int(rng.integers(2, 80))
+        if L * P * NB * S > (96 << 20):
+            continue
+        g = orc.Dims(L, P, NB, B, H, D, e)
+        n = int(rng.integers(1, NB + 1))
+        bpc = int(rng.integers(1, n + 2))
+        pool = wl.random_bits(int(rng.integers(1 << 30)), g.pool_bytes + (g.pool_bytes & 1))[:g.pool_bytes]
+        src = rng.permutation(NB)[:n].astype(np.int32)
+        dst = rng.permutation(NB)[:n].astype(np.int32)
+        variant = int(rng.choice(VARIANTS))
+        stages = int(rng.choice([0, 2, 3, 4, 8, 16]))
+        tuning = dict(
+            group=int(rng.choice([0, 1, 2, 4, 8, 16, 32, kvc.KVC_GROUP_FORCE_KERNEL])),
+            stages=stages,
+            lag=int(rng.integers(0, max(1, stages - 1))) if stages > 2 else 0,
+            max_ctas=int(rng.choice([0, 0, 1, 3, 17, 148])),
+            items_per_cta=int(rng.choice([0, 1, 2, 5, 40])),
+            vec_threads=int(rng.choice([0, 32, 64, 128, 256])),
+            l2_hint=int(rng.integers(0, 5)),
+            pdl=int(rng.integers(0, 3)),
+        )
+        tile = int(rng.choice([0, 0, 1024, 4096, 8192, 16384]))
+        order = int(rng.choice([0, 1, 2, 3]))
+        mode = str(rng.choice(["chunk", "chunk_dev", "batch", "batch_dev"]))
+        try:
+            run_pack_unpack(g, pool, src, dst, bpc * B, variant, order, mode, tile, **tuning)
+        except AssertionError as err:
+            raise AssertionError("%s with geometry %r, %d blocks in chunks of %d, variant %d, order %d, "
+                                 "mode %s, tile %d, tuning %r" % (err, g, n, bpc, variant, order, mode,
+                                                                  tile, tuning))
+        done += 1
+
+
 # ------------------------------------------------------------------ layout variants
 @pytest.mark.parametrize("variant", VARIANTS)
 @pytest.mark.parametrize("mode", ["chunk", "batch_dev", "copy_engine", "static"])
