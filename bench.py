@@ -1130,24 +1130,37 @@ def suite_file_pipeline(torch, kvc, dev, root):
     for base in root.split(","):
         if not os.path.isdir(base):
             continue
-        for use_ce in (False, True):
+        # (copies by the DMA engines or by kernels, I/O threads, FIFO ring or pool mode)
+        for use_ce, threads, pool_mode in ((False, 4, False), (True, 4, False), (False, 8, True),
+                                           (False, 16, True)):
             d = tempfile.mkdtemp(prefix="kvc_suite_", dir=base)
             try:
                 lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
                 kvc.kvc_layout_set_tuning(lay, max_ctas=16)
                 cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
-                ring = kvc.kvc_staging_ring_create(cb, 8, kvc.KVC_RING_HOST_MAPPED)
+                ring = kvc.kvc_staging_ring_create(cb, 8 if not pool_mode else 2 * threads,
+                                                   kvc.KVC_RING_HOST_MAPPED)
+                if pool_mode:
+                    kvc.kvc_staging_ring_set_policy(ring, 0)
                 store = kvc.kvc_store_open(d, "8b", direct_io=True)
                 hashes = [kvc.kvc_fnv1a64(b"chunk%d" % c) for c in range(kvc.kvc_layout_num_chunks(lay, n))]
-                st = kvc.kvc_pipeline_store(lay, ring, store, src, hashes, io_threads=4,
+                st = kvc.kvc_pipeline_store(lay, ring, store, src, hashes, io_threads=threads,
                                             use_copy_engine=use_ce)
                 torch.cuda.synchronize()
                 t0 = time.perf_counter()
-                ld = kvc.kvc_pipeline_load(lay, ring, store, dst, hashes, io_threads=4,
-                                           use_copy_engine=use_ce)
+                if pool_mode:
+                    ld, _ = kvc.kvc_pipeline_load_many(
+                        lay, ring, store, [dict(ids=dst, hashes=hashes, cls=kvc.KVC_CLASS_DEMAND_LOAD)],
+                        io_threads=threads)
+                    ld["bytes"] = ld["bytes_read"]
+                else:
+                    ld = kvc.kvc_pipeline_load(lay, ring, store, dst, hashes, io_threads=threads,
+                                               use_copy_engine=use_ce)
                 torch.cuda.synchronize()
                 load_s = time.perf_counter() - t0
                 out.append({"root": base, "copies": "copy engines" if use_ce else "kernels (16 CTAs)",
+                            "io_threads": threads,
+                            "staging": ("pool mode, %d slots" % (2 * threads)) if pool_mode else "FIFO ring, 8 slots",
                             "bytes": st["bytes"], "store_s": st["seconds"],
                             "store_gbs": st["bytes"] / st["seconds"] / 1e9,
                             "load_s": load_s, "load_gbs": ld["bytes"] / load_s / 1e9,
