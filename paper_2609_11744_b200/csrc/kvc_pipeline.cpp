@@ -610,8 +610,14 @@ kvc_status kvc_pipeline_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store,
                               uint32_t io_threads, int use_copy_engine, void *stream,
                               kvc_pipeline_stats *stats)
 {
-    return run_store(lay, ring, store, ids, n_blocks, hashes, n_hashes, io_threads, use_copy_engine, stream,
-                     stats);
+    // (the bookkeeping containers are sized up front; should an allocation still fail inside, the
+    // exception must not cross the C boundary)
+    try {
+        return run_store(lay, ring, store, ids, n_blocks, hashes, n_hashes, io_threads, use_copy_engine,
+                         stream, stats);
+    } catch (...) {
+        return KVC_ERR_NOMEM;
+    }
 }
 
 kvc_status kvc_pipeline_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const int32_t *ids,
@@ -628,7 +634,12 @@ kvc_status kvc_pipeline_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, 
     q.n_hashes = n_hashes;
     q.cls = KVC_CLASS_DEMAND_LOAD;
     kvc_load_many_stats ms = {};
-    const kvc_status rc = run_load(lay, ring, store, &q, 1, io_threads, use_copy_engine, stream, &ms);
+    kvc_status rc;
+    try {
+        rc = run_load(lay, ring, store, &q, 1, io_threads, use_copy_engine, stream, &ms);
+    } catch (...) {
+        rc = KVC_ERR_NOMEM;
+    }
     if (stats) {
         kvc_pipeline_stats st = {};
         st.bytes = ms.bytes_read;
@@ -646,7 +657,11 @@ kvc_status kvc_pipeline_load_many(kvc_layout *lay, kvc_ring *ring, kvc_store *st
 {
     if (ring && !kvc_staging_ring_pool_mode(ring))
         return KVC_ERR_STATE;
-    return run_load(lay, ring, store, reqs, n_reqs, io_threads, 0, stream, stats);
+    try {
+        return run_load(lay, ring, store, reqs, n_reqs, io_threads, 0, stream, stats);
+    } catch (...) {
+        return KVC_ERR_NOMEM;
+    }
 }
 
 }  // extern "C"
