@@ -42,3 +42,25 @@ def test_host_only_library_parts_are_clean_under_asan_and_ubsan(tmp_path):
     scratch.mkdir()
     run = subprocess.run([exe, str(scratch)], capture_output=True, text=True, timeout=120)
     assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr
+
+
+@pytest.mark.skipif(shutil.which("g++") is None, reason="needs g++")
+def test_staging_ring_is_clean_under_asan_and_ubsan(tmp_path):
+    """The ring's bookkeeping, FIFO and pool mode, compiled as plain C++ (the CUDA runtime calls it
+    names are stubbed in the driver and never reached) and driven by a long random walk."""
+    cuda_inc = os.path.join(os.environ.get("CUDA_HOME", "/usr/local/cuda"), "include")
+    if not os.path.isdir(cuda_inc):
+        pytest.skip("needs the CUDA toolkit headers")
+    csrc = os.path.join(ROOT, "paper_2609_11744_b200", "csrc")
+    exe = str(tmp_path / "ring_san")
+    build = subprocess.run(
+        ["g++", "-O1", "-g", "-std=c++17", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
+         "-I", os.path.join(ROOT, "include"), "-I", csrc, "-I", cuda_inc,
+         "-x", "c++", os.path.join(csrc, "kvc_ring.cu"), os.path.join(csrc, "kvc_slot_pool.cpp"),
+         os.path.join(ROOT, "tests", "native", "ring_sanitizer_driver.cpp"), "-o", exe, "-lpthread"],
+        capture_output=True, text=True)
+    if build.returncode != 0 and "sanitize" in build.stderr:
+        pytest.skip("sanitizer runtime not installed")
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=120)
+    assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr
