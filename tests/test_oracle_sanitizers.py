@@ -64,3 +64,26 @@ def test_staging_ring_is_clean_under_asan_and_ubsan(tmp_path):
     assert build.returncode == 0, build.stderr
     run = subprocess.run([exe], capture_output=True, text=True, timeout=120)
     assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr
+
+
+@pytest.mark.skipif(shutil.which("g++") is None, reason="needs g++")
+def test_layout_mapper_and_launch_front_ends_are_clean_under_asan_and_ubsan(tmp_path):
+    """kvc_layout.cu compiled as plain C++ with host stand-ins for the CUDA runtime and a launch
+    recorder instead of the kernels: validation, the chunk mapper, the shared-prefix trie and the
+    per-block tables over 200 random geometries, tunings and request sets."""
+    cuda_inc = os.path.join(os.environ.get("CUDA_HOME", "/usr/local/cuda"), "include")
+    if not os.path.isdir(cuda_inc):
+        pytest.skip("needs the CUDA toolkit headers")
+    csrc = os.path.join(ROOT, "paper_2609_11744_b200", "csrc")
+    exe = str(tmp_path / "layout_san")
+    build = subprocess.run(
+        ["g++", "-O1", "-g", "-std=c++17", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
+         "-I", os.path.join(ROOT, "include"), "-I", csrc, "-I", cuda_inc,
+         "-x", "c++", os.path.join(csrc, "kvc_layout.cu"),
+         os.path.join(ROOT, "tests", "native", "layout_sanitizer_driver.cpp"), "-o", exe, "-lpthread"],
+        capture_output=True, text=True)
+    if build.returncode != 0 and "sanitize" in build.stderr:
+        pytest.skip("sanitizer runtime not installed")
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=300)
+    assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr[-3000:]
