@@ -550,7 +550,11 @@ def suite_chunk_sweep(torch, kvc, dev, reps):
         modes.append(("per_chunk", lambda: per_chunk(0, src), lambda: per_chunk(1, dst)))
         modes.append(("per_chunk_4_streams", lambda: per_chunk_streams(0, src),
                       lambda: per_chunk_streams(1, dst)))
+        # the same one-stream loop with the launches declared independent of one another (pdl = 3)
+        modes.append(("per_chunk_independent", lambda: per_chunk(0, src), lambda: per_chunk(1, dst)))
         for name, fp, fu in modes:
+            kvc.kvc_layout_set_tuning(lay, pdl=3 if name == "per_chunk_independent" else 0,
+                                      slot_memory=1)
             # 5000 single-chunk launches of 2 MiB are launch-bound by design: fewer repetitions
             r = reps if len(descs) <= 400 or name == "batch" else max(3, reps // 4)
             pm, pd = _time_ms(torch, fp, r)

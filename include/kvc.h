@@ -157,7 +157,16 @@ typedef struct {
                             BULK, 32 KiB for VEC) */
     uint32_t pdl;        /* 0 = default (= 2), 1 = plain launches, 2 = programmatic dependent launch:
                             a kernel's blocks may be scheduled while the previous kernel of the
-                            stream drains; they wait for its completion before reading memory */
+                            stream drains; they wait for its completion before reading memory.
+                            3 = the same WITHOUT that wait, for a sequence of calls on one stream
+                            whose kernels are independent of one another (packing the chunks of a
+                            request into different slots; unpacking chunks into different blocks):
+                            a kernel then runs beside the last blocks of the previous one instead
+                            of after them.  The caller vouches for the independence: a pack right
+                            after an unpack of the same blocks would read stale bytes.  Work of other
+                            kinds queued earlier on the stream (copies, waits for events) is
+                            complete either way, and an event recorded after a call still covers
+                            that call and everything before it */
     uint32_t group;      /* BULK: slabs per work item.  0 = default: when a slab is at most half a
                             tile, as many whole slabs as fit one tile (a power of two, at most 16;
                             the default tile is 16 KiB for slabs under 4 KiB)

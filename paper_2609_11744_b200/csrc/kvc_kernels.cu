@@ -116,9 +116,14 @@ __device__ __forceinline__ Item decode(const KvcLaunch &a, uint32_t w, bool coun
 // global memory may be read before grid_dependency_wait() returns (it waits for the previous
 // grid to complete and its writes to be visible); after it, the next kernel is let in early.
 // Without the attribute both instructions do nothing.
-__device__ __forceinline__ void grid_dependency_wait()
+// With overlap != 0 the wait is skipped: the caller has declared that this launch does not touch
+// what the previous kernel of the stream reads or writes, so its blocks may run beside that
+// kernel's last blocks (work that preceded the previous kernel has completed either way, because
+// that kernel could not start before it).
+__device__ __forceinline__ void grid_dependency_wait(uint32_t overlap = 0)
 {
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!overlap)
+        asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
@@ -183,7 +188,7 @@ kvc_vec_kernel(const __grid_constant__ KvcLaunch a)
     const uint32_t n_items = (uint32_t)a.n_items;
     const uint64_t stride = (uint64_t)gridDim.x * TEAMS;
     uint64_t w = (uint64_t)blockIdx.x * TEAMS + threadIdx.x / TEAM;
-    grid_dependency_wait();
+    grid_dependency_wait(a.pdl == 2u);
     if (w >= n_items)
         return;
     Item cur = decode<TABLE>(a, (uint32_t)w, t == 0);
@@ -245,7 +250,7 @@ kvc_vec_group_kernel(const __grid_constant__ KvcLaunch a)
     const uint64_t n_items = a.n_items, n_slabs = a.n_slabs;
     const uint64_t stride = (uint64_t)gridDim.x * WARPS;
     uint64_t w = (uint64_t)blockIdx.x * WARPS + (threadIdx.x >> 5);
-    grid_dependency_wait();
+    grid_dependency_wait(a.pdl == 2u);
     if (w >= n_items)
         return;
     auto decode_mine = [&](uint64_t item) {
@@ -425,7 +430,7 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
     const uint32_t stages = a.stages, lag = a.lag, tile = a.g.tile_bytes;
     const uint32_t n_items = (uint32_t)a.n_items;
     if (blockIdx.x >= n_items) {
-        grid_dependency_wait();
+        grid_dependency_wait(a.pdl == 2u);
         return;
     }
     const uint32_t K = (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x;  // my items
@@ -436,7 +441,7 @@ kvc_bulk_kernel(const __grid_constant__ KvcLaunch a)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    grid_dependency_wait();
+    grid_dependency_wait(a.pdl == 2u);
     __syncwarp();
 
     const bool hint_ld = (a.l2_evict_first & 1u) != 0, hint_st = (a.l2_evict_first & 2u) != 0;
@@ -548,7 +553,7 @@ kvc_bulk_group_kernel(const __grid_constant__ KvcLaunch a)
     const uint64_t n_slabs = a.n_slabs;
     unsigned char *data = smem + KVC_GROUP_SMEM_HEADER(stages);
     if (blockIdx.x >= n_items) {
-        grid_dependency_wait();
+        grid_dependency_wait(a.pdl == 2u);
         return;
     }
     const uint32_t K = (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x;  // my items
@@ -559,7 +564,7 @@ kvc_bulk_group_kernel(const __grid_constant__ KvcLaunch a)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    grid_dependency_wait();
+    grid_dependency_wait(a.pdl == 2u);
     __syncwarp();
 
     const uint32_t per_round = 32u >> ksh;          // items decoded per round

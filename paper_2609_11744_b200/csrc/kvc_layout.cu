@@ -199,7 +199,10 @@ kvc_status kvc_make_plan(kvc_layout *lay, uint64_t n_ent, const void *slot_probe
     a->lag = lag;
     // bit 0: loads, bit 1: stores
     a->l2_evict_first = t.l2_hint == 2 ? 3u : t.l2_hint == 3 ? 1u : t.l2_hint == 4 ? 2u : 0u;
-    a->pdl = t.pdl != 1;  // on unless switched off
+    // 0 = plain launch, 1 = programmatic dependent launch, 2 = the same without waiting for the
+    // previous kernel (only where the launch reads nothing a kernel could have written: the
+    // batched calls read a table that an asynchronous copy delivers, which is ordered by an event)
+    a->pdl = t.pdl == 1 ? 0u : (t.pdl == 3 ? 2u : 1u);
     a->status = lay->d_status;
     uint64_t grid;
     if (t.max_ctas) {
@@ -679,7 +682,7 @@ kvc_status kvc_layout_set_tuning(kvc_layout *lay, const kvc_tuning *t)
         return KVC_ERR_INVALID_ARG;
     if (t->stages == 1 || t->stages > KVC_BULK_MAX_STAGES)
         return KVC_ERR_INVALID_ARG;
-    if (t->ctas_per_sm > 4 || t->l2_hint > 4 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 2 || t->items_per_cta > (1u << 20))
+    if (t->ctas_per_sm > 4 || t->l2_hint > 4 || t->lag > KVC_BULK_MAX_STAGES || t->pdl > 3 || t->items_per_cta > (1u << 20))
         return KVC_ERR_INVALID_ARG;
     if ((t->group & ~KVC_GROUP_FORCE_KERNEL) > KVC_GROUP_MAX_SLABS || t->slot_memory > 2)
         return KVC_ERR_INVALID_ARG;

@@ -118,12 +118,16 @@ int main(int argc, char **argv)
         CK(kvc_layout_create(&desc, &lay));
         const uint32_t bpc = kvc_layout_blocks_per_chunk(lay);
         const uint32_t n_chunks = kvc_layout_num_chunks(lay, n);
-        for (int hint = 0; hint < 2; ++hint) {
+        for (int v = 0; v < 3; ++v) {
+        /* v = 1: the caller vouches that slots are device memory; v = 2: and that consecutive
+         * launches are independent of one another (pdl = 3) */
+        const int hint = v >= 1, independent = v == 2;
         kvc_tuning tun;
         memset(&tun, 0, sizeof(tun));
-        tun.slot_memory = (uint32_t)hint; /* 1: the caller vouches that slots are device memory */
+        tun.slot_memory = (uint32_t)hint;
+        tun.pdl = independent ? 3u : 0u;
         CK(kvc_layout_set_tuning(lay, &tun));
-        if (hint && ci != 0)
+        if (v == 1 && ci != 0)
             continue;
         for (int dir = 0; dir < 2; ++dir) {
             for (int ns = 1; ns <= NSTREAMS; ns += NSTREAMS - 1) {
@@ -161,9 +165,9 @@ int main(int argc, char **argv)
                 }
                 const double hm = median(host_us, reps), dm = median(dev_ms, reps);
                 printf("{\"case\": \"per_chunk\", \"direction\": \"%s\", \"chunk_tokens\": %u, \"calls\": %u, "
-                       "\"streams\": %d, \"slot_memory_hint\": %d, \"host_us_per_call\": %.3f, "
+                       "\"streams\": %d, \"slot_memory_hint\": %d, \"independent_launches\": %d, \"host_us_per_call\": %.3f, "
                        "\"device_ms\": %.4f, \"device_us_per_call\": %.3f, \"gbs\": %.1f}\n",
-                       dir ? "unpack" : "pack", chunk_tokens[ci], n_chunks, ns, hint, hm, dm,
+                       dir ? "unpack" : "pack", chunk_tokens[ci], n_chunks, ns, hint, independent, hm, dm,
                        dm * 1e3 / n_chunks, 2.0 * per_block * n / dm / 1e6);
             }
         }

@@ -253,3 +253,45 @@ def test_offload_and_load_share_one_staging_pool_at_the_same_time(kind):
     assert (c["n_free"], c["acquires"]) == (4, len(da) + len(db))
     kvc.kvc_staging_ring_destroy(ring)
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+@pytest.mark.parametrize("variant", [kvc.KVC_VARIANT_BULK, kvc.KVC_VARIANT_VEC])
+def test_independent_launches_may_overlap_and_stay_exact(variant):
+    """pdl = 3: consecutive per-chunk calls on one stream whose kernels do not depend on each other
+    (the chunks of a request packed into different places; then unpacked into different blocks)
+    skip the wait for the previous kernel.  Many small chunks, so that kernels really run beside
+    their predecessors' last blocks; bytes against the oracle."""
+    g = orc.Dims(8, 2, 600, 16, 8, 128, 2)
+    pool = wl.random_bits(4242, g.pool_bytes)
+    pool_t = to_dev(pool)
+    lay = dense_layout(pool_t, g, 32)                     # chunks of 2 blocks: 1 MiB each
+    kvc.kvc_layout_set_tuning(lay, variant=variant, pdl=3, slot_memory=1)
+    src, dst = wl.block_ids(41, g.NB, 301), wl.block_ids(42, g.NB, 301)
+    descs = kvc.kvc_map_request(lay, len(src))
+    total = sum(d[4] for d in descs)
+    staging = torch.full((total + 4096,), 0x3E, dtype=torch.uint8, device=DEV)
+    want_chunks = orc.pack_request(g, pool, src, 32)
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, want_chunks, dst, 32)
+    torch.cuda.synchronize()
+    for rep in range(3):
+        staging.fill_(0x3E)
+        pool_t.copy_(torch.from_numpy(pool))
+        torch.cuda.synchronize()
+        off = 0
+        for (_, _, first, nb, nbytes) in descs:
+            kvc.kvc_pack(lay, src[first:first + nb], staging[off:off + nbytes])
+            off += nbytes
+        done = torch.cuda.Event()
+        done.record()                                      # an event after the calls covers all of them
+        done.synchronize()
+        host = staging.cpu().numpy()
+        assert np.array_equal(host[:total], np.concatenate(want_chunks)), "pack, pass %d" % rep
+        assert (host[total:] == 0x3E).all()
+        off = 0
+        for (_, _, first, nb, nbytes) in descs:
+            kvc.kvc_unpack(lay, staging[off:off + nbytes], dst[first:first + nb])
+            off += nbytes
+        torch.cuda.synchronize()
+        assert np.array_equal(pool_t.cpu().numpy(), want_pool), "unpack, pass %d" % rep
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
