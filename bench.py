@@ -47,7 +47,7 @@ TRAFFIC_8B_80K = {
     "bytes": 20_920_170_000.0,
     "source": "profiles/kvc_bulk_kernel_8b_80k_dram_traffic.md",
     "kernel_file": "paper_2609_11744_b200/csrc/kvc_kernels.cu",
-    "kernel_file_sha256_at_last_check": "b528a8cad9dd4a79956e3dfa7ad5a988ff000f81ad03ee6eac235525eea9939a",
+    "kernel_file_sha256_at_last_check": "372d51959538a4b208716ac5e245c751f5d2247fb86df750d1a596d13a7471f7",
 }
 
 
