@@ -356,6 +356,17 @@ def run_ours(args, rank, world, local_rank):
         if world > 1:
             dist.destroy_process_group()
         return
+    overlap = None
+    if world == 1 and not args.no_overlap:
+        # config 5 in brief, after the timed region: chunks streamed through the ring to and from
+        # the host while a bf16 matmul loop runs -- what the copies cost a compute stream
+        ov = suite_ring_overlap(torch, kvc, cuda_rt, dev, 1.5, brief=True)
+        overlap = {"gemm": ov["gemm"], "prefix_bytes": ov["prefix_bytes"],
+                   "runs": [{"copy_blocks": "KVC_PRESET_BESIDE_COMPUTE" if r["tuning"].get("tile_bytes")
+                             else "default", "direction": r["direction"],
+                             "link_gbs_alone": r["link_gbs_alone"], "link_gbs_with_gemm": r["link_gbs_with_gemm"],
+                             "gemm_slowdown": r["gemm_slowdown"], "overlap_efficiency": r["overlap_efficiency"]}
+                            for r in ov["runs"]]}
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         sample = OracleSample(s, args.chunk_tokens, w.seed + 50)
@@ -378,6 +389,8 @@ def run_ours(args, rank, world, local_rank):
     }
     if e2e:
         line["e2e"] = e2e
+    if overlap:
+        line["overlap_with_compute"] = overlap
     if cpu:
         line["cpu_baseline"] = cpu
     print(json.dumps(line), flush=True)
@@ -875,14 +888,18 @@ def _grouped_runs(torch, kvc, cuda_rt, pool, s, NB, n, src, dst, hptr, one_way, 
     return out
 
 
-def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
+def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds, brief=False):
     """Config 5: a 32k-token prefix (8B shape, 4 GiB) streamed through an 8-slot ring of 256-token
     slots to/from pinned host memory while a bf16 GEMM loop runs on another stream.  Destinations:
     device slots drained by cudaMemcpyAsync, or slots in mapped pinned host memory that the
     kernels write/read directly.  Reports link GB/s, GEMM slowdown and overlap efficiency
-    1 - (T_both - max(T_gemm, T_xfer)) / min(T_gemm, T_xfer)."""
+    1 - (T_both - max(T_gemm, T_xfer)) / min(T_gemm, T_xfer).
+    brief: device slots only, default blocks and the beside-compute preset (the part of this
+    measurement that the default benchmark line carries)."""
     w = wl.WORKLOADS["8b_ring"]
     s, NB, n = w.shape, w.pool_blocks, w.request_blocks
+    if brief:
+        n //= 2   # a 16k-token prefix (2 GiB) per pass keeps the brief run short
     pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
     src, dst = wl.block_ids(w.seed, NB, n), wl.block_ids(w.dst_seed, NB, n)
     one_way = n * s.bytes_per_block
@@ -935,8 +952,12 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
              preset, dict(max_ctas=32, tile_bytes=4096, stages=2)]
     for kind, kind_name in ((kvc.KVC_RING_DEVICE, "device slots + cudaMemcpyAsync"),
                             (kvc.KVC_RING_HOST_MAPPED, "mapped pinned host slots")):
+        if brief and kind != kvc.KVC_RING_DEVICE:
+            continue
         tunings = [dict(max_ctas=c) for c in ((16, 0) if kind == kvc.KVC_RING_DEVICE else (4, 16, 64))]
-        if kind == kvc.KVC_RING_DEVICE:
+        if brief:
+            tunings = [dict(max_ctas=0), preset]
+        elif kind == kvc.KVC_RING_DEVICE:
             tunings += small
         else:   # one-warp vector blocks (about 2000 registers each): measured WORSE for the GEMM
             tunings += [dict(max_ctas=128, vec_threads=32)]
@@ -981,6 +1002,10 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds):
                 results[-1]["tuning"] = tuning
             kvc.kvc_staging_ring_destroy(ring)
             kvc.kvc_layout_destroy(lay)
+    if brief:
+        return {"gemm": "bf16 %dx%dx%d torch.matmul loop" % (N, N, N), "ms_per_gemm": per_iter,
+                "ring_slots": int(w.extra["ring_slots"]), "slot_bytes": cb, "prefix_bytes": one_way,
+                "seconds_per_phase": seconds, "runs": results}
     for GROUP, n_ring in ((4, int(w.extra["ring_slots"])), (8, 16)):
         results.extend(_grouped_runs(torch, kvc, cuda_rt, pool, s, NB, n, src, dst, hptr, one_way, N,
                                      gemm_loop, s_gemm, s_k, s_c, iters, seconds, GROUP, n_ring, TO))
@@ -1328,6 +1353,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-overlap", action="store_true",
+                    help="skip the brief ring-streaming-beside-a-GEMM measurement after the timed region")
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
                          "host_link,launch_shapes,chunk_sweep,small_slabs,row_gather,call_overhead,prefix_8k,batch_70b,"

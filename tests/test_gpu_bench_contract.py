@@ -35,6 +35,11 @@ def test_bench_line_has_the_contract_keys():
         assert t["min_ms"] <= t["median_ms"] <= t["max_ms"] and t["min_ms"] <= t["ms"] <= t["max_ms"]
         assert len(roof["per_step_ms"][side]) == 3
     assert "traffic_source" in roof and roof["traffic"] is None   # not the workload the capture was of
+    ov = d["overlap_with_compute"]                      # config 5 in brief, after the timed region
+    assert {r["copy_blocks"] for r in ov["runs"]} == {"default", "KVC_PRESET_BESIDE_COMPUTE"}
+    assert {r["direction"] for r in ov["runs"]} == {"offload", "load"}
+    for r in ov["runs"]:
+        assert r["link_gbs_with_gemm"] > 5 and 0.8 < r["gemm_slowdown"] < 2.0
     e2e = d["e2e"]
     assert e2e["h2d_bytes_per_step"] == e2e["d2h_bytes_per_step"] == d["config"]["bytes_each_way"]
     assert 0 < e2e["value"] < d["value"]                # the host link is slower than HBM
