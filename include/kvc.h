@@ -199,8 +199,8 @@ kvc_status kvc_layout_set_tuning(kvc_layout *layout, const kvc_tuning *tuning);
  *       about 1000 registers per block), small enough to sit on an SM BESIDE a resident GEMM block
  *       instead of waiting for one to retire and then keeping the next one out.  Measured on B200
  *       next to a bf16 8192^3 matmul loop: the host link stays saturated (56.7 / 55.0 GB/s) and the
- *       GEMM loop slows down by 0-2 % (two runs), against 7-8 % with the default 66 KB blocks and
- *       about 1 % with the copy engines, which hold a lower link rate.  Its own ceiling is a few hundred GB/s: not for
+ *       GEMM loop slows down by about 2 % (0-2.6 % over four runs), against 7-8 % with the default
+ *       66 KB blocks and about 1 % with the copy engines, which hold a lower link rate.  Its own ceiling is a few hundred GB/s: not for
  *       device-to-device staging at HBM speed.
  * Fills *out; pass it to kvc_layout_set_tuning.  INVALID_ARG for an unknown preset or NULL. */
 typedef enum { KVC_PRESET_DEFAULT = 0, KVC_PRESET_BESIDE_COMPUTE = 1 } kvc_preset;
