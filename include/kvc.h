@@ -123,9 +123,9 @@ uint64_t kvc_layout_chunk_bytes(const kvc_layout *layout, uint32_t n_blocks); /*
 uint32_t kvc_layout_num_chunks(const kvc_layout *layout, uint32_t n_blocks);  /* ceil(n / bpc) */
 
 /* How the copy kernels run (no counterpart in the paper: launch-shape knobs of this
- * implementation, used by its benchmarks and tests).  Zero in every field means "library default" (AUTO: the bulk-copy
- * kernel for slots in device memory, the vector kernel with 16 persistent blocks for slots in
- * mapped host memory; chunk-major order). */
+ * implementation, used by its benchmarks and tests).  Zero in every field means "library default"
+ * (AUTO: the bulk-copy kernel for slots in device memory, the vector kernel with 16 persistent
+ * blocks for slots in mapped host memory; chunk-major order). */
 typedef enum {
     KVC_VARIANT_AUTO = 0,
     KVC_VARIANT_VEC = 1,  /* 16- or 32-byte vector loads/stores through registers */
@@ -173,7 +173,8 @@ typedef struct {
                             -- consecutive slabs of a chunk are contiguous in the slot, so one item
                             is several copies on the pool side and one on the slot side;
                             1 = one slab (or one tile of a slab) per item; N > 1 = at most N (<= 32).
-                            VEC: slabs of at most 4 KiB are moved several per warp the same way.
+                            VEC: slabs of at most 16 KiB go one warp per item, and as many whole
+                            slabs as fit 8 KiB per item.
                             Adding KVC_GROUP_FORCE_KERNEL runs the multi-slab kernel even when that
                             leaves one slab per item (for same-process comparisons) */
     uint32_t slot_memory; /* where the staging slots of this handle's calls live: 0 = ask the CUDA
@@ -183,10 +184,11 @@ typedef struct {
                             itself can save the query; a wrong answer picks a kernel tuned for the
                             other kind of memory */
     uint32_t vec_threads; /* VEC: threads per block, a multiple of 32 up to 256 (0 = 256).  Fewer than
-                            256 makes every warp copy its own tile of at most 4 KiB; one-warp blocks
-                            (32) hold about 2000 registers and can share an SM with a resident
-                            compute block.  With fewer threads per block, max_ctas still counts
-                            blocks: give 8 times as many one-warp blocks for the same bytes in flight */
+                            256 makes every warp copy its own tile of at most 4 KiB.  max_ctas still
+                            counts blocks.  An experiment knob: spreading the warps of the
+                            mapped-host path over many small blocks was measured to disturb a
+                            concurrent GEMM more, not less (the 16 full blocks of the default
+                            occupy the fewest SMs) */
 } kvc_tuning;
 #define KVC_GROUP_FORCE_KERNEL 0x100u
 /* Errors: INVALID_ARG (unknown enum, tile_bytes not a multiple of 16, stages*tile too large). */
@@ -200,8 +202,8 @@ kvc_status kvc_layout_set_tuning(kvc_layout *layout, const kvc_tuning *tuning);
  *       instead of waiting for one to retire and then keeping the next one out.  Measured on B200
  *       next to a bf16 8192^3 matmul loop: the host link stays saturated (56.7 / 55.0 GB/s) and the
  *       GEMM loop slows down by about 2 % (0-2.6 % over four runs), against 7-8 % with the default
- *       66 KB blocks and about 1 % with the copy engines, which hold a lower link rate.  Its own ceiling is a few hundred GB/s: not for
- *       device-to-device staging at HBM speed.
+ *       66 KB blocks and about 1 % with the copy engines, which hold a lower link rate.  Its own
+ *       ceiling is a few hundred GB/s: not for device-to-device staging at HBM speed.
  * Fills *out; pass it to kvc_layout_set_tuning.  INVALID_ARG for an unknown preset or NULL. */
 typedef enum { KVC_PRESET_DEFAULT = 0, KVC_PRESET_BESIDE_COMPUTE = 1 } kvc_preset;
 kvc_status kvc_tuning_preset(kvc_preset which, kvc_tuning *out);
