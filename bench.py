@@ -1160,15 +1160,19 @@ def suite_file_pipeline(torch, kvc, dev, root):
         if not os.path.isdir(base):
             continue
         # (copies by the DMA engines or by kernels, I/O threads, FIFO ring or pool mode)
-        for use_ce, threads, pool_mode in ((False, 4, False), (True, 4, False), (False, 8, True),
-                                           (False, 16, True)):
+        M, ST = kvc.KVC_RING_HOST_MAPPED, kvc.KVC_RING_DEVICE_STAGED
+        for use_ce, threads, pool_mode, kind in ((False, 4, False, M), (True, 4, False, M), (False, 8, True, M),
+                                                 (False, 16, True, M), (False, 4, False, ST),
+                                                 (False, 16, True, ST)):
             d = tempfile.mkdtemp(prefix="kvc_suite_", dir=base)
             try:
                 lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
-                kvc.kvc_layout_set_tuning(lay, max_ctas=16)
+                if kind == ST:
+                    kvc.kvc_layout_set_tuning(lay, **kvc.kvc_tuning_preset(kvc.KVC_PRESET_BESIDE_COMPUTE))
+                else:
+                    kvc.kvc_layout_set_tuning(lay, max_ctas=16)
                 cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
-                ring = kvc.kvc_staging_ring_create(cb, 8 if not pool_mode else 2 * threads,
-                                                   kvc.KVC_RING_HOST_MAPPED)
+                ring = kvc.kvc_staging_ring_create(cb, 8 if not pool_mode else 2 * threads, kind)
                 if pool_mode:
                     kvc.kvc_staging_ring_set_policy(ring, 0)
                 store = kvc.kvc_store_open(d, "8b", direct_io=True)
@@ -1187,9 +1191,13 @@ def suite_file_pipeline(torch, kvc, dev, root):
                                                use_copy_engine=use_ce)
                 torch.cuda.synchronize()
                 load_s = time.perf_counter() - t0
-                out.append({"root": base, "copies": "copy engines" if use_ce else "kernels (16 CTAs)",
+                copies = "copy engines, pool <-> host" if use_ce else "kernels (16 CTAs) across the link"
+                if kind == ST:
+                    copies = "kernels (beside-compute preset) to device halves + one async copy per chunk"
+                out.append({"root": base, "copies": copies,
                             "io_threads": threads,
-                            "staging": ("pool mode, %d slots" % (2 * threads)) if pool_mode else "FIFO ring, 8 slots",
+                            "staging": (("pool mode, %d slots" % (2 * threads)) if pool_mode else "FIFO ring, 8 slots")
+                            + (", device + pinned host halves" if kind == ST else ", mapped pinned"),
                             "bytes": st["bytes"], "store_s": st["seconds"],
                             "store_gbs": st["bytes"] / st["seconds"] / 1e9,
                             "load_s": load_s, "load_gbs": ld["bytes"] / load_s / 1e9,

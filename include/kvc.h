@@ -347,8 +347,17 @@ kvc_status kvc_layout_kernel_time(kvc_layout *layout, uint32_t *launches, double
 
 typedef struct kvc_ring kvc_ring;
 typedef enum {
-    KVC_RING_DEVICE = 0,     /* slots in device memory; the caller drains them with async copies */
-    KVC_RING_HOST_MAPPED = 1 /* slots in mapped pinned host memory; kernels write them directly */
+    KVC_RING_DEVICE = 0,      /* slots in device memory; the caller drains them with async copies */
+    KVC_RING_HOST_MAPPED = 1, /* slots in mapped pinned host memory; kernels write them directly */
+    KVC_RING_DEVICE_STAGED = 2 /* every slot is a pair: a device half that the kernels touch and a
+                                 pinned host half of the same size that file I/O touches; one
+                                 asynchronous copy moves a slot between the two (the store / load
+                                 pipelines do it; other callers get both addresses from acquire).
+                                 Kernels then run at HBM speed, with small blocks if a model is
+                                 running (KVC_PRESET_BESIDE_COMPUTE), and the copy engines cross the
+                                 link -- the combination that measured best beside a compute stream
+                                 and with both directions busy.  The host half is always allocated
+                                 by the library */
 } kvc_ring_kind;
 
 /* A ring of n_slots fixed slots of slot_bytes each (a multiple of 4096; use
@@ -367,8 +376,9 @@ kvc_status kvc_staging_ring_destroy(kvc_ring *ring);
  * by its last release has completed (polled on the host; no device-wide synchronisation).
  * timeout_us == 0: try once (WOULD_BLOCK); > 0: poll until the deadline (TIMEOUT);
  * < 0: INVALID_ARG (unbounded waits are not offered).
- * *dev_ptr is the address kernels and async copies use; *host_ptr the host address
- * (HOST_MAPPED rings) or NULL.  Either may be NULL. */
+ * *dev_ptr is the address kernels and async copies use; *host_ptr the host address of the same
+ * bytes (HOST_MAPPED rings), the slot's separate pinned host half (DEVICE_STAGED rings), or NULL.
+ * Either may be NULL. */
 kvc_status kvc_staging_ring_acquire(kvc_ring *ring, int64_t timeout_us, uint32_t *slot,
                                     void **dev_ptr, void **host_ptr);
 /* Records the slot's "filled" event on the producer stream.  STATE unless acquired. */
@@ -406,6 +416,7 @@ uint32_t kvc_staging_ring_trace_count(const kvc_ring *ring);
 uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *ring);
 uint32_t kvc_staging_ring_num_slots(const kvc_ring *ring);
 int kvc_staging_ring_pool_mode(const kvc_ring *ring); /* 1 after kvc_staging_ring_set_policy */
+kvc_ring_kind kvc_staging_ring_kind(const kvc_ring *ring);
 
 /* ------------------------------------------------------------------ chunk files (Sec. 6.3) */
 

@@ -12,8 +12,12 @@
 // again, demand loads go before preloads, and everything that became ready during one pass of
 // the loop, for whichever requests, is scattered by ONE fused unpack launch (Sec. 6.4).
 //
-// Built only from the public entry points of this library.  Every exit, error exits included,
-// hands every slot it took back to the staging memory.
+// Staging slots may be mapped pinned memory (the kernels cross the host link themselves) or
+// device-plus-host pairs (KVC_RING_DEVICE_STAGED: the kernels fill the device half and one
+// asynchronous copy per chunk, on a copy stream of the call's own, crosses the link).
+//
+// Built from the public entry points of this library, plus the CUDA runtime for those copies.
+// Every exit, error exits included, hands every slot it took back to the staging memory.
 #include <chrono>
 #include <condition_variable>
 #include <deque>
@@ -23,9 +27,51 @@
 #include <thread>
 #include <vector>
 
+#include <cuda_runtime.h>
+
 #include "kvc.h"
 
 namespace {
+
+// DEVICE_STAGED rings: the call's own copy stream and one "copy done" event per slot.
+struct StagedCopies {
+    bool on = false;
+    cudaStream_t stream = nullptr;
+    std::vector<cudaEvent_t> done;
+    kvc_status start(kvc_ring *ring)
+    {
+        on = kvc_staging_ring_kind(ring) == KVC_RING_DEVICE_STAGED;
+        if (!on)
+            return KVC_OK;
+        if (cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking) != cudaSuccess)
+            return KVC_ERR_CUDA;
+        done.assign(kvc_staging_ring_num_slots(ring), nullptr);
+        for (cudaEvent_t &e : done)
+            if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess)
+                return KVC_ERR_CUDA;
+        return KVC_OK;
+    }
+    // dst <- src on the copy stream, then the slot's "copy done" event
+    kvc_status copy(uint32_t slot, void *dst, const void *src, uint64_t bytes, cudaMemcpyKind kind)
+    {
+        if (cudaMemcpyAsync(dst, src, bytes, kind, stream) != cudaSuccess ||
+            cudaEventRecord(done[slot], stream) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return KVC_ERR_CUDA;
+        }
+        return KVC_OK;
+    }
+    ~StagedCopies()
+    {
+        if (stream)
+            cudaStreamSynchronize(stream);
+        for (cudaEvent_t e : done)
+            if (e)
+                cudaEventDestroy(e);
+        if (stream)
+            cudaStreamDestroy(stream);
+    }
+};
 
 struct Job {
     uint32_t tag;  // store: chunk index; load: slot index
@@ -35,6 +81,7 @@ struct Job {
     uint64_t bytes, hash;
     kvc_status status;
     bool existed;
+    cudaEvent_t copied;  // DEVICE_STAGED store: the event behind the slot's device-to-host copy
 };
 
 // Work queue for the I/O threads and completion queue back to the calling thread.
@@ -58,8 +105,12 @@ void io_worker(Queues *q, kvc_ring *ring, kvc_store *store, bool storing)
             q->work.pop_front();
         }
         if (storing) {
-            // the slot's copy was only enqueued: wait for its "filled" event, then write the file
-            j.status = kvc_staging_ring_sync_filled(ring, j.slot);
+            // the slot's copy was only enqueued: wait for its "filled" event (or, for a staged
+            // slot, for the copy into its host half), then write the file
+            if (j.copied)
+                j.status = cudaEventSynchronize(j.copied) == cudaSuccess ? KVC_OK : KVC_ERR_CUDA;
+            else
+                j.status = kvc_staging_ring_sync_filled(ring, j.slot);
             if (j.status == KVC_OK) {
                 j.status = kvc_store_publish(store, j.hash, j.host_ptr, j.bytes);
                 if (j.status == KVC_ERR_EXISTS) {
@@ -179,6 +230,10 @@ kvc_status run_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const in
         if (descs[c].bytes > slot_bytes)
             return KVC_ERR_INVALID_ARG;
     const bool pool = kvc_staging_ring_pool_mode(ring) != 0;
+    StagedCopies staged;  // destroyed after the workers below: their copies are waited for first
+    rc = staged.start(ring);
+    if (rc != KVC_OK)
+        return rc;
     Workers w;
     if (!start_workers(w, io_threads, ring, store, true))
         return KVC_ERR_NOMEM;
@@ -260,7 +315,20 @@ kvc_status run_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const in
             first_err = s;
             break;
         }
-        Job j = {c, slot, hptr, dptr, d.bytes, hashes[c], KVC_OK, false};
+        Job j = {c, slot, hptr, dptr, d.bytes, hashes[c], KVC_OK, false, nullptr};
+        if (staged.on && !use_copy_engine) {
+            // device half -> host half once the pack has run; the file is written from the host half
+            s = kvc_staging_ring_wait_filled(ring, slot, staged.stream);
+            if (s == KVC_OK)
+                s = staged.copy(slot, hptr, dptr, d.bytes, cudaMemcpyDeviceToHost);
+            if (s != KVC_OK) {
+                kvc_staging_ring_sync_filled(ring, slot);
+                kvc_staging_ring_release_host(ring, slot);
+                first_err = s;
+                break;
+            }
+            j.copied = staged.done[slot];
+        }
         submit(w, j);
         ++issued;
         ++st.chunks;
@@ -272,6 +340,8 @@ kvc_status run_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const in
         reap(false);
         for (const Job &j : dropped) {
             kvc_staging_ring_sync_filled(ring, j.slot);
+            if (j.copied)
+                cudaEventSynchronize(j.copied);
             kvc_staging_ring_release_host(ring, j.slot);
             ++finished;
         }
@@ -285,6 +355,8 @@ kvc_status run_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const in
         reap(false);
         for (const Job &j : dropped) {
             kvc_staging_ring_sync_filled(ring, j.slot);
+            if (j.copied)
+                cudaEventSynchronize(j.copied);
             kvc_staging_ring_release_host(ring, j.slot);
             ++finished;
         }
@@ -376,6 +448,12 @@ kvc_status run_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, kvc_load_
     } catch (const std::bad_alloc &) {
         return KVC_ERR_NOMEM;
     }
+    StagedCopies staged;
+    {
+        const kvc_status rc = staged.start(ring);
+        if (rc != KVC_OK)
+            return rc;
+    }
     Workers w;
     if (!start_workers(w, io_threads, ring, store, false))
         return KVC_ERR_NOMEM;
@@ -421,6 +499,19 @@ kvc_status run_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, kvc_load_
                 continue;
             }
             st.bytes_read += j.bytes;
+            if (staged.on && !use_copy_engine) {
+                // host half -> device half; the unpack stream waits for this copy only
+                kvc_status s = staged.copy(j.slot, sw.dev_ptr, sw.host_ptr, j.bytes, cudaMemcpyHostToDevice);
+                if (s == KVC_OK && cudaStreamWaitEvent((cudaStream_t)stream, staged.done[j.slot], 0) != cudaSuccess)
+                    s = KVC_ERR_CUDA;
+                if (s != KVC_OK) {
+                    note_error(s);
+                    for (size_t i = 0; i < sw.waiters.size(); ++i)
+                        kvc_staging_ring_release_host(ring, j.slot);
+                    sw.waiters.clear();
+                    continue;
+                }
+            }
             for (const Waiter &wt : sw.waiters)
                 ready.push_back({wt, j.slot});
             sw.waiters.clear();
@@ -554,7 +645,7 @@ kvc_status run_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, kvc_load_
                 sw.reading = true;
                 sw.waiters.clear();
                 sw.waiters.push_back(wt);
-                Job j = {slot, slot, hptr, dptr, d.bytes, hash, KVC_OK, false};
+                Job j = {slot, slot, hptr, dptr, d.bytes, hash, KVC_OK, false, nullptr};
                 submit(w, j);
                 ++reading;
                 ++st.reads;

@@ -1,6 +1,8 @@
 // Bounded staging ring (Sec. 6.4): a fixed pool of equal slots shared by every transfer; a
 // slot returns to the pool only after the event recorded behind its last copy has completed.
 // Host bookkeeping plus two events per slot; no kernel, no device-wide synchronisation.
+#include <stdlib.h>
+
 #include <chrono>
 #include <mutex>
 #include <new>
@@ -77,6 +79,8 @@ struct kvc_ring {
     unsigned char *dev_base;   // address for kernels and async copies
     unsigned char *host_base;  // host address (HOST_MAPPED) or nullptr
     bool owns_mem;
+    bool owns_host_part;       // DEVICE_STAGED: the pinned host half always belongs to the ring
+    bool host_part_is_malloc;  // ... and is plain memory when a test's event provider stands in for CUDA
     std::vector<Slot> slots;
     uint32_t head;             // next slot to hand out
     uint64_t acquires, stalls;
@@ -166,7 +170,8 @@ kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ri
     if (!out)
         return KVC_ERR_INVALID_ARG;
     *out = nullptr;
-    if (slot_bytes == 0 || n_slots == 0 || (kind != KVC_RING_DEVICE && kind != KVC_RING_HOST_MAPPED))
+    if (slot_bytes == 0 || n_slots == 0 ||
+        (kind != KVC_RING_DEVICE && kind != KVC_RING_HOST_MAPPED && kind != KVC_RING_DEVICE_STAGED))
         return KVC_ERR_INVALID_ARG;
     if (slot_bytes % 4096)
         return KVC_ERR_ALIGNMENT;
@@ -192,6 +197,8 @@ kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ri
     r->n_slots = n_slots;
     r->dev_base = r->host_base = nullptr;
     r->owns_mem = false;
+    r->owns_host_part = false;
+    r->host_part_is_malloc = false;
     r->head = 0;
     r->acquires = r->stalls = 0;
     r->trace = nullptr;
@@ -219,7 +226,7 @@ kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ri
                 }
             }
         }
-    } else if (kind == KVC_RING_DEVICE) {
+    } else if (kind == KVC_RING_DEVICE || kind == KVC_RING_DEVICE_STAGED) {
         void *p = nullptr;
         if (cudaMalloc(&p, total) != cudaSuccess) {
             (void)cudaGetLastError();
@@ -240,6 +247,22 @@ kvc_status kvc_staging_ring_create(uint64_t slot_bytes, uint32_t n_slots, kvc_ri
             r->host_base = static_cast<unsigned char *>(h);
             r->dev_base = static_cast<unsigned char *>(d);
             r->owns_mem = true;
+        }
+    }
+    if (rc == KVC_OK && kind == KVC_RING_DEVICE_STAGED) {
+        // the host half of every slot: pinned memory the copy engines can reach at full speed
+        void *h = nullptr;
+        if (r->custom_events) {
+            if (posix_memalign(&h, 4096, total) != 0)
+                rc = KVC_ERR_NOMEM;
+            r->host_part_is_malloc = rc == KVC_OK;
+        } else if (cudaHostAlloc(&h, total, cudaHostAllocDefault) != cudaSuccess) {
+            (void)cudaGetLastError();
+            rc = KVC_ERR_NOMEM;
+        }
+        if (rc == KVC_OK) {
+            r->host_base = static_cast<unsigned char *>(h);
+            r->owns_host_part = true;
         }
     }
     for (uint32_t i = 0; rc == KVC_OK && i < n_slots; ++i) {
@@ -275,8 +298,14 @@ kvc_status kvc_staging_ring_destroy(kvc_ring *r)
     if (r->policy)
         kvc_slot_pool_destroy(r->policy);
     if (r->owns_mem) {
-        if (r->kind == KVC_RING_DEVICE)
+        if (r->kind == KVC_RING_HOST_MAPPED)
+            cudaFreeHost(r->host_base);
+        else
             cudaFree(r->dev_base);
+    }
+    if (r->owns_host_part) {
+        if (r->host_part_is_malloc)
+            free(r->host_base);
         else
             cudaFreeHost(r->host_base);
     }
@@ -618,6 +647,7 @@ kvc_status kvc_staging_ring_policy_counters(kvc_ring *r, kvc_slot_pool_counters 
 }
 
 int kvc_staging_ring_pool_mode(const kvc_ring *r) { return r && r->policy ? 1 : 0; }
+kvc_ring_kind kvc_staging_ring_kind(const kvc_ring *r) { return r ? r->kind : KVC_RING_DEVICE; }
 uint64_t kvc_staging_ring_slot_bytes(const kvc_ring *r) { return r ? r->slot_bytes : 0; }
 uint32_t kvc_staging_ring_num_slots(const kvc_ring *r) { return r ? r->n_slots : 0; }
 

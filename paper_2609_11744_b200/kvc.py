@@ -25,7 +25,7 @@ KVC_OK, KVC_ERR_INVALID_ARG, KVC_ERR_OUT_OF_RANGE, KVC_ERR_ALIGNMENT, KVC_ERR_CO
     KVC_ERR_TOO_LARGE, KVC_ERR_EXISTS, KVC_ERR_NOT_FOUND, KVC_ERR_IO = range(14)
 KVC_VARIANT_AUTO, KVC_VARIANT_VEC, KVC_VARIANT_BULK = 0, 1, 2
 KVC_ORDER_AUTO, KVC_ORDER_PLANE_MAJOR, KVC_ORDER_BLOCK_MAJOR, KVC_ORDER_CHUNK_MAJOR = 0, 1, 2, 3
-KVC_RING_DEVICE, KVC_RING_HOST_MAPPED = 0, 1
+KVC_RING_DEVICE, KVC_RING_HOST_MAPPED, KVC_RING_DEVICE_STAGED = 0, 1, 2
 KVC_CHUNK_LAYER_MAJOR, KVC_CHUNK_BLOCK_MAJOR = 0, 1
 KVC_MAP_FULL_CHUNKS_ONLY = 1
 KVC_GROUP_FORCE_KERNEL = 0x100
@@ -180,6 +180,7 @@ def lib() -> ctypes.CDLL:
                                         P(kvc_load_many_stats)]),
         "kvc_store_get_counters": (ci, [vp, P(kvc_store_counters)]),
         "kvc_staging_ring_pool_mode": (ci, [vp]),
+        "kvc_staging_ring_kind": (ci, [vp]),
         "kvc_slot_pool_create": (ci, [u32, u32, u32, ci, P(vp)]),
         "kvc_slot_pool_destroy": (ci, [vp]),
         "kvc_slot_pool_acquire": (ci, [vp, ci, u64, P(u32), P(ci)]),
@@ -778,6 +779,10 @@ def kvc_store_get_counters(store) -> dict:
 
 def kvc_staging_ring_pool_mode(ring) -> bool:
     return bool(lib().kvc_staging_ring_pool_mode(ring.handle))
+
+
+def kvc_staging_ring_kind(ring) -> int:
+    return lib().kvc_staging_ring_kind(ring.handle)
 
 
 # ------------------------------------------------------------------ slot policy

@@ -117,6 +117,18 @@ int main()
     CHECK(kvc_staging_ring_trace_count(ring) > trace.size());  // counted past the buffer, not written
     CHECK(kvc_staging_ring_destroy(ring) == KVC_OK);
 
+    // ---- a staged ring: device half on caller memory, host half owned by the ring
+    CHECK(kvc_staging_ring_create(sb, n, KVC_RING_DEVICE_STAGED, mem, n * sb, &ring) == KVC_OK);
+    for (uint32_t i = 0; i < n; ++i) {
+        uint32_t slot = 0;
+        void *dp = nullptr, *hp = nullptr;
+        CHECK(kvc_staging_ring_acquire(ring, 0, &slot, &dp, &hp) == KVC_OK && hp && hp != dp);
+        memset(hp, 0x22, sb);
+        memset(dp, 0x33, sb);
+    }
+    CHECK(kvc_staging_ring_kind(ring) == KVC_RING_DEVICE_STAGED);
+    CHECK(kvc_staging_ring_destroy(ring) == KVC_OK);
+
     // ---- pool mode: random walk over classes, keys, joins, releases, cancels
     CHECK(kvc_staging_ring_create(sb, n, KVC_RING_DEVICE, mem, n * sb, &ring) == KVC_OK);
     CHECK(kvc_staging_ring_set_policy(ring, 2, 2, 1) == KVC_OK);

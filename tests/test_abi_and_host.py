@@ -544,6 +544,23 @@ def test_pool_mode_random_walk_keeps_its_invariants(fake_events, seed):
     kvc.kvc_staging_ring_destroy(ring)
 
 
+def test_staged_ring_has_a_device_half_and_a_host_half(fake_events):
+    n, sb = 3, 8192
+    mem = np.zeros(n * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    ring = kvc.kvc_staging_ring_create(sb, n, kvc.KVC_RING_DEVICE_STAGED, base, n * sb)
+    assert kvc.kvc_staging_ring_kind(ring) == kvc.KVC_RING_DEVICE_STAGED
+    seen = []
+    for i in range(n):
+        slot, dp, hp = kvc.kvc_staging_ring_acquire(ring)
+        assert dp == base + slot * sb and hp != 0 and hp % 4096 == 0
+        assert not (base <= hp < base + n * sb)              # a separate buffer, not an alias
+        ctypes.memset(hp, 0x40 + i, sb)                      # the whole host half is writable
+        seen.append(hp)
+    assert sorted(seen) == [seen[0] + i * sb for i in range(n)]
+    kvc.kvc_staging_ring_destroy(ring)
+
+
 def test_ring_create_validation(fake_events):
     for args, want in [((4096, 0, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
                        ((0, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),

@@ -15,15 +15,19 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda:0"
 
 
+@pytest.mark.parametrize("ring_kind", [kvc.KVC_RING_HOST_MAPPED, kvc.KVC_RING_DEVICE_STAGED])
 @pytest.mark.parametrize("use_copy_engine", [False, True])
-def test_store_then_load_through_files(tmp_path, use_copy_engine):
+def test_store_then_load_through_files(tmp_path, use_copy_engine, ring_kind):
     g = orc.Dims(6, 2, 96, 16, 8, 128, 2)            # 8B shape cut to 6 layers; chunk = 6 MiB
     pool = wl.random_bits(700, g.pool_bytes)
     pool_t = torch.from_numpy(pool).to(DEV)
     lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256)
     src, dst = wl.block_ids(71, g.NB, 44), wl.block_ids(72, g.NB, 44)     # 2 full chunks + 12 blocks
     cb = kvc.kvc_layout_chunk_bytes(lay, 16)
-    ring = kvc.kvc_staging_ring_create(cb, 2, kvc.KVC_RING_HOST_MAPPED)    # request > ring
+    ring = kvc.kvc_staging_ring_create(cb, 2, ring_kind)                  # request > ring
+    if ring_kind == kvc.KVC_RING_DEVICE_STAGED and not use_copy_engine:
+        # device halves at HBM speed, copy engines across the link: the set-up for a busy GPU
+        kvc.kvc_layout_set_tuning(lay, **kvc.kvc_tuning_preset(kvc.KVC_PRESET_BESIDE_COMPUTE))
     store = kvc.kvc_store_open(str(tmp_path), "shape-6x2x8x128-bf16", direct_io=True)
     tokens = np.arange(44 * 16, dtype=np.int32) * 7 + 3
     hashes, h = [], 0
@@ -78,8 +82,9 @@ def _hashes(seed, n_chunks, shared=0, shared_seed=999):
     return out
 
 
+@pytest.mark.parametrize("ring_kind", [kvc.KVC_RING_HOST_MAPPED, kvc.KVC_RING_DEVICE_STAGED])
 @pytest.mark.parametrize("pool_mode", [False, True])
-def test_failing_pack_inside_the_store_pipeline_returns_every_slot(tmp_path, pool_mode):
+def test_failing_pack_inside_the_store_pipeline_returns_every_slot(tmp_path, pool_mode, ring_kind):
     """An out-of-range block id in the third chunk: the call reports OUT_OF_RANGE, no slot stays
     taken, and the next store on the same ring runs normally."""
     g = orc.Dims(4, 2, 96, 16, 8, 128, 2)
@@ -87,7 +92,7 @@ def test_failing_pack_inside_the_store_pipeline_returns_every_slot(tmp_path, poo
     pool_t = torch.from_numpy(pool).to(DEV)
     lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256)
     cb = kvc.kvc_layout_chunk_bytes(lay, 16)
-    ring = kvc.kvc_staging_ring_create(cb, 3, kvc.KVC_RING_HOST_MAPPED)
+    ring = kvc.kvc_staging_ring_create(cb, 3, ring_kind)
     if pool_mode:
         kvc.kvc_staging_ring_set_policy(ring, 1)
     store = kvc.kvc_store_open(str(tmp_path), "m", direct_io=True)
@@ -134,7 +139,8 @@ def test_failing_pack_inside_the_store_pipeline_returns_every_slot(tmp_path, poo
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
 
 
-def test_four_requests_sharing_a_prefix_are_served_from_one_pool(tmp_path):
+@pytest.mark.parametrize("ring_kind", [kvc.KVC_RING_HOST_MAPPED, kvc.KVC_RING_DEVICE_STAGED])
+def test_four_requests_sharing_a_prefix_are_served_from_one_pool(tmp_path, ring_kind):
     """Four requests whose first 1024 tokens (4 chunks) are the same prefix, loaded at once through
     files and one staging pool (Sec. 6.5): every shared chunk is read once and joined by the other
     three requests, every request's blocks equal the oracle's, and chunks preloaded by an earlier
@@ -171,7 +177,7 @@ def test_four_requests_sharing_a_prefix_are_served_from_one_pool(tmp_path):
     for r in range(4):
         orc.unpack_request(g, want_pool, want_chunks[r], dsts[r], 256)
 
-    ring = kvc.kvc_staging_ring_create(cb, 6, kvc.KVC_RING_HOST_MAPPED)
+    ring = kvc.kvc_staging_ring_create(cb, 6, ring_kind)
     kvc.kvc_staging_ring_set_policy(ring, foreground_reserve=2, max_speculative=4)
     reads0 = kvc.kvc_store_get_counters(store)["reads"]
     # 1. a preload of request 2's prefix, issued before anything is scheduled
