@@ -1212,6 +1212,126 @@ def suite_file_pipeline(torch, kvc, dev, root):
     return out
 
 
+def suite_pipeline_beside_gemm(torch, kvc, dev, roots):
+    """The paper's actual situation (Sec. 2.3, 5.1): chunks go to storage while the model computes.
+    A 4 GiB request (8B shape) is offloaded to chunk files again and again while a bf16 8192^3
+    matmul loop of about 3 s runs on another stream; then loaded back the same way.  Mapped pinned
+    slots written / read by the kernels themselves against device + pinned-host slot pairs with the
+    beside-compute kernel shape and copy-engine transfers.  Files on the memory-backed file system
+    when there is one (the scratch disk would only measure the disk)."""
+    import shutil
+    import tempfile
+    w = wl.WORKLOADS["8b_ring"]
+    s, NB, n = w.shape, w.pool_blocks, w.request_blocks
+    pool = wl.random_bits_cuda(w.seed, NB * s.bytes_per_block, dev)
+    src, dst = wl.block_ids(w.seed, NB, n), wl.block_ids(w.dst_seed, NB, n)
+    lo, hi = torch.cuda.Stream.priority_range()
+    s_gemm, s_io = torch.cuda.Stream(priority=lo), torch.cuda.Stream(priority=hi)
+    N, GRAPH_ITERS = 8192, 64
+    A = torch.randn(N, N, device=dev, dtype=torch.bfloat16)
+    B = torch.randn(N, N, device=dev, dtype=torch.bfloat16)
+    C = torch.empty(N, N, device=dev, dtype=torch.bfloat16)
+    with torch.cuda.stream(s_gemm):
+        for _ in range(5):
+            torch.matmul(A, B, out=C)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=s_gemm):
+        for _ in range(GRAPH_ITERS):
+            torch.matmul(A, B, out=C)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+    def gemm_loop(replays):
+        e0.record(s_gemm)
+        with torch.cuda.stream(s_gemm):
+            for _ in range(replays):
+                graph.replay()
+        e1.record(s_gemm)
+
+    gemm_loop(4)
+    torch.cuda.synchronize()
+    replays = max(8, int(3000.0 / (e0.elapsed_time(e1) / 4)))
+    gemm_loop(replays)
+    torch.cuda.synchronize()
+    t_alone = e0.elapsed_time(e1)
+    roots_ok = [r for r in roots.split(",") if os.path.isdir(r)]
+    base = "/dev/shm" if "/dev/shm" in roots_ok else (roots_ok[0] if roots_ok else None)
+    out = {"gemm": "bf16 %d^3 matmul loop, %d launches" % (N, replays * GRAPH_ITERS), "gemm_alone_ms": t_alone,
+           "files_on": base, "runs": []}
+    if base is None:
+        return out
+    for kind, name in ((kvc.KVC_RING_HOST_MAPPED, "mapped pinned slots, kernels cross the link (16 blocks)"),
+                       (kvc.KVC_RING_DEVICE_STAGED, "device + pinned-host slot pairs, beside-compute kernels, "
+                                                    "copy engines cross the link")):
+        d = tempfile.mkdtemp(prefix="kvc_gemm_", dir=base)
+        try:
+            lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 256)
+            if kind == kvc.KVC_RING_DEVICE_STAGED:
+                kvc.kvc_layout_set_tuning(lay, **kvc.kvc_tuning_preset(kvc.KVC_PRESET_BESIDE_COMPUTE))
+            else:
+                kvc.kvc_layout_set_tuning(lay, max_ctas=16)
+            cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
+            ring = kvc.kvc_staging_ring_create(cb, 16, kind)
+            kvc.kvc_staging_ring_set_policy(ring, 0)
+            n_chunks = kvc.kvc_layout_num_chunks(lay, n)
+            for direction in ("store", "load"):
+                stores = []
+
+                def one_pass(k):
+                    if direction == "store":
+                        store = kvc.kvc_store_open(os.path.join(d, "p%d" % k), "8b", direct_io=True)
+                        hashes = [kvc.kvc_fnv1a64(b"c%d" % c) for c in range(n_chunks)]
+                        st = kvc.kvc_pipeline_store(lay, ring, store, src, hashes, io_threads=8, stream=s_io)
+                        stores.append((store, hashes))
+                        return st["bytes"]
+                    store, hashes = loaded
+                    st, _ = kvc.kvc_pipeline_load_many(
+                        lay, ring, store, [dict(ids=dst, hashes=hashes, cls=kvc.KVC_CLASS_DEMAND_LOAD)],
+                        io_threads=8, stream=s_io)
+                    s_io.synchronize()
+                    return st["bytes_read"]
+
+                if direction == "load":
+                    loaded = keep_store
+                res = {}
+                for with_gemm in (False, True):
+                    os.makedirs(d, exist_ok=True)
+                    torch.cuda.synchronize()
+                    if with_gemm:
+                        gemm_loop(replays)
+                    t0 = time.perf_counter()
+                    moved, k = 0, 0
+                    while True:
+                        moved += one_pass(k)
+                        k += 1
+                        elapsed = time.perf_counter() - t0
+                        if (with_gemm and e1.query()) or (not with_gemm and elapsed > 1.5) or k >= 24:
+                            break
+                    s_io.synchronize()
+                    elapsed = time.perf_counter() - t0
+                    torch.cuda.synchronize()
+                    res["with_gemm" if with_gemm else "alone"] = moved / elapsed / 1e9
+                    if with_gemm:
+                        res["gemm_slowdown"] = e0.elapsed_time(e1) / t_alone
+                    if direction == "store":
+                        keep_store = stores[0]
+                        for st_, _h in stores[1:]:
+                            kvc.kvc_store_close(st_)
+                        for kk in range(1, k):
+                            shutil.rmtree(os.path.join(d, "p%d" % kk), ignore_errors=True)
+                        stores = []
+                out["runs"].append({"slots": name, "direction": direction, "file_gbs_alone": res["alone"],
+                                    "file_gbs_beside_gemm": res["with_gemm"],
+                                    "gemm_slowdown": res["gemm_slowdown"]})
+            assert kvc.kvc_poll_device_status(lay) == (0, 0)
+            kvc.kvc_store_close(keep_store[0])
+            kvc.kvc_staging_ring_destroy(ring)
+            kvc.kvc_layout_destroy(lay)
+        finally:
+            shutil.rmtree(d, ignore_errors=True)
+    return out
+
+
 def suite_preload_trace(torch, kvc, dev, roots):
     """Sec. 6.5 in miniature: a queue of requests, each needing its 2048-token prefix (8 chunks of
     32 MiB, 8B shape; the first 1024 tokens are common to all) loaded from chunk files before a
@@ -1331,7 +1451,9 @@ def run_suite(args):
                                                                  args.overlap_seconds)),
                      ("duplex", lambda: suite_duplex(torch, kvc, cuda_rt, dev, args.steps)),
                      ("file_pipeline", lambda: suite_file_pipeline(torch, kvc, dev, args.file_roots)),
-                     ("preload_trace", lambda: suite_preload_trace(torch, kvc, dev, args.file_roots))):
+                     ("preload_trace", lambda: suite_preload_trace(torch, kvc, dev, args.file_roots)),
+                     ("pipeline_beside_gemm", lambda: suite_pipeline_beside_gemm(torch, kvc, dev,
+                                                                                 args.file_roots))):
         if "all" in parts or name in parts:
             out[name] = fn()
             torch.cuda.synchronize()
@@ -1366,7 +1488,8 @@ def main():
     ap.add_argument("--suite", default="",
                     help="run the other configs instead of the bench step: all, or a comma list of "
                          "host_link,launch_shapes,chunk_sweep,small_slabs,row_gather,call_overhead,prefix_8k,batch_70b,"
-                         "ring_overlap,duplex,file_pipeline,preload_trace (1 GPU; prints one JSON line)")
+                         "ring_overlap,duplex,file_pipeline,preload_trace,pipeline_beside_gemm (1 GPU; prints "
+                         "one JSON line)")
     ap.add_argument("--small-slab-sizes", default="",
                     help="small_slabs suite part: comma list of slab sizes in bytes (default: all)")
     ap.add_argument("--small-slab-mib", type=int, default=2048,
