@@ -561,6 +561,39 @@ def test_staged_ring_has_a_device_half_and_a_host_half(fake_events):
     kvc.kvc_staging_ring_destroy(ring)
 
 
+def test_load_many_argument_checks_need_no_gpu(fake_events, tmp_path):
+    """What kvc_pipeline_load_many decides before it touches the GPU: the ring must be in pool mode,
+    classes must be demand load or preload, hashes must cover the chunks, and a request none of whose
+    chunks is in the store is simply empty."""
+    lay = _layout(chunk_tokens=64, NB=64)
+    store = kvc.kvc_store_open(str(tmp_path), "m", direct_io=False)
+    sb = kvc.kvc_layout_chunk_bytes(lay, 4)                               # a whole chunk fits a slot
+    mem = np.zeros(4 * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    fifo = kvc.kvc_staging_ring_create(sb, 4, kvc.KVC_RING_DEVICE, base, 4 * sb)
+    ids = np.arange(10, dtype=np.int32)
+    req = dict(ids=ids, hashes=[1, 2, 3], cls=kvc.KVC_CLASS_DEMAND_LOAD)
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_pipeline_load_many(lay, fifo, store, [req])
+    assert e.value.status == kvc.KVC_ERR_STATE
+    kvc.kvc_staging_ring_set_policy(fifo, 1)
+    stats, res = kvc.kvc_pipeline_load_many(lay, fifo, store, [req])      # nothing stored: nothing to do
+    assert (stats["chunks"], stats["reads"], stats["unpack_launches"]) == (0, 0, 0)
+    assert res[0]["loaded_chunks"] == 0
+    with pytest.raises(kvc.KvcError) as e:                                # 10 blocks = 3 chunks, 2 hashes
+        kvc.kvc_pipeline_load_many(lay, fifo, store, [dict(ids=ids, hashes=[1, 2], cls=0)])
+    assert e.value.status == kvc.KVC_ERR_INVALID_ARG
+    with pytest.raises(kvc.KvcError) as e:                                # stores are not loads
+        kvc.kvc_pipeline_load_many(lay, fifo, store, [dict(ids=ids, hashes=[1, 2, 3], cls=kvc.KVC_CLASS_STORE)])
+    assert e.value.status == kvc.KVC_ERR_INVALID_ARG
+    stats, res = kvc.kvc_pipeline_load_many(lay, fifo, store, [])
+    assert stats["chunks"] == 0 and res == []
+    c = kvc.kvc_staging_ring_policy_counters(fifo)
+    assert c["n_free"] == 4 and c["acquires"] == 0
+    kvc.kvc_staging_ring_destroy(fifo)
+    kvc.kvc_store_close(store)
+
+
 def test_ring_create_validation(fake_events):
     for args, want in [((4096, 0, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
                        ((0, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
