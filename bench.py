@@ -404,8 +404,25 @@ def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, di
     descs = kvc.kvc_map_request(lay, len(src))
     cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
     slot_bytes = (cb + 4095) // 4096 * 4096
-    ring = kvc.kvc_staging_ring_create(slot_bytes, args.ring_slots, kvc.KVC_RING_DEVICE)
-    host = torch.empty(one_way, dtype=torch.uint8, pin_memory=True)
+    # Every rank pins a host buffer as large as the prefix.  If one of them cannot (N replicas share
+    # the host's memory), all of them skip this leg together: the ranks meet in collectives below.
+    ring = host = None
+    problem = ""
+    try:
+        ring = kvc.kvc_staging_ring_create(slot_bytes, args.ring_slots, kvc.KVC_RING_DEVICE)
+        host = torch.empty(one_way, dtype=torch.uint8, pin_memory=True)
+    except Exception as e:  # out of pinned or device memory
+        problem = "%s: %s" % (type(e).__name__, str(e)[:200])
+    ok = 0.0 if problem else 1.0
+    if world > 1:
+        t = torch.tensor([ok], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MIN)
+        ok = float(t.item())
+    if ok < 1.0:
+        if ring is not None:
+            kvc.kvc_staging_ring_destroy(ring)
+        return {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                "unavailable": problem or "another rank could not allocate its staging memory"}
     hptr = host.data_ptr()
     s_k, s_c = torch.cuda.Stream(), torch.cuda.Stream()
     TO = 10_000_000
