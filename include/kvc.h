@@ -294,7 +294,8 @@ kvc_status kvc_poll_device_status(kvc_layout *layout, void *stream, uint32_t *n_
  * ops, and at most KVC_STATIC_MAX_PLANES planes for layouts given as plane pointers; beyond
  * either the call returns KVC_ERR_TOO_LARGE and enqueues nothing.
  * The tables travel to the device inside the parameters of small kernels enqueued on `stream`
- * ahead of the copy kernel (one per 32 KiB of table: 1 to 9 launches), so the call does not wait
+ * ahead of the copy kernel -- chunk records and 4-byte ids, expanded into table entries on the
+ * device: one launch per ~32 KiB of those, typically one or two -- so the call does not wait
  * for the stream and the host arrays may be reused as soon as it returns.
  * The first call on a device looks up the array's device address and the device's limits; make
  * that first call outside any stream capture.  Every call shares the one array, which keeps the

@@ -16,7 +16,8 @@
 // streams) race on it.
 //
 // The tables reach the device inside kernel parameters: a tiny kernel stores its own parameter
-// block into the array.  A launch copies its parameters before it returns, so the host-side
+// block into the array (the plane pointers), or expands the compact chunk records and ids it
+// carries into table entries.  A launch copies its parameters before it returns, so the host-side
 // staging buffer can be refilled at once, the call never waits for the stream (an asynchronous
 // copy from pageable memory would: the runtime documents that it first synchronises the stream
 // and returns only when the bytes sit in a driver staging buffer), and no pinned buffer -- which
@@ -58,6 +59,45 @@ __global__ void __launch_bounds__(256) kvc_static_upload_kernel(const __grid_con
         dst[i] = p.data[i];
 }
 
+// The id table is not shipped entry by entry (32 bytes per block) but in the compact form the
+// caller gave it -- one record per chunk and 4 bytes per block id -- and expanded on the device:
+// one thread block per chunk writes that chunk's entries.  A parameter block of 32 KiB carries
+// about 5000 blocks in 256-token chunks, so a typical call needs one or two of these launches.
+struct ChunkRec {
+    uint64_t slot;        // chunk base in the staging memory
+    uint64_t ent_step;    // bytes between consecutive blocks of a plane inside the chunk
+    uint64_t plane_step;  // bytes between consecutive planes of a block inside the chunk
+    uint32_t first_ent;   // index of the chunk's first table entry
+    uint32_t n_blocks;
+    uint32_t ids_off;     // where the chunk's ids start in the id area of this parameter block
+    uint32_t pad;
+};
+static_assert(sizeof(ChunkRec) == 40, "parameter block layout");
+constexpr uint32_t kExpandPayload = 32512;  // bytes: ChunkRec[n_chunks], then int32 ids
+struct alignas(16) ExpandParams {
+    uint32_t n_chunks;
+    uint32_t ids_at;  // byte offset of the id area inside payload (8-byte aligned)
+    uint32_t pad[2];
+    unsigned char payload[kExpandPayload];
+};
+static_assert(sizeof(ExpandParams) <= 32764, "parameter block too large");
+
+__global__ void __launch_bounds__(128) kvc_static_expand_kernel(const __grid_constant__ ExpandParams p)
+{
+    const ChunkRec c = reinterpret_cast<const ChunkRec *>(p.payload)[blockIdx.x];
+    const int32_t *ids = reinterpret_cast<const int32_t *>(p.payload + p.ids_at) + c.ids_off;
+    KvcEnt *table = reinterpret_cast<KvcEnt *>(kvc_static_scratch + kTableOffset);
+    for (uint32_t j = threadIdx.x; j < c.n_blocks; j += blockDim.x) {
+        KvcEnt e;
+        e.slot_addr = c.slot + (uint64_t)j * c.ent_step;
+        e.id_or_ptr = (uint64_t)(uint32_t)ids[j];
+        e.plane_step = c.plane_step;
+        e.nb_c = c.n_blocks;
+        e.first_ent = c.first_ent;
+        table[c.first_ent + j] = e;
+    }
+}
+
 constexpr int kMaxDevices = 64;
 struct DeviceSetup {
     bool ready;
@@ -68,6 +108,7 @@ struct DeviceSetup {
 std::mutex g_mu;
 DeviceSetup g_setup[kMaxDevices];
 UploadParams g_params;        // host-side staging of one parameter block
+ExpandParams g_expand;        // ... and of one compact table block
 uint32_t g_host_status[2];    // landing place of kvc_poll_static_status
 
 // Once per device, with that device current.  Caller holds g_mu.
@@ -185,29 +226,75 @@ extern "C" kvc_status kvc_pack_batch_static(kvc_layout *lay, const kvc_chunk_op 
         if (s != KVC_OK)
             return s;
     }
-    // the id table, one parameter block at a time
-    static KvcEnt ents[kUploadVecs / 2];
-    uint32_t filled = 0, base = 0;
-    uint64_t k = 0;
-    for (uint32_t i = 0; i < n_ops; ++i) {
-        uint64_t ent_step, plane_step;
-        kvc_chunk_steps(lay, ops[i].n_blocks, &ent_step, &plane_step);
-        const uint32_t first = (uint32_t)k;
-        for (uint32_t j = 0; j < ops[i].n_blocks; ++j, ++k) {
-            KvcEnt &e = ents[filled++];
-            e.slot_addr = (uint64_t)(uintptr_t)ops[i].slot + (uint64_t)j * ent_step;
-            e.id_or_ptr = (uint64_t)(uint32_t)ops[i].ids[j];
-            e.plane_step = plane_step;
-            e.nb_c = ops[i].n_blocks;
-            e.first_ent = first;
-            if (filled == kUploadVecs / 2 || k + 1 == n_ent) {
-                s = upload(kTableOffset + base * (uint32_t)sizeof(KvcEnt), ents,
-                           (uint64_t)filled * sizeof(KvcEnt), st);
-                if (s != KVC_OK)
-                    return s;
-                base += filled;
-                filled = 0;
+    // the id table, in compact form: as many whole chunks per parameter block as fit
+    {
+        uint64_t k = 0;     // table entries described so far
+        uint32_t i = 0;     // next op
+        while (i < n_ops) {
+            // how many ops fit: 40 bytes per chunk record + 4 bytes per id (+ alignment slack)
+            uint32_t n_c = 0, n_ids = 0, j = i;
+            for (; j < n_ops; ++j) {
+                if (ops[j].n_blocks == 0)
+                    continue;
+                const uint64_t need = (uint64_t)(n_c + 1) * sizeof(ChunkRec) + 8 +
+                                      (uint64_t)(n_ids + ops[j].n_blocks) * sizeof(int32_t);
+                if (need > kExpandPayload)
+                    break;
+                ++n_c;
+                n_ids += ops[j].n_blocks;
             }
+            if (n_c == 0) {
+                if (j >= n_ops)
+                    break;  // only empty ops were left
+                // a single chunk with more ids than one parameter block holds: ship its entries
+                // ready-made, 32 bytes each, through the plain upload path
+                static KvcEnt ents[kUploadVecs / 2];
+                uint64_t ent_step, plane_step;
+                kvc_chunk_steps(lay, ops[j].n_blocks, &ent_step, &plane_step);
+                const uint32_t first = (uint32_t)k;
+                uint32_t filled = 0, base = first;
+                for (uint32_t b = 0; b < ops[j].n_blocks; ++b) {
+                    KvcEnt &e = ents[filled++];
+                    e.slot_addr = (uint64_t)(uintptr_t)ops[j].slot + (uint64_t)b * ent_step;
+                    e.id_or_ptr = (uint64_t)(uint32_t)ops[j].ids[b];
+                    e.plane_step = plane_step;
+                    e.nb_c = ops[j].n_blocks;
+                    e.first_ent = first;
+                    if (filled == kUploadVecs / 2 || b + 1 == ops[j].n_blocks) {
+                        s = upload(kTableOffset + base * (uint32_t)sizeof(KvcEnt), ents,
+                                   (uint64_t)filled * sizeof(KvcEnt), st);
+                        if (s != KVC_OK)
+                            return s;
+                        base += filled;
+                        filled = 0;
+                    }
+                }
+                k += ops[j].n_blocks;
+                i = j + 1;
+                continue;
+            }
+            g_expand.n_chunks = n_c;
+            g_expand.ids_at = (uint32_t)((n_c * sizeof(ChunkRec) + 7u) & ~7u);
+            ChunkRec *recs = reinterpret_cast<ChunkRec *>(g_expand.payload);
+            int32_t *ids_area = reinterpret_cast<int32_t *>(g_expand.payload + g_expand.ids_at);
+            uint32_t c = 0, ids_off = 0;
+            for (; i < j; ++i) {
+                if (ops[i].n_blocks == 0)
+                    continue;
+                ChunkRec &r = recs[c++];
+                r.slot = (uint64_t)(uintptr_t)ops[i].slot;
+                kvc_chunk_steps(lay, ops[i].n_blocks, &r.ent_step, &r.plane_step);
+                r.first_ent = (uint32_t)k;
+                r.n_blocks = ops[i].n_blocks;
+                r.ids_off = ids_off;
+                r.pad = 0;
+                memcpy(ids_area + ids_off, ops[i].ids, (size_t)ops[i].n_blocks * sizeof(int32_t));
+                ids_off += ops[i].n_blocks;
+                k += ops[i].n_blocks;
+            }
+            kvc_static_expand_kernel<<<n_c, 128, 0, st>>>(g_expand);
+            if (cudaGetLastError() != cudaSuccess)
+                return KVC_ERR_CUDA;
         }
     }
     unsigned char *scratch = dev->scratch;

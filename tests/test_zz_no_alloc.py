@@ -122,3 +122,40 @@ def test_static_pack_rejects_what_it_cannot_hold():
     assert np.array_equal(host[:want.size], want)
     assert (host[want.size:] == 0).all()
     assert kvc.kvc_poll_static_status() == (0, 0)
+
+
+def test_static_pack_of_thousands_of_small_chunks_with_empty_ops_between():
+    """The table travels as chunk records plus ids and is expanded on the device; thousands of
+    one-to-five-block chunks need several such launches, and empty ops sit between them and at
+    both ends.  Every chunk against the oracle, the gaps between chunks untouched."""
+    s = wl.TINY
+    NB = 1500
+    g = orc.Dims(s.L, s.P, NB, s.B, s.H, s.D, s.e)
+    pool_np = wl.random_bits(wl.BASE_SEED + 930, g.pool_bytes)
+    pool = torch.from_numpy(pool_np).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool, s.L, s.P, NB, s.B, s.H, s.D, s.e, 16 * 8)
+    rng = np.random.default_rng(wl.BASE_SEED + 931)
+    sizes, total = [0], 0
+    while total + 5 <= kvc.KVC_STATIC_MAX_BLOCKS - 3:
+        n = int(rng.integers(1, 6)) if rng.random() > 0.05 else 0
+        sizes.append(n)
+        total += n
+    sizes += [3, 0]
+    total += 3
+    assert sum(1 for n in sizes if n) > 2400
+    stride = 5 * s.bytes_per_block + 64                    # a gap behind every chunk
+    staging = torch.full((len(sizes) * stride,), 0x77, dtype=torch.uint8, device=DEV)
+    ids = [rng.integers(0, NB, size=max(n, 1)).astype(np.int32) for n in sizes]   # repeats allowed
+    ops = kvc.make_chunk_ops([staging.data_ptr() + i * stride for i in range(len(sizes))],
+                             [a.ctypes.data for a in ids], sizes)
+    kvc.kvc_pack_batch_static(lay, ops)
+    torch.cuda.synchronize()
+    host = staging.cpu().numpy()
+    for i, n in enumerate(sizes):
+        lo = i * stride
+        if n:
+            want = orc.pack_chunk(g, pool_np, ids[i][:n])
+            assert np.array_equal(host[lo:lo + want.size], want), i
+            lo += want.size
+        assert (host[lo:(i + 1) * stride] == 0x77).all(), i
+    assert kvc.kvc_poll_static_status() == (0, 0)
