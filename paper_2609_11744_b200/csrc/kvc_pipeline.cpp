@@ -20,7 +20,6 @@
 // Every exit, error exits included, hands every slot it took back to the staging memory.
 #include <chrono>
 #include <condition_variable>
-#include <deque>
 #include <map>
 #include <mutex>
 #include <new>
@@ -84,11 +83,32 @@ struct Job {
     cudaEvent_t copied;  // DEVICE_STAGED store: the event behind the slot's device-to-host copy
 };
 
+// A queue of jobs with all its memory taken up front: a job holds a staging slot, so there are never
+// more jobs than slots, and neither the calling thread nor an I/O thread (where an allocation
+// failure could not be reported) allocates while the pipeline runs.
+struct JobQueue {
+    std::vector<Job> buf;
+    size_t head = 0, count = 0;
+    bool empty() const { return count == 0; }
+    void push(const Job &j)
+    {
+        buf[(head + count) % buf.size()] = j;
+        ++count;
+    }
+    Job pop()
+    {
+        const Job j = buf[head];
+        head = (head + 1) % buf.size();
+        --count;
+        return j;
+    }
+};
+
 // Work queue for the I/O threads and completion queue back to the calling thread.
 struct Queues {
     std::mutex mu;
     std::condition_variable work_cv, done_cv;
-    std::deque<Job> work, done;
+    JobQueue work, done;
     bool closing = false;
 };
 
@@ -101,8 +121,7 @@ void io_worker(Queues *q, kvc_ring *ring, kvc_store *store, bool storing)
             q->work_cv.wait(lk, [&] { return q->closing || !q->work.empty(); });
             if (q->closing)
                 return;  // jobs still queued are dropped; the caller returns their slots
-            j = q->work.front();
-            q->work.pop_front();
+            j = q->work.pop();
         }
         if (storing) {
             // the slot's copy was only enqueued: wait for its "filled" event (or, for a staged
@@ -123,7 +142,7 @@ void io_worker(Queues *q, kvc_ring *ring, kvc_store *store, bool storing)
         }
         {
             std::lock_guard<std::mutex> lk(q->mu);
-            q->done.push_back(j);
+            q->done.push(j);
         }
         q->done_cv.notify_one();
     }
@@ -133,13 +152,13 @@ struct Workers {
     Queues q;
     std::vector<std::thread> threads;
     // Stops the threads after the job each one is running; returns the jobs that never started.
-    std::deque<Job> stop()
+    JobQueue stop()
     {
-        std::deque<Job> dropped;
+        JobQueue dropped;
         {
             std::lock_guard<std::mutex> lk(q.mu);
             q.closing = true;
-            dropped.swap(q.work);
+            std::swap(dropped, q.work);  // (moves the buffers: nothing is allocated)
         }
         q.work_cv.notify_all();
         for (std::thread &t : threads)
@@ -161,6 +180,9 @@ bool start_workers(Workers &w, uint32_t io_threads, kvc_ring *ring, kvc_store *s
 {
     const uint32_t n = io_threads ? io_threads : 4;
     try {
+        const size_t cap = (size_t)kvc_staging_ring_num_slots(ring) + 1;
+        w.q.work.buf.resize(cap);
+        w.q.done.buf.resize(cap);
         for (uint32_t i = 0; i < n; ++i)
             w.threads.emplace_back(io_worker, &w.q, ring, store, storing);
     } catch (...) {
@@ -173,7 +195,7 @@ void submit(Workers &w, const Job &j)
 {
     {
         std::lock_guard<std::mutex> lk(w.q.mu);
-        w.q.work.push_back(j);
+        w.q.work.push(j);
     }
     w.q.work_cv.notify_one();
 }
@@ -184,10 +206,8 @@ void collect(Workers &w, bool block, std::vector<Job> *out)
     std::unique_lock<std::mutex> lk(w.q.mu);
     if (block && w.q.done.empty())
         w.q.done_cv.wait_for(lk, std::chrono::milliseconds(200));
-    while (!w.q.done.empty()) {
-        out->push_back(w.q.done.front());
-        w.q.done.pop_front();
-    }
+    while (!w.q.done.empty())
+        out->push_back(w.q.done.pop());
 }
 
 // One slot for (cls, key): FIFO order for a plain ring, the slot policy for a pool.
@@ -241,6 +261,7 @@ kvc_status run_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const in
     uint32_t issued = 0, finished = 0;
     kvc_status first_err = KVC_OK;
     std::vector<Job> done;
+    done.reserve((size_t)kvc_staging_ring_num_slots(ring) + 1);
     auto reap = [&](bool block) {
         done.clear();
         collect(w, block && finished < issued, &done);
@@ -336,9 +357,10 @@ kvc_status run_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const in
     // Drain.  After an error nothing new starts: jobs not yet picked up are dropped, and their
     // slots go back once the copy that was enqueued into them has run.
     if (first_err != KVC_OK) {
-        std::deque<Job> dropped = w.stop();
+        JobQueue dropped = w.stop();
         reap(false);
-        for (const Job &j : dropped) {
+        while (!dropped.empty()) {
+            const Job j = dropped.pop();
             kvc_staging_ring_sync_filled(ring, j.slot);
             if (j.copied)
                 cudaEventSynchronize(j.copied);
@@ -351,9 +373,10 @@ kvc_status run_store(kvc_layout *lay, kvc_ring *ring, kvc_store *store, const in
     if (finished < issued) {
         // out of time with writes still running: wait for the threads (each finishes its current
         // file), then return what is left
-        std::deque<Job> dropped = w.stop();
+        JobQueue dropped = w.stop();
         reap(false);
-        for (const Job &j : dropped) {
+        while (!dropped.empty()) {
+            const Job j = dropped.pop();
             kvc_staging_ring_sync_filled(ring, j.slot);
             if (j.copied)
                 cudaEventSynchronize(j.copied);
@@ -448,6 +471,22 @@ kvc_status run_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, kvc_load_
     } catch (const std::bad_alloc &) {
         return KVC_ERR_NOMEM;
     }
+    std::vector<std::pair<Waiter, uint32_t>> ready;  // (who, slot) whose bytes are in the slot
+    std::vector<Job> done;
+    std::vector<kvc_chunk_op> ops;
+    try {
+        // everything the loop below appends to, at its largest possible size
+        ready.reserve(pending.size());
+        ops.reserve(pending.size());
+        done.reserve((size_t)n_slots + 1);
+        size_t most = 1;  // the most requests that can wait for one chunk
+        for (const auto &kv : by_hash)
+            most = kv.second.size() > most ? kv.second.size() : most;
+        for (SlotWork &sw : slots)
+            sw.waiters.reserve(most);
+    } catch (const std::bad_alloc &) {
+        return KVC_ERR_NOMEM;
+    }
     StagedCopies staged;
     {
         const kvc_status rc = staged.start(ring);
@@ -461,9 +500,6 @@ kvc_status run_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, kvc_load_
     kvc_status first_err = KVC_OK;
     size_t next = 0;           // next entry of `pending` to issue
     uint32_t reading = 0;      // read jobs in flight
-    std::vector<std::pair<Waiter, uint32_t>> ready;  // (who, slot) whose bytes are in the slot
-    std::vector<Job> done;
-    std::vector<kvc_chunk_op> ops;
     const double deadline = now_s() + kDeadlineSeconds;
     double preload_refused_since = -1;
     auto note_error = [&](kvc_status s) {
@@ -665,10 +701,10 @@ kvc_status run_load(kvc_layout *lay, kvc_ring *ring, kvc_store *store, kvc_load_
     if (first_err != KVC_OK) {
         // Error exit: nothing new starts.  Reads that never started give their slots back at once,
         // reads in progress are waited for, and every reference this call still holds is dropped.
-        std::deque<Job> dropped = w.stop();
+        JobQueue dropped = w.stop();
         collect(w, false, &done);
-        for (const Job &j : dropped)
-            done.push_back(j);
+        while (!dropped.empty())
+            done.push_back(dropped.pop());
         for (const Job &j : done) {
             SlotWork &sw = slots[j.slot];
             kvc_staging_ring_commit_host(ring, j.slot);
