@@ -239,6 +239,15 @@ kvc_status kvc_launch_timed(kvc_layout *lay, int dir, int variant, const KvcLaun
                             uint32_t smem, cudaStream_t st)
 {
     cudaEvent_t e0 = nullptr, e1 = nullptr;
+    // on a failure the events taken for this launch are destroyed, not leaked
+    auto fail = [&](kvc_status s) {
+        (void)cudaGetLastError();
+        if (e0)
+            cudaEventDestroy(e0);
+        if (e1)
+            cudaEventDestroy(e1);
+        return s;
+    };
     if (lay->time_kernels) {
         cudaEvent_t *ev[2] = {&e0, &e1};
         for (cudaEvent_t *e : ev) {
@@ -246,22 +255,24 @@ kvc_status kvc_launch_timed(kvc_layout *lay, int dir, int variant, const KvcLaun
                 *e = lay->spare_events.back();
                 lay->spare_events.pop_back();
             } else if (cudaEventCreate(e) != cudaSuccess) {
-                return KVC_ERR_CUDA;
+                *e = nullptr;
+                return fail(KVC_ERR_CUDA);
             }
         }
+        try {
+            lay->timed.reserve(lay->timed.size() + 1);
+        } catch (const std::bad_alloc &) {
+            return fail(KVC_ERR_NOMEM);
+        }
         if (cudaEventRecord(e0, st) != cudaSuccess)
-            return KVC_ERR_CUDA;
+            return fail(KVC_ERR_CUDA);
     }
     if (kvc_launch_copy(dir, variant, a, grid, smem, st) != cudaSuccess)
-        return KVC_ERR_CUDA;
+        return fail(KVC_ERR_CUDA);
     if (lay->time_kernels) {
         if (cudaEventRecord(e1, st) != cudaSuccess)
-            return KVC_ERR_CUDA;
-        try {
-            lay->timed.emplace_back(e0, e1);
-        } catch (const std::bad_alloc &) {
-            return KVC_ERR_NOMEM;
-        }
+            return fail(KVC_ERR_CUDA);
+        lay->timed.emplace_back(e0, e1);  // room was reserved above
     }
     ++lay->launches;
     return KVC_OK;
