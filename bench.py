@@ -582,9 +582,23 @@ def suite_chunk_sweep(torch, kvc, dev, reps):
                       lambda: per_chunk_streams(1, dst)))
         # the same one-stream loop with the launches declared independent of one another (pdl = 3)
         modes.append(("per_chunk_independent", lambda: per_chunk(0, src), lambda: per_chunk(1, dst)))
+        # ... and both one-stream loops captured once into a CUDA graph and replayed: no host work
+        # per chunk at all (host ids travel in the kernel parameters, so a captured call is
+        # self-contained)
+        modes.append(("per_chunk_graph", None, None))
+        modes.append(("per_chunk_independent_graph", None, None))
         for name, fp, fu in modes:
-            kvc.kvc_layout_set_tuning(lay, pdl=3 if name == "per_chunk_independent" else 0,
-                                      slot_memory=1)
+            kvc.kvc_layout_set_tuning(lay, pdl=3 if "independent" in name else 0, slot_memory=1)
+            if name.endswith("_graph"):
+                graphs = []
+                for direction, ids in ((0, src), (1, dst)):
+                    per_chunk(direction, ids)              # the launch shape's first use, outside capture
+                    torch.cuda.synchronize()
+                    gr = torch.cuda.CUDAGraph()
+                    with torch.cuda.graph(gr):
+                        per_chunk(direction, ids)
+                    graphs.append(gr)
+                fp, fu = graphs[0].replay, graphs[1].replay
             # 5000 single-chunk launches of 2 MiB are launch-bound by design: fewer repetitions
             r = reps if len(descs) <= 400 or name == "batch" else max(3, reps // 4)
             pm, pd = _time_ms(torch, fp, r)
