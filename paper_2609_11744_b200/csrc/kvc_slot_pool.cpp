@@ -178,13 +178,13 @@ kvc_status kvc_slot_pool_acquire(kvc_slot_pool *p, kvc_slot_class cls, uint64_t 
             ++p->c.foreground_refusals;
             return KVC_ERR_WOULD_BLOCK;
         }
+        p->by_key[key] = (uint32_t)take;  // first: if this allocation fails, the slot is still free
         PSlot &s = p->slots[take];
         s.state = IN_FLIGHT;
         s.key = key;
         s.refs = 1;
         s.speculative = !foreground;
         s.stamp = ++p->clock;
-        p->by_key[key] = (uint32_t)take;
         ++p->c.acquires;
         *slot = (uint32_t)take;
         *joined = 0;

@@ -154,23 +154,27 @@ uint64_t kvc_fnv1a64(const void *data, uint64_t n)
 
 kvc_status kvc_store_open(const char *root, const char *model_tag, int direct_io, kvc_store **out)
 {
-    if (!root || !model_tag || !out || !*root || !*model_tag || strchr(model_tag, '/'))
-        return KVC_ERR_INVALID_ARG;
-    *out = nullptr;
-    kvc_store *st = new (std::nothrow) kvc_store();
-    if (!st)
-        return KVC_ERR_NOMEM;
-    st->root = std::string(root) + "/" + model_tag;
-    st->want_direct = direct_io != 0;
-    st->direct_refused = 0;
-    st->seq = 0;
-    st->reads = st->read_bytes = st->publishes = st->publish_bytes = 0;
-    if (!mkdir_p(st->root)) {
-        delete st;
-        return KVC_ERR_IO;
+    try {
+        if (!root || !model_tag || !out || !*root || !*model_tag || strchr(model_tag, '/'))
+            return KVC_ERR_INVALID_ARG;
+        *out = nullptr;
+        kvc_store *st = new (std::nothrow) kvc_store();
+        if (!st)
+            return KVC_ERR_NOMEM;
+        st->root = std::string(root) + "/" + model_tag;
+        st->want_direct = direct_io != 0;
+        st->direct_refused = 0;
+        st->seq = 0;
+        st->reads = st->read_bytes = st->publishes = st->publish_bytes = 0;
+        if (!mkdir_p(st->root)) {
+            delete st;
+            return KVC_ERR_IO;
+        }
+        *out = st;
+        return KVC_OK;
+    } catch (const std::bad_alloc &) {
+        return KVC_ERR_NOMEM;  // path strings are the only allocations in here
     }
-    *out = st;
-    return KVC_OK;
 }
 
 kvc_status kvc_store_close(kvc_store *st)
@@ -183,93 +187,109 @@ kvc_status kvc_store_close(kvc_store *st)
 
 kvc_status kvc_store_path(const kvc_store *st, uint64_t hash, char *buf, uint32_t cap)
 {
-    if (!st || !buf)
-        return KVC_ERR_INVALID_ARG;
-    std::string p;
-    entry_path(st, hash, &p);
-    if (p.size() + 1 > cap)
-        return KVC_ERR_INVALID_ARG;
-    memcpy(buf, p.c_str(), p.size() + 1);
-    return KVC_OK;
+    try {
+        if (!st || !buf)
+            return KVC_ERR_INVALID_ARG;
+        std::string p;
+        entry_path(st, hash, &p);
+        if (p.size() + 1 > cap)
+            return KVC_ERR_INVALID_ARG;
+        memcpy(buf, p.c_str(), p.size() + 1);
+        return KVC_OK;
+    } catch (const std::bad_alloc &) {
+        return KVC_ERR_NOMEM;  // path strings are the only allocations in here
+    }
 }
 
 kvc_status kvc_store_lookup(const kvc_store *st, uint64_t hash, uint64_t *bytes)
 {
-    if (!st || !bytes)
-        return KVC_ERR_INVALID_ARG;
-    std::string p;
-    entry_path(st, hash, &p);
-    struct stat sb;
-    if (stat(p.c_str(), &sb) != 0) {
-        *bytes = 0;
-        return errno == ENOENT ? KVC_ERR_NOT_FOUND : KVC_ERR_IO;
+    try {
+        if (!st || !bytes)
+            return KVC_ERR_INVALID_ARG;
+        std::string p;
+        entry_path(st, hash, &p);
+        struct stat sb;
+        if (stat(p.c_str(), &sb) != 0) {
+            *bytes = 0;
+            return errno == ENOENT ? KVC_ERR_NOT_FOUND : KVC_ERR_IO;
+        }
+        *bytes = (uint64_t)sb.st_size;
+        return KVC_OK;
+    } catch (const std::bad_alloc &) {
+        return KVC_ERR_NOMEM;  // path strings are the only allocations in here
     }
-    *bytes = (uint64_t)sb.st_size;
-    return KVC_OK;
 }
 
 kvc_status kvc_store_publish(kvc_store *st, uint64_t hash, const void *host_buf, uint64_t bytes)
 {
-    if (!st || !host_buf || bytes == 0)
-        return KVC_ERR_INVALID_ARG;
-    std::string dir, final_path;
-    entry_dir(st, hash, &dir);
-    entry_path(st, hash, &final_path);
-    struct stat sb;
-    if (stat(final_path.c_str(), &sb) == 0)
-        return KVC_ERR_EXISTS;  // already published: nothing to write
-    if (!mkdir_p(dir))
-        return KVC_ERR_IO;
-    char tmp_name[96];
-    snprintf(tmp_name, sizeof(tmp_name), "/.tmp.%016llx.%ld.%llu", (unsigned long long)hash,
-             (long)getpid(), (unsigned long long)st->seq.fetch_add(1));
-    const std::string tmp = dir + tmp_name;
-    const bool direct = st->want_direct && direct_ok(host_buf, bytes);
-    int fd = open_maybe_direct(st, tmp.c_str(), O_WRONLY | O_CREAT | O_EXCL, 0666, direct);
-    if (fd < 0) {
-        unlink(tmp.c_str());  // a failed create may still have left the name behind
-        return KVC_ERR_IO;
+    try {
+        if (!st || !host_buf || bytes == 0)
+            return KVC_ERR_INVALID_ARG;
+        std::string dir, final_path;
+        entry_dir(st, hash, &dir);
+        entry_path(st, hash, &final_path);
+        struct stat sb;
+        if (stat(final_path.c_str(), &sb) == 0)
+            return KVC_ERR_EXISTS;  // already published: nothing to write
+        if (!mkdir_p(dir))
+            return KVC_ERR_IO;
+        char tmp_name[96];
+        snprintf(tmp_name, sizeof(tmp_name), "/.tmp.%016llx.%ld.%llu", (unsigned long long)hash,
+                 (long)getpid(), (unsigned long long)st->seq.fetch_add(1));
+        const std::string tmp = dir + tmp_name;
+        const bool direct = st->want_direct && direct_ok(host_buf, bytes);
+        int fd = open_maybe_direct(st, tmp.c_str(), O_WRONLY | O_CREAT | O_EXCL, 0666, direct);
+        if (fd < 0) {
+            unlink(tmp.c_str());  // a failed create may still have left the name behind
+            return KVC_ERR_IO;
+        }
+        kvc_status rc = write_all(fd, static_cast<const unsigned char *>(host_buf), bytes);
+        if (close(fd) != 0 && rc == KVC_OK)
+            rc = KVC_ERR_IO;
+        if (rc == KVC_OK) {
+            // atomic publication: the link fails if another writer got there first
+            if (link(tmp.c_str(), final_path.c_str()) != 0)
+                rc = errno == EEXIST ? KVC_ERR_EXISTS : KVC_ERR_IO;
+        }
+        unlink(tmp.c_str());
+        if (rc == KVC_OK) {
+            st->publishes.fetch_add(1);
+            st->publish_bytes.fetch_add(bytes);
+        }
+        return rc;
+    } catch (const std::bad_alloc &) {
+        return KVC_ERR_NOMEM;  // path strings are the only allocations in here
     }
-    kvc_status rc = write_all(fd, static_cast<const unsigned char *>(host_buf), bytes);
-    if (close(fd) != 0 && rc == KVC_OK)
-        rc = KVC_ERR_IO;
-    if (rc == KVC_OK) {
-        // atomic publication: the link fails if another writer got there first
-        if (link(tmp.c_str(), final_path.c_str()) != 0)
-            rc = errno == EEXIST ? KVC_ERR_EXISTS : KVC_ERR_IO;
-    }
-    unlink(tmp.c_str());
-    if (rc == KVC_OK) {
-        st->publishes.fetch_add(1);
-        st->publish_bytes.fetch_add(bytes);
-    }
-    return rc;
 }
 
 kvc_status kvc_store_read(kvc_store *st, uint64_t hash, void *host_buf, uint64_t bytes)
 {
-    if (!st || !host_buf || bytes == 0)
-        return KVC_ERR_INVALID_ARG;
-    std::string p;
-    entry_path(st, hash, &p);
-    const bool direct = st->want_direct && direct_ok(host_buf, bytes);
-    int fd = open_maybe_direct(st, p.c_str(), O_RDONLY, 0, direct);
-    if (fd < 0)
-        return errno == ENOENT ? KVC_ERR_NOT_FOUND : KVC_ERR_IO;
-    struct stat sb;
-    kvc_status rc = KVC_OK;
-    if (fstat(fd, &sb) != 0)
-        rc = KVC_ERR_IO;
-    else if ((uint64_t)sb.st_size != bytes)
-        rc = KVC_ERR_INVALID_ARG;  // the entry is not the size the caller's layout implies
-    else
-        rc = read_all(fd, static_cast<unsigned char *>(host_buf), bytes);
-    close(fd);
-    if (rc == KVC_OK) {
-        st->reads.fetch_add(1);
-        st->read_bytes.fetch_add(bytes);
+    try {
+        if (!st || !host_buf || bytes == 0)
+            return KVC_ERR_INVALID_ARG;
+        std::string p;
+        entry_path(st, hash, &p);
+        const bool direct = st->want_direct && direct_ok(host_buf, bytes);
+        int fd = open_maybe_direct(st, p.c_str(), O_RDONLY, 0, direct);
+        if (fd < 0)
+            return errno == ENOENT ? KVC_ERR_NOT_FOUND : KVC_ERR_IO;
+        struct stat sb;
+        kvc_status rc = KVC_OK;
+        if (fstat(fd, &sb) != 0)
+            rc = KVC_ERR_IO;
+        else if ((uint64_t)sb.st_size != bytes)
+            rc = KVC_ERR_INVALID_ARG;  // the entry is not the size the caller's layout implies
+        else
+            rc = read_all(fd, static_cast<unsigned char *>(host_buf), bytes);
+        close(fd);
+        if (rc == KVC_OK) {
+            st->reads.fetch_add(1);
+            st->read_bytes.fetch_add(bytes);
+        }
+        return rc;
+    } catch (const std::bad_alloc &) {
+        return KVC_ERR_NOMEM;  // path strings are the only allocations in here
     }
-    return rc;
 }
 
 int kvc_store_direct_io_refused(const kvc_store *st) { return st ? st->direct_refused.load() : 0; }
