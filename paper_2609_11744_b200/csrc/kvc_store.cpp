@@ -161,7 +161,12 @@ kvc_status kvc_store_open(const char *root, const char *model_tag, int direct_io
         kvc_store *st = new (std::nothrow) kvc_store();
         if (!st)
             return KVC_ERR_NOMEM;
-        st->root = std::string(root) + "/" + model_tag;
+        try {
+            st->root = std::string(root) + "/" + model_tag;
+        } catch (const std::bad_alloc &) {
+            delete st;
+            return KVC_ERR_NOMEM;
+        }
         st->want_direct = direct_io != 0;
         st->direct_refused = 0;
         st->seq = 0;
