@@ -399,9 +399,9 @@ def run_ours(args, rank, world, local_rank):
 
 
 def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, dist):
-    """Offload the prefix to pinned host memory and load it back, chunk by chunk through a
-    bounded ring of device staging slots (pack -> slot -> D2H; H2D -> slot -> unpack)."""
-    descs = kvc.kvc_map_request(lay, len(src))
+    """Offload the prefix to pinned host memory and load it back with the library's host-buffer
+    entry points: chunk by chunk through a bounded ring of device staging slots
+    (pack -> slot -> D2H; H2D -> slot -> unpack)."""
     cb = kvc.kvc_layout_chunk_bytes(lay, kvc.kvc_layout_blocks_per_chunk(lay))
     slot_bytes = (cb + 4095) // 4096 * 4096
     # Every rank pins a host buffer as large as the prefix.  If one of them cannot (N replicas share
@@ -428,26 +428,12 @@ def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, di
     TO = 10_000_000
 
     def offload():
-        off = 0
-        for (_, c, first, nb, nbytes) in descs:
-            slot, dptr, _ = kvc.kvc_staging_ring_acquire(ring, TO)
-            kvc.kvc_pack(lay, src[first:first + nb], dptr, nbytes, stream=s_k)
-            kvc.kvc_staging_ring_commit(ring, slot, s_k)
-            kvc.kvc_staging_ring_wait_filled(ring, slot, s_c)
-            cuda_rt.memcpy_async(hptr + off, dptr, nbytes, cuda_rt.D2H, s_c)
-            kvc.kvc_staging_ring_release(ring, slot, s_c)
-            off += nbytes
+        kvc.kvc_offload_to_host(lay, ring, src, hptr, host_bytes=one_way, kernel_stream=s_k,
+                                copy_stream=s_c, slot_timeout_us=TO)
 
     def load():
-        off = 0
-        for (_, c, first, nb, nbytes) in descs:
-            slot, dptr, _ = kvc.kvc_staging_ring_acquire(ring, TO)
-            cuda_rt.memcpy_async(dptr, hptr + off, nbytes, cuda_rt.H2D, s_c)
-            kvc.kvc_staging_ring_commit(ring, slot, s_c)
-            kvc.kvc_staging_ring_wait_filled(ring, slot, s_k)
-            kvc.kvc_unpack(lay, dptr, dst[first:first + nb], nbytes, stream=s_k)
-            kvc.kvc_staging_ring_release(ring, slot, s_k)
-            off += nbytes
+        kvc.kvc_load_from_host(lay, ring, hptr, dst, host_bytes=one_way, kernel_stream=s_k,
+                               copy_stream=s_c, slot_timeout_us=TO)
 
     offload()
     load()
@@ -477,8 +463,8 @@ def run_e2e(args, torch, kvc, cuda_rt, lay, s, src, dst, one_way, dev, world, di
         "offload_ms": statistics.mean(t_off) * 1e3, "load_ms": statistics.mean(t_load) * 1e3,
         "host_link_gbs_offload": one_way / statistics.mean(t_off) / 1e9,
         "host_link_gbs_load": one_way / statistics.mean(t_load) / 1e9,
-        "path": "kvc_pack -> %d-slot device ring -> cudaMemcpyAsync D2H to pinned host; "
-                "cudaMemcpyAsync H2D -> ring -> kvc_unpack" % args.ring_slots,
+        "path": "kvc_offload_to_host (kvc_pack -> %d-slot device ring -> copy engine to pinned host), then "
+                "kvc_load_from_host (copy engine -> ring -> kvc_unpack): one C call each way" % args.ring_slots,
         "ring_acquires": acquires, "ring_stalls": stalls,
     }
 

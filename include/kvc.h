@@ -121,6 +121,7 @@ uint64_t kvc_layout_bytes_per_token(const kvc_layout *layout);      /* Sec. 2.1 
 uint32_t kvc_layout_blocks_per_chunk(const kvc_layout *layout);     /* chunk_tokens / block_size */
 uint64_t kvc_layout_chunk_bytes(const kvc_layout *layout, uint32_t n_blocks); /* L*P*n*slab */
 uint32_t kvc_layout_num_chunks(const kvc_layout *layout, uint32_t n_blocks);  /* ceil(n / bpc) */
+uint32_t kvc_layout_num_blocks(const kvc_layout *layout);           /* blocks in the pool (NB) */
 
 /* How the copy kernels run (no counterpart in the paper: launch-shape knobs of this
  * implementation, used by its benchmarks and tests).  Zero in every field means "library default"
@@ -503,6 +504,43 @@ kvc_status kvc_pipeline_load(kvc_layout *layout, kvc_ring *ring, kvc_store *stor
  * again.  On any error exit every slot the call took is handed back: a slot whose copy was never
  * enqueued at once, the others after the copy or file operation in progress on them has ended;
  * queued file operations that had not started are dropped. */
+
+/* ------------------------------------------------------------------ to and from HOST memory (Sec. 5.1, 6.4) */
+
+/* A whole request between the paged pool and a HOST buffer, chunk by chunk through the ring: the
+ * GPU <-> CPU transfer of Sec. 5.1 at the granularity of the layout's chunk_tokens, through the
+ * bounded staging memory of Sec. 6.4, so the request may be far larger than the ring.
+ *   kvc_offload_to_host: for every chunk (kvc_map_request order) acquire a slot, kvc_pack the
+ *     chunk's blocks into it on `kernel_stream`, copy the slot to the host buffer on `copy_stream`
+ *     (which waits for the slot's "filled" event only), release the slot behind that copy.
+ *   kvc_load_from_host: the reverse -- host buffer -> slot on `copy_stream`, kvc_unpack into ids on
+ *     `kernel_stream`, release behind the kernel.
+ * The chunks lie back to back in the host buffer in request order (chunk c starts at the sum of
+ * the earlier chunks' bytes; the last may be short); host_bytes must cover them all.  The host
+ * buffer should be pinned: from pageable memory the runtime's copies stop being asynchronous.
+ * `ring`: a FIFO ring (KVC_ERR_STATE in pool mode) of any kind whose slots hold a full chunk; with
+ * KVC_RING_HOST_MAPPED the kernels cross the host link themselves and the copy is host to host.
+ * The two streams may be the same; different streams let one chunk's kernel run beside another
+ * chunk's copy.  ids is a HOST array and is validated as a whole before anything is enqueued
+ * (OUT_OF_RANGE; load: CONFLICT on a repeated id anywhere in the request).
+ * The calls block only while the ring is full (each wait for a slot is bounded by slot_timeout_us
+ * > 0: TIMEOUT) and return when the last chunk is ENQUEUED: synchronise `copy_stream` (offload) or
+ * `kernel_stream` (load) before using the result.  On an error exit nothing further is enqueued,
+ * every slot taken is handed back, and stats->chunks says how many chunks were enqueued in full.
+ * Not re-entrant on the same ring.
+ * Errors: INVALID_ARG, STATE, OUT_OF_RANGE, CONFLICT, TIMEOUT, NOMEM, CUDA. */
+typedef struct {
+    uint64_t bytes;        /* chunk bytes enqueued for transfer */
+    uint64_t ring_stalls;  /* polls that found the next slot still busy */
+    uint32_t chunks;       /* chunks enqueued in full */
+    uint32_t total_chunks; /* chunks of the request */
+} kvc_host_transfer_stats;
+kvc_status kvc_offload_to_host(kvc_layout *layout, kvc_ring *ring, const int32_t *ids, uint32_t n_blocks,
+                               void *host_dst, uint64_t host_bytes, void *kernel_stream, void *copy_stream,
+                               int64_t slot_timeout_us, kvc_host_transfer_stats *stats);
+kvc_status kvc_load_from_host(kvc_layout *layout, kvc_ring *ring, const void *host_src, uint64_t host_bytes,
+                              const int32_t *ids, uint32_t n_blocks, void *kernel_stream, void *copy_stream,
+                              int64_t slot_timeout_us, kvc_host_transfer_stats *stats);
 
 /* Several requests served at once from one staging pool (Sec. 6.4: every mapping that became ready
  * during one pass of the loop, from whichever request, goes into ONE fused unpack launch; Sec. 6.5:

@@ -6,7 +6,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(_HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(_HERE), "include")
 LIB = os.path.join(_HERE, "libkvc.so")
-SOURCES = ["kvc_kernels.cu", "kvc_layout.cu", "kvc_ring.cu", "kvc_noalloc.cu", "kvc_copy_engine.cu", "kvc_store.cpp", "kvc_pipeline.cpp", "kvc_slot_pool.cpp"]
+SOURCES = ["kvc_kernels.cu", "kvc_layout.cu", "kvc_ring.cu", "kvc_noalloc.cu", "kvc_copy_engine.cu", "kvc_store.cpp", "kvc_pipeline.cpp", "kvc_slot_pool.cpp",
+           "kvc_host_transfer.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-Wall", "-cudart", "static"]
 

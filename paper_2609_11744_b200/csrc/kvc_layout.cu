@@ -900,6 +900,7 @@ kvc_status kvc_poll_device_status(kvc_layout *lay, void *stream, uint32_t *n_ski
 }
 
 uint64_t kvc_layout_launch_count(const kvc_layout *lay) { return lay ? lay->launches : 0; }
+uint32_t kvc_layout_num_blocks(const kvc_layout *lay) { return lay ? lay->d.num_blocks : 0; }
 
 kvc_status kvc_layout_set_kernel_timing(kvc_layout *lay, int on)
 {

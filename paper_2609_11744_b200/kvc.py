@@ -66,6 +66,11 @@ class kvc_chunk_desc(ctypes.Structure):
                 ("bytes", ctypes.c_uint64)]
 
 
+class kvc_host_transfer_stats(ctypes.Structure):
+    _fields_ = [("bytes", ctypes.c_uint64), ("ring_stalls", ctypes.c_uint64), ("chunks", ctypes.c_uint32),
+                ("total_chunks", ctypes.c_uint32)]
+
+
 class kvc_pipeline_stats(ctypes.Structure):
     _fields_ = [("bytes", ctypes.c_uint64), ("seconds", ctypes.c_double), ("chunks", ctypes.c_uint32),
                 ("published", ctypes.c_uint32), ("already_present", ctypes.c_uint32),
@@ -141,6 +146,11 @@ def lib() -> ctypes.CDLL:
         "kvc_layout_blocks_per_chunk": (u32, [vp]),
         "kvc_layout_chunk_bytes": (u64, [vp, u32]),
         "kvc_layout_num_chunks": (u32, [vp, u32]),
+        "kvc_layout_num_blocks": (u32, [vp]),
+        "kvc_offload_to_host": (ci, [vp, vp, vp, u32, vp, u64, vp, vp, ctypes.c_int64,
+                                     P(kvc_host_transfer_stats)]),
+        "kvc_load_from_host": (ci, [vp, vp, vp, u64, vp, u32, vp, vp, ctypes.c_int64,
+                                    P(kvc_host_transfer_stats)]),
         "kvc_layout_set_tuning": (ci, [vp, P(kvc_tuning)]),
         "kvc_tuning_preset": (ci, [ci, P(kvc_tuning)]),
         "kvc_map_request": (ci, [vp, u32, u32, P(kvc_chunk_desc), u32, P(u32)]),
@@ -351,6 +361,10 @@ def kvc_layout_chunk_bytes(layout, n_blocks: int) -> int:
 
 def kvc_layout_num_chunks(layout, n_blocks: int) -> int:
     return lib().kvc_layout_num_chunks(layout.handle, n_blocks)
+
+
+def kvc_layout_num_blocks(layout) -> int:
+    return lib().kvc_layout_num_blocks(layout.handle)
 
 
 def kvc_layout_set_tuning(layout, variant=0, order=0, max_ctas=0, tile_bytes=0, stages=0,
@@ -726,6 +740,40 @@ def _pipeline(fn_name, layout, ring, store, ids, hashes, io_threads, use_copy_en
                                  ctypes.byref(stats))
     _check(st, fn_name)
     return {k: getattr(stats, k) for k, _ in kvc_pipeline_stats._fields_}
+
+
+def _host_transfer(fn_name: str, layout, ring, ids, host, host_bytes, kernel_stream, copy_stream,
+                   slot_timeout_us: int) -> dict:
+    keep, p, n, dev = _ids(ids)
+    if dev:
+        raise TypeError("the host transfers take host-resident ids")
+    nb = _nbytes(host) if host_bytes is None else host_bytes
+    ks = _stream(kernel_stream)
+    cs = ks if copy_stream is None else _stream(copy_stream)
+    stats = kvc_host_transfer_stats()
+    if fn_name == "kvc_offload_to_host":
+        st = lib().kvc_offload_to_host(layout.handle, ring.handle, p, n, _ptr(host), nb, ks, cs,
+                                       int(slot_timeout_us), ctypes.byref(stats))
+    else:
+        st = lib().kvc_load_from_host(layout.handle, ring.handle, _ptr(host), nb, p, n, ks, cs,
+                                      int(slot_timeout_us), ctypes.byref(stats))
+    _check(st, fn_name)
+    return {k: getattr(stats, k) for k, _ in kvc_host_transfer_stats._fields_}
+
+
+def kvc_offload_to_host(layout, ring, ids, host_dst, host_bytes: Optional[int] = None, kernel_stream=None,
+                        copy_stream=None, slot_timeout_us: int = 10_000_000) -> dict:
+    """Pack a request chunk by chunk through the ring into a (pinned) host buffer; returns the stats.
+    copy_stream None = the kernel stream.  Synchronise the copy stream before reading the buffer."""
+    return _host_transfer("kvc_offload_to_host", layout, ring, ids, host_dst, host_bytes, kernel_stream,
+                          copy_stream, slot_timeout_us)
+
+
+def kvc_load_from_host(layout, ring, host_src, ids, host_bytes: Optional[int] = None, kernel_stream=None,
+                       copy_stream=None, slot_timeout_us: int = 10_000_000) -> dict:
+    """The reverse: host buffer -> ring slots -> unpack into ids.  Synchronise the kernel stream."""
+    return _host_transfer("kvc_load_from_host", layout, ring, ids, host_src, host_bytes, kernel_stream,
+                          copy_stream, slot_timeout_us)
 
 
 def kvc_pipeline_store(layout, ring, store, ids, hashes, io_threads: int = 0,

@@ -594,6 +594,54 @@ def test_load_many_argument_checks_need_no_gpu(fake_events, tmp_path):
     kvc.kvc_store_close(store)
 
 
+def test_host_transfer_argument_checks_need_no_gpu(fake_events):
+    """What kvc_offload_to_host / kvc_load_from_host decide before anything is enqueued: FIFO ring
+    only, a positive slot timeout, a host buffer that covers every chunk, slots that hold a chunk,
+    and the WHOLE block table in range (load: without repeats, also across chunks)."""
+    lay = _layout(chunk_tokens=64, NB=64)
+    assert kvc.kvc_layout_num_blocks(lay) == 64
+    sb = kvc.kvc_layout_chunk_bytes(lay, 4)
+    mem = np.zeros(4 * sb + 64, dtype=np.uint8)
+    base = (mem.ctypes.data + 15) // 16 * 16
+    ring = kvc.kvc_staging_ring_create(sb, 4, kvc.KVC_RING_DEVICE, base, 4 * sb)
+    ids = np.arange(10, dtype=np.int32)
+    need = kvc.kvc_layout_chunk_bytes(lay, 10)
+    host = np.zeros(need, dtype=np.uint8)
+
+    def both(want, ids=ids, host=host, host_bytes=None, ring=ring, **kw):
+        for fn, args in ((kvc.kvc_offload_to_host, (lay, ring, ids, host)),
+                         (kvc.kvc_load_from_host, (lay, ring, host, ids))):
+            with pytest.raises(kvc.KvcError) as e:
+                fn(*args, host_bytes=host_bytes, kernel_stream=0, copy_stream=0, **kw)
+            assert e.value.status == want, fn.__name__
+
+    both(kvc.KVC_ERR_INVALID_ARG, host_bytes=need - 1)                    # buffer one byte short
+    both(kvc.KVC_ERR_INVALID_ARG, slot_timeout_us=0)                      # every wait must be bounded
+    bad = ids.copy()
+    bad[9] = 64
+    both(kvc.KVC_ERR_OUT_OF_RANGE, ids=bad)                               # last id of the last chunk
+    bad[9] = -1
+    both(kvc.KVC_ERR_OUT_OF_RANGE, ids=bad)
+    dup = ids.copy()
+    dup[9] = dup[0]                                                       # same block in chunks 0 and 2
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_load_from_host(lay, ring, host, dup, kernel_stream=0, copy_stream=0)
+    assert e.value.status == kvc.KVC_ERR_CONFLICT
+    small = kvc.kvc_staging_ring_create(4096, 4, kvc.KVC_RING_DEVICE, base, 4 * sb)
+    both(kvc.KVC_ERR_INVALID_ARG, ring=small)                             # a chunk does not fit a slot
+    kvc.kvc_staging_ring_destroy(small)
+    in_flight, acquires, _ = kvc.kvc_staging_ring_stats(ring)
+    assert (in_flight, acquires) == (0, 0)                                # nothing was taken
+    kvc.kvc_staging_ring_set_policy(ring, 1)
+    both(kvc.KVC_ERR_STATE)                                               # pool mode: slots are keyed by hash
+    # an empty request is a no-op
+    fifo = kvc.kvc_staging_ring_create(sb, 2, kvc.KVC_RING_DEVICE, base, 4 * sb)
+    st = kvc.kvc_offload_to_host(lay, fifo, ids[:0], host, kernel_stream=0, copy_stream=0)
+    assert (st["chunks"], st["total_chunks"], st["bytes"]) == (0, 0, 0)
+    kvc.kvc_staging_ring_destroy(fifo)
+    kvc.kvc_staging_ring_destroy(ring)
+
+
 def test_ring_create_validation(fake_events):
     for args, want in [((4096, 0, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),
                        ((0, 2, 0, 0x1000, 1 << 20), kvc.KVC_ERR_INVALID_ARG),

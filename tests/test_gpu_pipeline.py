@@ -258,3 +258,71 @@ def test_retained_chunks_serve_a_later_call_without_a_read(tmp_path):
     assert s3["reads"] >= 2                                          # evicted chunks are read again
     assert np.array_equal(pool_t.cpu().numpy(), want_pool)
     assert kvc.kvc_poll_device_status(lay) == (0, 0)
+
+
+# ------------------------------------------------------------------ request <-> host buffer, one call each way
+@pytest.mark.parametrize("ring_kind", [kvc.KVC_RING_DEVICE, kvc.KVC_RING_HOST_MAPPED, kvc.KVC_RING_DEVICE_STAGED])
+@pytest.mark.parametrize("two_streams", [False, True])
+def test_offload_to_host_and_load_back_match_the_oracle(ring_kind, two_streams):
+    """kvc_offload_to_host / kvc_load_from_host: 139 blocks (8 chunks of 16 and one of 11) through
+    a 3-slot ring into a pinned host buffer and back into other blocks, on one stream or on a kernel
+    stream and a copy stream; host bytes and the pool against the oracle, twice in a row (the
+    second pass reuses slots whose events the first pass recorded)."""
+    g = orc.Dims(6, 2, 200, 16, 8, 128, 2)
+    pool = wl.random_bits(760, g.pool_bytes)
+    pool_t = torch.from_numpy(pool).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 256)
+    src, dst = wl.block_ids(76, g.NB, 139), wl.block_ids(77, g.NB, 139)
+    cb = kvc.kvc_layout_chunk_bytes(lay, 16)
+    ring = kvc.kvc_staging_ring_create(cb, 3, ring_kind)
+    total = 139 * g.bytes_per_block
+    host = torch.full((total + 4096,), 0x5A, dtype=torch.uint8).pin_memory()
+    s_k = torch.cuda.Stream()
+    s_c = torch.cuda.Stream() if two_streams else None
+    want_chunks = orc.pack_request(g, pool, src, 256)
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, want_chunks, dst, 256)
+    for rep in range(2):
+        host.fill_(0x5A)
+        pool_t.copy_(torch.from_numpy(pool))
+        torch.cuda.synchronize()
+        st = kvc.kvc_offload_to_host(lay, ring, src, host, host_bytes=total, kernel_stream=s_k, copy_stream=s_c)
+        assert (st["chunks"], st["total_chunks"], st["bytes"]) == (9, 9, total)
+        (s_c or s_k).synchronize()
+        h = host.numpy()
+        assert np.array_equal(h[:total], np.concatenate(want_chunks)), "offload, pass %d" % rep
+        assert (h[total:] == 0x5A).all()
+        st = kvc.kvc_load_from_host(lay, ring, host, dst, host_bytes=total, kernel_stream=s_k, copy_stream=s_c)
+        assert (st["chunks"], st["bytes"]) == (9, total)
+        s_k.synchronize()
+        assert np.array_equal(pool_t.cpu().numpy(), want_pool), "load, pass %d" % rep
+    torch.cuda.synchronize()
+    in_flight, acquires, _ = kvc.kvc_staging_ring_stats(ring)
+    assert in_flight == 0 and acquires == 4 * 9
+    assert kvc.kvc_poll_device_status(lay) == (0, 0)
+    kvc.kvc_staging_ring_destroy(ring)
+
+
+def test_host_transfer_error_exit_leaves_the_ring_usable():
+    """A request whose last id is out of range is refused as a whole: nothing reaches the host
+    buffer, no slot is taken, and the next transfer through the same ring works."""
+    g = orc.Dims(2, 2, 64, 16, 4, 64, 2)
+    pool = wl.random_bits(770, g.pool_bytes)
+    pool_t = torch.from_numpy(pool).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 64)
+    ring = kvc.kvc_staging_ring_create(kvc.kvc_layout_chunk_bytes(lay, 4), 2, kvc.KVC_RING_DEVICE)
+    ids = wl.block_ids(78, g.NB, 30)
+    bad = ids.copy()
+    bad[-1] = g.NB
+    total = 30 * g.bytes_per_block
+    host = torch.full((total,), 0x11, dtype=torch.uint8).pin_memory()
+    with pytest.raises(kvc.KvcError) as e:
+        kvc.kvc_offload_to_host(lay, ring, bad, host)
+    assert e.value.status == kvc.KVC_ERR_OUT_OF_RANGE
+    torch.cuda.synchronize()
+    assert bool((host == 0x11).all())
+    assert kvc.kvc_staging_ring_stats(ring)[:2] == (0, 0)
+    kvc.kvc_offload_to_host(lay, ring, ids, host)
+    torch.cuda.synchronize()
+    assert np.array_equal(host.numpy(), np.concatenate(orc.pack_request(g, pool, ids, 64)))
+    kvc.kvc_staging_ring_destroy(ring)
