@@ -87,3 +87,28 @@ def test_layout_mapper_and_launch_front_ends_are_clean_under_asan_and_ubsan(tmp_
     assert build.returncode == 0, build.stderr
     run = subprocess.run([exe], capture_output=True, text=True, timeout=300)
     assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr[-3000:]
+
+
+@pytest.mark.skipif(shutil.which("g++") is None, reason="needs g++")
+def test_host_transfers_move_whole_requests_on_the_host_under_asan_and_ubsan(tmp_path):
+    """kvc_offload_to_host / kvc_load_from_host with the library's host code compiled as plain C++, the
+    CUDA runtime replaced by host stand-ins and the kernel launch by a loop over the slabs the launch
+    names: 120 random geometries, ring sizes and kinds; host images and pools checked byte for byte,
+    every buffer exactly as large as the interface requires."""
+    cuda_inc = os.path.join(os.environ.get("CUDA_HOME", "/usr/local/cuda"), "include")
+    if not os.path.isdir(cuda_inc):
+        pytest.skip("needs the CUDA toolkit headers")
+    csrc = os.path.join(ROOT, "paper_2609_11744_b200", "csrc")
+    exe = str(tmp_path / "host_transfer_san")
+    build = subprocess.run(
+        ["g++", "-O1", "-g", "-std=c++17", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
+         "-I", os.path.join(ROOT, "include"), "-I", csrc, "-I", cuda_inc,
+         "-x", "c++", os.path.join(csrc, "kvc_layout.cu"), os.path.join(csrc, "kvc_ring.cu"),
+         os.path.join(csrc, "kvc_slot_pool.cpp"), os.path.join(csrc, "kvc_host_transfer.cpp"),
+         os.path.join(ROOT, "tests", "native", "host_transfer_sanitizer_driver.cpp"), "-o", exe, "-lpthread"],
+        capture_output=True, text=True)
+    if build.returncode != 0 and "sanitize" in build.stderr:
+        pytest.skip("sanitizer runtime not installed")
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([exe], capture_output=True, text=True, timeout=300)
+    assert run.returncode == 0 and run.stdout.strip() == "ok", run.stdout + run.stderr[-3000:]
