@@ -521,7 +521,9 @@ kvc_status kvc_pipeline_load(kvc_layout *layout, kvc_ring *ring, kvc_store *stor
  * `ring`: a FIFO ring (KVC_ERR_STATE in pool mode) of any kind whose slots hold a full chunk; with
  * KVC_RING_HOST_MAPPED the kernels cross the host link themselves and the copy is host to host.
  * The two streams may be the same; different streams let one chunk's kernel run beside another
- * chunk's copy.  ids is a HOST array and is validated as a whole before anything is enqueued
+ * chunk's copy.  The transfer is bound by the host link either way, so while a model is running
+ * give the handle the KVC_PRESET_BESIDE_COMPUTE tuning: same link rate, a quarter of the cost to
+ * the model.  ids is a HOST array and is validated as a whole before anything is enqueued
  * (OUT_OF_RANGE; load: CONFLICT on a repeated id anywhere in the request).
  * The calls block only while the ring is full (each wait for a slot is bounded by slot_timeout_us
  * > 0: TIMEOUT) and return when the last chunk is ENQUEUED: synchronise `copy_stream` (offload) or
