@@ -1,5 +1,6 @@
 /* Plain C use of the library through its header: one pack and one unpack of a small request on
- * the current GPU, checked against a straightforward host loop.  Exit code 0 on success. */
+ * the current GPU, then the same request to a pinned host buffer and back through a two-slot ring
+ * in chunks of four blocks, all checked against a straightforward host loop.  Exit code 0 on success. */
 #include <cuda_runtime.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -52,6 +53,37 @@ int main(void)
         }
     uint32_t skipped = 9, expired = 9;
     CK(kvc_poll_device_status(lay, NULL, &skipped, &expired));
+    CK(kvc_layout_destroy(lay));
+
+    /* request <-> host buffer: chunks of 4 blocks (4 + 4 + 1) through a ring of two slots */
+    CK(kvc_layout_desc_init_dense(&desc, d_pool, L, P, NB, B, H, D, e, 4 * 16, KVC_CHUNK_LAYER_MAJOR));
+    CK(kvc_layout_create(&desc, &lay));
+    kvc_ring *ring = NULL;
+    CK(kvc_staging_ring_create(kvc_layout_chunk_bytes(lay, 4), 2, KVC_RING_DEVICE, NULL, 0, &ring));
+    unsigned char *h_req = NULL;
+    if (cudaMallocHost((void **)&h_req, cb) != cudaSuccess)
+        return 2;
+    cudaMemcpy(d_pool, h_pool, pool_bytes, cudaMemcpyHostToDevice);
+    kvc_host_transfer_stats ts;
+    CK(kvc_offload_to_host(lay, ring, ids, n, h_req, cb, NULL, NULL, 1000000, &ts));
+    cudaDeviceSynchronize();
+    bad |= ts.chunks != 3 || ts.bytes != cb;
+    size_t off = 0;
+    for (uint32_t first = 0; first < n; first += 4) {
+        const uint32_t nb = n - first < 4 ? n - first : 4;
+        for (uint32_t lp = 0; lp < L * P; ++lp)
+            for (uint32_t j = 0; j < nb; ++j)
+                bad |= memcmp(h_req + off + ((size_t)lp * nb + j) * slab,
+                              h_pool + lp * plane + ids[first + j] * slab, slab);
+        off += (size_t)L * P * nb * slab;
+    }
+    CK(kvc_load_from_host(lay, ring, h_req, cb, dst, n, NULL, NULL, 1000000, &ts));
+    cudaDeviceSynchronize();
+    cudaMemcpy(h_after, d_pool, pool_bytes, cudaMemcpyDeviceToHost);
+    for (uint32_t lp = 0; lp < L * P; ++lp)
+        for (uint32_t j = 0; j < n; ++j)
+            bad |= memcmp(h_after + lp * plane + dst[j] * slab, h_pool + lp * plane + ids[j] * slab, slab);
+    CK(kvc_staging_ring_destroy(ring));
     CK(kvc_layout_destroy(lay));
     printf(bad || skipped || expired ? "MISMATCH\n" : "ok\n");
     return bad || skipped || expired;

@@ -303,6 +303,28 @@ def test_offload_to_host_and_load_back_match_the_oracle(ring_kind, two_streams):
     kvc.kvc_staging_ring_destroy(ring)
 
 
+def test_host_transfers_accept_a_pageable_host_buffer():
+    """Pinned memory is a matter of speed, not of correctness: the same round trip through an
+    ordinary numpy array."""
+    g = orc.Dims(3, 2, 80, 16, 4, 64, 2)
+    pool = wl.random_bits(765, g.pool_bytes)
+    pool_t = torch.from_numpy(pool).to(DEV)
+    lay = kvc.kvc_layout_create_dense(pool_t, g.L, g.P, g.NB, g.B, g.H, g.D, g.e, 128)
+    ring = kvc.kvc_staging_ring_create(kvc.kvc_layout_chunk_bytes(lay, 8), 2, kvc.KVC_RING_DEVICE)
+    src, dst = wl.block_ids(79, g.NB, 53), wl.block_ids(80, g.NB, 53)
+    host = np.full(53 * g.bytes_per_block + 64, 0x42, dtype=np.uint8)
+    kvc.kvc_offload_to_host(lay, ring, src, host, host_bytes=53 * g.bytes_per_block)
+    torch.cuda.synchronize()
+    want_chunks = orc.pack_request(g, pool, src, 128)
+    assert np.array_equal(host[:-64], np.concatenate(want_chunks)) and (host[-64:] == 0x42).all()
+    kvc.kvc_load_from_host(lay, ring, host, dst, host_bytes=53 * g.bytes_per_block)
+    torch.cuda.synchronize()
+    want_pool = pool.copy()
+    orc.unpack_request(g, want_pool, want_chunks, dst, 128)
+    assert np.array_equal(pool_t.cpu().numpy(), want_pool)
+    kvc.kvc_staging_ring_destroy(ring)
+
+
 def test_host_transfer_error_exit_leaves_the_ring_usable():
     """A request whose last id is out of range is refused as a whole: nothing reaches the host
     buffer, no slot is taken, and the next transfer through the same ring works."""
