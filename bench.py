@@ -730,6 +730,26 @@ def suite_row_gather(torch, dev, reps):
             out.append(dict(row_bytes=S, rows=n, **best))
             del src, dst, idx
             torch.cuda.empty_cache()
+        # linear streams over 8 GiB for context: read only, write only, copy (bytes moved / time)
+        L.probe_stream.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_size_t, ctypes.c_int, ctypes.c_int,
+                                   ctypes.c_void_p, ctypes.c_void_p]
+        L.probe_stream.restype = ctypes.c_int
+        nbytes = 8 << 30
+        a = wl.random_bits_cuda(wl.BASE_SEED + 5, nbytes, dev)
+        b = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        sink = torch.zeros(1, dtype=torch.int32, device=dev)
+        streams = {}
+        for mode, name, moved in ((0, "read_only_gbs", nbytes), (1, "write_only_gbs", nbytes),
+                                  (2, "copy_gbs", 2 * nbytes)):
+            best = 0.0
+            for grid in (148 * 4, 148 * 8, 148 * 16, 148 * 32):
+                def run():
+                    rc = L.probe_stream(a.data_ptr(), b.data_ptr(), nbytes, mode, grid, sink.data_ptr(), st)
+                    assert rc == 0
+                _, med = _time_ms(torch, run, max(5, reps // 2))
+                best = max(best, moved / med / 1e6)
+            streams[name] = best
+        out.append({"linear_streams_8GiB": streams})
     return out
 
 

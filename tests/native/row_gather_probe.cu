@@ -56,3 +56,49 @@ extern "C" int probe_rows(const void *src, void *dst, const int *idx, int n_rows
                                                            row_bytes / 16, rows_per_warp, scatter);
     return (int)cudaGetLastError();
 }
+
+// Three linear streams over one large array, for context: how far is a copy from what the memory
+// does when it only reads, or only writes?  Every thread keeps U 16-byte accesses in flight.
+//   mode 0: read only (the values are folded into one word per thread, stored if it is ever zero
+//           so that the loads cannot be dropped);  mode 1: write only;  mode 2: copy src -> dst.
+template <int U>
+__global__ void __launch_bounds__(256)
+stream_kernel(const uint4 *__restrict__ src, uint4 *__restrict__ dst, size_t n_vec, int mode, uint32_t *sink)
+{
+    const size_t tid = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const size_t nthreads = (size_t)gridDim.x * blockDim.x;
+    uint32_t acc = 1;
+    for (size_t v0 = tid; v0 < n_vec; v0 += nthreads * U) {
+        uint4 r[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t v = v0 + (size_t)u * nthreads;
+            r[u] = make_uint4(1u, 2u, 3u, (uint32_t)v);
+            if (mode != 1 && v < n_vec)
+                asm volatile("ld.global.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                             : "=r"(r[u].x), "=r"(r[u].y), "=r"(r[u].z), "=r"(r[u].w)
+                             : "l"(src + v));
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const size_t v = v0 + (size_t)u * nthreads;
+            if (v >= n_vec)
+                continue;
+            if (mode == 0)
+                acc |= r[u].x ^ r[u].y ^ r[u].z ^ r[u].w;
+            else
+                asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(dst + v), "r"(r[u].x), "r"(r[u].y),
+                             "r"(r[u].z), "r"(r[u].w)
+                             : "memory");
+        }
+    }
+    if (acc == 0)
+        *sink = 0;
+}
+
+extern "C" int probe_stream(const void *src, void *dst, size_t bytes, int mode, int grid, void *sink, void *stream)
+{
+    stream_kernel<8><<<grid, 256, 0, (cudaStream_t)stream>>>((const uint4 *)src, (uint4 *)dst, bytes / 16, mode,
+                                                             (uint32_t *)sink);
+    return (int)cudaGetLastError();
+}
