@@ -246,11 +246,18 @@ def _nbytes(x) -> int:
     raise TypeError("need an explicit size for %r" % type(x))
 
 
+_torch_cuda = None  # torch.cuda once it is known to be initialised (per-chunk callers call this a lot)
+
+
 def _stream(s) -> int:
+    global _torch_cuda
     if s is None:
+        if _torch_cuda is not None:
+            return _torch_cuda.current_stream().cuda_stream
         try:
             import torch
             if torch.cuda.is_available() and torch.cuda.is_initialized():
+                _torch_cuda = torch.cuda
                 return int(torch.cuda.current_stream().cuda_stream)
         except ImportError:
             pass
@@ -263,6 +270,8 @@ def _stream(s) -> int:
 def _ids(ids) -> Tuple[object, int, int, int]:
     """(keep-alive object, address, count, on_device) of a block-id list.
     Host ids are converted to a contiguous int32 array; a CUDA tensor must already be int32."""
+    if type(ids) is np.ndarray and ids.dtype == np.int32 and ids.flags.c_contiguous:
+        return ids, ids.ctypes.data, ids.size, 0   # the common case, without a conversion
     if hasattr(ids, "data_ptr"):
         import torch
         if ids.is_cuda:
