@@ -107,10 +107,28 @@ class ClockSampler(threading.Thread):
             try:
                 sm = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
                 rs = int(reasons_fn(self.h))
-                self.samples.append((time.perf_counter(), float(sm), rs))
+                try:
+                    watts = nv.nvmlDeviceGetPowerUsage(self.h) / 1000.0
+                except Exception:
+                    watts = None
+                self.samples.append((time.perf_counter(), float(sm), rs, watts))
             except Exception:
                 pass
             time.sleep(0.01)
+
+    def window(self, t0: float, t1: float):
+        """Median SM clock, median board power and the reasons seen between two perf_counter times
+        (the sampler keeps running)."""
+        inside = [x for x in list(self.samples) if t0 <= x[0] <= t1]
+        if not inside:
+            return None
+        bits = 0
+        for x in inside:
+            bits |= x[2]
+        watts = [x[3] for x in inside if x[3] is not None]
+        return {"sm_mhz": statistics.median(x[1] for x in inside),
+                "watts": statistics.median(watts) if watts else None,
+                "reasons": sorted(v for k, v in self.REASONS.items() if bits & k), "samples": len(inside)}
 
     def summary(self, t0: float, t1: float):
         self._halt.set()
@@ -365,7 +383,8 @@ def run_ours(args, rank, world, local_rank):
                    "runs": [{"copy_blocks": "KVC_PRESET_BESIDE_COMPUTE" if r["tuning"].get("tile_bytes")
                              else "default", "direction": r["direction"],
                              "link_gbs_alone": r["link_gbs_alone"], "link_gbs_with_gemm": r["link_gbs_with_gemm"],
-                             "gemm_slowdown": r["gemm_slowdown"], "overlap_efficiency": r["overlap_efficiency"]}
+                             "gemm_slowdown": r["gemm_slowdown"], "overlap_efficiency": r["overlap_efficiency"],
+                             "clocks": r["clocks"]}
                             for r in ov["runs"]]}
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
@@ -832,6 +851,9 @@ def suite_batch(torch, kvc, dev, reps):
             "pack_ms_min": pm, "pack_ms_median": pd, "pack_gbs": 2 * total / pd / 1e6}
 
 
+_OVERLAP_SAMPLER = None  # a running ClockSampler while an overlap suite part is measured
+
+
 def _overlap_case(torch, fn, gemm_loop, s_gemm, s_k, s_c, iters, seconds, one_way, N, name,
                   direction, max_ctas):
     """Transfer alone, GEMM loop alone, both at once; see suite_ring_overlap."""
@@ -855,6 +877,7 @@ def _overlap_case(torch, fn, gemm_loop, s_gemm, s_k, s_c, iters, seconds, one_wa
     g1.record(s_gemm)
     torch.cuda.synchronize()
     t_gemm = time.perf_counter() - t0
+    w_gemm = (t0, t0 + t_gemm)
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     g0.record(s_gemm)
@@ -869,7 +892,12 @@ def _overlap_case(torch, fn, gemm_loop, s_gemm, s_k, s_c, iters, seconds, one_wa
     t_both = time.perf_counter() - t0
     t_gemm_in_both = g0.elapsed_time(g1) * 1e-3
     eff = 1 - (t_both - max(t_gemm, t_xfer)) / min(t_gemm, t_xfer)
-    return {"destination": name, "direction": direction, "max_ctas": max_ctas,
+    clocks = None
+    if _OVERLAP_SAMPLER is not None:
+        # the GPU's clock and power while the GEMM loop runs alone and while the transfer runs beside it
+        clocks = {"gemm_alone": _OVERLAP_SAMPLER.window(*w_gemm),
+                  "gemm_with_transfer": _OVERLAP_SAMPLER.window(t0, t0 + min(t_x_in_both, t_gemm_in_both))}
+    return {"clocks": clocks, "destination": name, "direction": direction, "max_ctas": max_ctas,
             "prefix_bytes": one_way, "passes": passes, "gemm_iters": iters,
             "once_ms": once * 1e3, "link_gbs_alone": passes * one_way / t_xfer / 1e9,
             "link_gbs_with_gemm": passes * one_way / t_x_in_both / 1e9,
@@ -981,6 +1009,9 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds, brief=False):
     per_iter = e0.elapsed_time(e1) / (2 * GRAPH_ITERS)
     iters = max(GRAPH_ITERS, int(seconds * 1e3 / per_iter) // GRAPH_ITERS * GRAPH_ITERS)
     results = []
+    global _OVERLAP_SAMPLER
+    _OVERLAP_SAMPLER = ClockSampler(torch, torch.cuda.current_device())
+    _OVERLAP_SAMPLER.start()
     # small shared-memory footprints (2 stages of 8 or 4 KiB per block) are there to see whether copy
     # blocks that fit beside a resident GEMM block disturb the GEMM less than 66 KB blocks do
     preset = {k: v for k, v in kvc.kvc_tuning_preset(kvc.KVC_PRESET_BESIDE_COMPUTE).items() if v}
@@ -1039,7 +1070,14 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds, brief=False):
                 results[-1]["tuning"] = tuning
             kvc.kvc_staging_ring_destroy(ring)
             kvc.kvc_layout_destroy(lay)
+    def stop_sampler():
+        global _OVERLAP_SAMPLER
+        _OVERLAP_SAMPLER._halt.set()
+        _OVERLAP_SAMPLER.join(timeout=2)
+        _OVERLAP_SAMPLER = None
+
     if brief:
+        stop_sampler()
         return {"gemm": "bf16 %dx%dx%d torch.matmul loop" % (N, N, N), "ms_per_gemm": per_iter,
                 "ring_slots": int(w.extra["ring_slots"]), "slot_bytes": cb, "prefix_bytes": one_way,
                 "seconds_per_phase": seconds, "runs": results}
@@ -1067,6 +1105,7 @@ def suite_ring_overlap(torch, kvc, cuda_rt, dev, seconds, brief=False):
         results.append(_overlap_case(torch, fn, gemm_loop, s_gemm, s_c, s_c, iters, seconds, one_way, N,
                                      "copy engines, pool <-> pinned host directly", direction, 0))
     kvc.kvc_layout_destroy(lay)
+    stop_sampler()
     return {"gemm": "bf16 %dx%dx%d torch.matmul loop" % (N, N, N), "ms_per_gemm": per_iter,
             "ring_slots": int(w.extra["ring_slots"]), "slot_bytes": cb, "runs": results}
 
